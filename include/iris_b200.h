@@ -1,0 +1,241 @@
+/*
+ * iris_b200.h -- C ABI of the B200 (sm_100a) implementation of the GEMM + all-scatter path of
+ * "Iris: First-Class Multi-GPU Programming Experience in Triton" (arXiv 2511.12500).
+ *
+ * The paper's W ranks are emulated as W equal partitions ("slots") of one allocation in a single
+ * GPU's HBM.  Slot r plays the role of rank r's symmetric heap: an object allocated at offset o
+ * exists at bases[r] + o in every slot (Section 3.1 "Adoption of Symmetric Heap Abstraction").
+ *
+ * Conventions
+ *   - Every function returns an int status (IRIS_OK == 0, errors negative) unless stated otherwise;
+ *     no exception crosses this boundary.  iris_last_error() gives a thread-local detail string.
+ *   - "device pointer" = address in the GPU's global memory; "host pointer" = ordinary CPU memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls that
+ *     take a stream only enqueue work; the caller synchronises.  Pointers are borrowed: they must
+ *     stay valid until the enqueued work has run.
+ *   - Argument errors are detected before anything is launched.  Problems that only the device
+ *     can see (a bounded wait that ran out) are recorded in the heap's status block and reported
+ *     by iris_status_check(); a kernel never traps and never spins without a deadline.
+ *   - The library is sm_100a only and has no CPU fallback: on a machine without such a GPU every
+ *     call that needs the device returns IRIS_ERR_CUDA.
+ */
+#ifndef IRIS_B200_H
+#define IRIS_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* ------------------------------------------------------------------------------------------ */
+/* Status codes, enumerations                                                                  */
+/* ------------------------------------------------------------------------------------------ */
+enum {
+  IRIS_OK = 0,
+  IRIS_ERR_ARG = -1,         /* bad argument value / alignment / divisibility                  */
+  IRIS_ERR_RANGE = -2,       /* an address or region leaves its rank's heap slot               */
+  IRIS_ERR_NOMEM = -3,       /* heap exhausted or device allocation failed                     */
+  IRIS_ERR_CUDA = -4,        /* a CUDA runtime/driver call failed (also: no usable GPU)        */
+  IRIS_ERR_UNSUPPORTED = -5, /* valid request that this build cannot serve                     */
+  IRIS_ERR_TIMEOUT = -6,     /* a device-side bounded wait expired (see iris_status_check)     */
+  IRIS_ERR_STATE = -7        /* heap used after destroy / inconsistent handle                  */
+};
+
+enum { IRIS_F16 = 0, IRIS_BF16 = 1 }; /* element type of A, B, C, bias (accumulation is fp32) */
+
+/* The three schedules of Section 4 ("Building Complex Multi-GPU Patterns"). */
+enum {
+  IRIS_MODE_BULK_SYNCHRONOUS = 0,     /* Listing 3: GEMM kernel, then an all-scatter kernel     */
+  IRIS_MODE_FUSED_SEQUENTIAL = 1,     /* Listing 4: each tile stored to all ranks from registers */
+  IRIS_MODE_WORKGROUP_SPECIALIZED = 2 /* Listing 5: producer CTAs + communication CTAs, locks   */
+};
+
+/* Memory order and scope of atomics (Table 3 note; Section 3.3 "Atomic Operations and Memory Model"). */
+enum { IRIS_SEM_RELAXED = 0, IRIS_SEM_ACQUIRE = 1, IRIS_SEM_RELEASE = 2, IRIS_SEM_ACQ_REL = 3 };
+enum { IRIS_SCOPE_BLOCK = 0, IRIS_SCOPE_GPU = 1, IRIS_SCOPE_SYS = 2 };
+
+#define IRIS_MAX_WORLD 8
+#define IRIS_TILE 128 /* publication tile edge: one ready flag per 128 x 128 block of C */
+
+typedef struct iris_heap iris_heap;
+
+const char* iris_last_error(void); /* never NULL; valid until the calling thread's next library call */
+const char* iris_version(void);
+
+/* ------------------------------------------------------------------------------------------ */
+/* Symmetric heap (Section 3.2 "Constructor and Initialization", steps 3 and 6)                */
+/* ------------------------------------------------------------------------------------------ */
+
+/* Create a heap of `world` slots of `bytes_per_rank` bytes each on the current CUDA device.
+ * 1 <= world <= IRIS_MAX_WORLD; bytes_per_rank > 0 and a multiple of 256.  The library allocates
+ * world * bytes_per_rank bytes of device memory (plus a 256-byte status block) and owns them.
+ * Returns NULL on failure (see iris_last_error). */
+iris_heap* iris_heap_create(int world, size_t bytes_per_rank);
+
+/* Same, with the status code returned and an optional caller-owned backing store:
+ * external_base != NULL must be a 256-byte aligned device pointer to world * bytes_per_rank bytes
+ * that outlives the heap (e.g. a torch tensor's storage); NULL = the library allocates. */
+int iris_heap_create_ex(int world, size_t bytes_per_rank, void* external_base, iris_heap** out);
+
+/* Free the heap (and its memory if the library owns it).  Synchronises the device first. */
+int iris_heap_destroy(iris_heap* heap);
+
+int iris_heap_world(const iris_heap* heap);                /* get_num_ranks(); <0 on bad handle */
+size_t iris_heap_bytes_per_rank(const iris_heap* heap);    /* 0 on bad handle                   */
+void* iris_heap_base(const iris_heap* heap, int rank);     /* device pointer; NULL on bad rank  */
+/* get_heap_bases(): writes `world` device addresses into the host array out[]. */
+int iris_heap_bases(const iris_heap* heap, uint64_t* out);
+
+/* Symmetric bump allocation: reserves `bytes` at one offset that is valid in every slot.
+ * align: power of two >= 16 (0 = 256).  There is no per-object free; iris_heap_reset() releases
+ * everything.  IRIS_ERR_NOMEM when the slot is exhausted.  offset_out: host pointer. */
+int iris_malloc(iris_heap* heap, size_t bytes, size_t align, uint64_t* offset_out);
+int iris_heap_reset(iris_heap* heap);
+
+/* Pointer translation (Listing 1, Section 3.3): *out = base[to_rank] + (ptr - base[from_rank]).
+ * `ptr` is a device address that is valid in from_rank's slot.  IRIS_ERR_RANGE if it is not inside
+ * [base[from_rank], base[from_rank] + bytes_per_rank); IRIS_ERR_ARG for a bad rank.  Pure host
+ * arithmetic; the kernels use the same formula on a by-value copy of the base table. */
+int iris_translate(const iris_heap* heap, const void* ptr, int from_rank, int to_rank, void** out);
+
+/* ------------------------------------------------------------------------------------------ */
+/* Device-detected errors                                                                      */
+/* ------------------------------------------------------------------------------------------ */
+
+/* Synchronise `stream`, read the heap's status block and clear it.  Returns IRIS_OK, or
+ * IRIS_ERR_TIMEOUT when a kernel gave up a bounded wait (detail[0..7], if not NULL, receives
+ * {code, kernel id, block, tile, slot, value seen, value expected, 0} on the host). */
+int iris_status_check(iris_heap* heap, void* stream, int32_t* detail);
+
+/* ------------------------------------------------------------------------------------------ */
+/* Tile memory operations and atomics on heap addresses (Table 3)                              */
+/* ------------------------------------------------------------------------------------------ */
+
+/* put: copy a 2-D region from from_rank's memory to to_rank's memory (local -> remote).
+ * src and dst are device addresses valid in from_rank's slot, exactly as in Listings 3 and 5
+ * (iris.put(C + offset, C + offset, cur_rank, remote_rank)): the region is read at src and
+ * written at translate(dst, from_rank, to_rank).  rows x row_bytes bytes; consecutive rows are
+ * src_pitch / dst_pitch bytes apart (pitch >= row_bytes).  A 16-byte vector path is used when
+ * both addresses, both pitches and row_bytes are multiples of 16, a byte path otherwise.
+ * IRIS_ERR_RANGE if either region leaves its slot.  rows == 0 or row_bytes == 0: no-op. */
+int iris_put_tile(iris_heap* heap, const void* src, void* dst, size_t rows, size_t row_bytes, size_t src_pitch,
+                  size_t dst_pitch, int from_rank, int to_rank, void* stream);
+
+/* get: the mirror image (remote -> local): read translate(src, from_rank, to_rank), write dst
+ * in from_rank's slot. */
+int iris_get_tile(iris_heap* heap, const void* src, void* dst, size_t rows, size_t row_bytes, size_t src_pitch,
+                  size_t dst_pitch, int from_rank, int to_rank, void* stream);
+
+/* atomic_add / atomic_cas on int32 words of to_rank's memory.  `ptr` is valid in from_rank's slot
+ * and is translated first.  Vector form: `count` words, `stride_bytes` apart (multiple of 4), one
+ * GPU thread per word; old_out (device pointer to count int32, or NULL) receives the previous
+ * values.  sem / scope select the PTX qualifiers (.relaxed/.acquire/.release/.acq_rel,
+ * .cta/.gpu/.sys). */
+int iris_atomic_add(iris_heap* heap, void* ptr, size_t count, size_t stride_bytes, int from_rank, int to_rank,
+                    int32_t value, int sem, int scope, int32_t* old_out, void* stream);
+int iris_atomic_cas(iris_heap* heap, void* ptr, size_t count, size_t stride_bytes, int from_rank, int to_rank,
+                    int32_t compare, int32_t value, int sem, int scope, int32_t* old_out, void* stream);
+
+/* Contended forms used by the protocol tests and the atomics microbenchmark: `threads` GPU
+ * threads all operate on the SAME word.  add: each adds `value`; cas: thread i tries
+ * compare -> value_base + i.  old_out: device pointer to `threads` int32 (or NULL). */
+int iris_atomic_add_contended(iris_heap* heap, void* ptr, size_t threads, int from_rank, int to_rank, int32_t value,
+                              int sem, int scope, int32_t* old_out, void* stream);
+int iris_atomic_cas_contended(iris_heap* heap, void* ptr, size_t threads, int from_rank, int to_rank,
+                              int32_t compare, int32_t value_base, int sem, int scope, int32_t* old_out,
+                              void* stream);
+
+/* Set `count` int32 words at heap offset `off` to `value` in every slot (flag / lock set-up). */
+int iris_flags_fill(iris_heap* heap, uint64_t off, size_t count, int32_t value, void* stream);
+
+/* All-store microbenchmark (Section 5.1, "all-store"): every rank r copies its block of S bytes
+ * (at payload_off in its own slot) into every slot s at recv_off + r*S, in tiles of tile_bytes
+ * (multiple of 16, <= 32768; the last tile of a block may be short), and after each tile's bytes
+ * sets flag[s][r*T + i] with atomic_cas(epoch-1 -> epoch, release, gpu), T = ceil(S/tile_bytes).
+ * S must be a multiple of 16.  ctas: grid size (0 = 8 per SM).  Reads W*S, writes W*W*S bytes.
+ * pull != 0 runs the all-load form instead: every rank s fetches (get) block r from rank r's
+ * slot into its own recv area; same end state. */
+int iris_all_store_bench(iris_heap* heap, uint64_t payload_off, uint64_t recv_off, uint64_t flag_off, size_t S,
+                         size_t tile_bytes, int32_t epoch, int ctas, int pull, void* stream);
+
+/* ------------------------------------------------------------------------------------------ */
+/* GEMM + all-scatter (Section 4, Listings 2-5)                                                */
+/* ------------------------------------------------------------------------------------------ */
+
+/* C = A . [B_0 | B_1 | ... | B_{W-1}] with fp32 accumulation, rounded once to the element type;
+ * rank r owns columns [r*N/W, (r+1)*N/W).  Each finished tile is stored into EVERY rank's slot at
+ * the tile's global offset (Listing 4: offset = rm*ldc + rn + cur_rank*N_local), and for each
+ * 128 x 128 publication tile t and each slot s the int32 ready flag flag[s][t] is then written
+ * with release semantics at gpu scope.
+ *
+ * Publication tiles are counted per rank shard so that none straddles two ranks:
+ *   TM = ceil(M/128), TNl = ceil((N/W)/128), t = tm*(W*TNl) + r*TNl + j.
+ *
+ * Layout in every slot: C row-major [M, N] (ldc = N) at c_off; int32 flag[TM*W*TNl] at flag_off;
+ * int32 lock[TM*W*TNl] at lock_off (workgroup-specialised mode only; lock t is used in the slot of
+ * the rank owning tile t, must be 0 before the call and is 0 again afterwards: Listing 5's
+ * cas(0->1, release) by the producer and cas(1->0, acquire) by the communication CTA).
+ */
+typedef struct iris_gemm_args {
+  const void* A;               /* device: [M, K] row-major, K contiguous, 16-byte aligned        */
+  const void* const* B_shards; /* HOST array of `world` DEVICE pointers; shard r is [N/W, K] with
+                                  K contiguous (= the K x N_local operand of Listing 2 stored
+                                  column-major), 16-byte aligned                                 */
+  iris_heap* heap;
+  int M, N, K;                 /* N = global width; N % world == 0, (N/world) % 8 == 0, K % 8 == 0;
+                                  M, N, K >= 0 (an empty problem publishes nothing and succeeds) */
+  int world;                   /* must equal the heap's world                                    */
+  int mode;                    /* IRIS_MODE_*                                                    */
+  int dtype;                   /* IRIS_F16 or IRIS_BF16                                          */
+  uint64_t c_off, flag_off, lock_off; /* offsets inside a slot; c_off % 256 == 0, others % 4     */
+  int32_t epoch;               /* value written to the flags; callers use 1, 2, 3, ...           */
+  int comm_ctas;               /* workgroup-specialised: communication CTAs (0 = 8)              */
+  int max_ctas;                /* cap on the persistent grid (0 = one CTA per SM)                */
+  int raster_group;            /* tile rows per raster group for L2 reuse (0 = 16)               */
+  int block_n;                 /* compute-tile width: 0 = auto, 128 or 256                       */
+  uint64_t spin_timeout_ns;    /* deadline of every device-side wait (0 = 2 s)                   */
+} iris_gemm_args;
+
+/* Enqueue the whole operation on `stream` (bulk-synchronous: two kernels; otherwise one).
+ * IRIS_ERR_ARG / IRIS_ERR_RANGE / IRIS_ERR_UNSUPPORTED are returned before any launch. */
+int iris_gemm_all_scatter_ex(const iris_gemm_args* args, void* stream);
+
+/* The short form named by the problem statement.  bf16; C at offset 0 of every slot, flags at
+ * align256(M*N*2), locks right after the flags (align256); epoch = a per-heap counter that starts
+ * at 1 and grows by one per call (iris_heap_epoch() returns the last value used); default stream.
+ * The heap must have been created with bytes_per_rank >= iris_gemm_heap_bytes(M, N, world). */
+int gemm_all_scatter(const void* A, const void* const* B_shards, iris_heap* heap, int M, int N, int K, int world,
+                     int mode);
+size_t iris_gemm_heap_bytes(int M, int N, int world);
+int32_t iris_heap_epoch(const iris_heap* heap);
+/* Number of publication tiles TM*W*TNl (0 for an empty problem, <0 on bad arguments). */
+int64_t iris_num_tiles(int M, int N, int world);
+
+/* Flag-gated consumer (Section 4.1, producer-consumer: the consumer side).  For every slot s and
+ * publication tile t: wait (acquire, gpu scope, bounded by timeout_ns, 0 = 2 s) until
+ * flag[s][t] >= epoch, then OUT[s] = C[s] + bias on that tile; bias: device pointer to N elements
+ * of `dtype`, broadcast over rows; the sum is formed in fp32 and rounded once.  OUT is a second
+ * row-major [M, N] region at out_off in every slot.  ctas: grid size (0 = 8 per SM). */
+int iris_consume_bias(iris_heap* heap, uint64_t c_off, uint64_t out_off, uint64_t flag_off, const void* bias, int M,
+                      int N, int world, int dtype, int32_t epoch, int ctas, uint64_t timeout_ns, void* stream);
+
+/* End-to-end form with HOST buffers: copies A and the W shards (and bias, if given) to device staging
+ * owned by the heap (allocated on first use, reused afterwards), runs gemm_all_scatter in `mode` with
+ * the short form's layout, then -- when bias_host != NULL -- the flag-gated consumer with OUT at
+ * iris_gemm_out_offset(M, N, world); copies slot `out_slot`'s C ([M, N], to C_host), its OUT (to
+ * OUT_host; bias_host and OUT_host are both NULL or both non-NULL) and the flags of all slots
+ * (world * iris_num_tiles int32, slot-major, to flags_host; may be NULL) back, and returns after
+ * everything has completed.  Runs on the legacy default stream.  Host buffers should be pinned for
+ * full copy speed.  With a bias the heap needs bytes_per_rank >= iris_gemm_out_offset + M*N*2. */
+int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_host, void* C_host,
+                               int32_t* flags_host, const void* bias_host, void* OUT_host, iris_heap* heap,
+                               int M, int N, int K, int world, int mode, int dtype, int out_slot);
+/* Offset of OUT in the short form's layout: right after the lock array (256-byte aligned). */
+uint64_t iris_gemm_out_offset(int M, int N, int world);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IRIS_B200_H */

@@ -1,0 +1,278 @@
+"""Thin ctypes binding of libiris_b200.so: same names as include/iris_b200.h, argument marshalling only.
+
+PyTorch appears here only to obtain device pointers and the current stream.  There is no fallback:
+if the shared library is missing or cannot be loaded, importing a symbol raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+IRIS_OK = 0
+IRIS_ERR_ARG, IRIS_ERR_RANGE, IRIS_ERR_NOMEM, IRIS_ERR_CUDA = -1, -2, -3, -4
+IRIS_ERR_UNSUPPORTED, IRIS_ERR_TIMEOUT, IRIS_ERR_STATE = -5, -6, -7
+IRIS_F16, IRIS_BF16 = 0, 1
+DTYPES = {"fp16": IRIS_F16, "bf16": IRIS_BF16}
+IRIS_MODE_BULK_SYNCHRONOUS, IRIS_MODE_FUSED_SEQUENTIAL, IRIS_MODE_WORKGROUP_SPECIALIZED = 0, 1, 2
+MODES = {"bulk_synchronous": 0, "fused_sequential": 1, "workgroup_specialized": 2}
+IRIS_SEM_RELAXED, IRIS_SEM_ACQUIRE, IRIS_SEM_RELEASE, IRIS_SEM_ACQ_REL = 0, 1, 2, 3
+IRIS_SCOPE_BLOCK, IRIS_SCOPE_GPU, IRIS_SCOPE_SYS = 0, 1, 2
+IRIS_MAX_WORLD = 8
+IRIS_TILE = 128
+
+LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "lib", "libiris_b200.so")
+
+# Every symbol include/iris_b200.h declares.
+EXPORTS = [
+    "iris_last_error", "iris_version", "iris_heap_create", "iris_heap_create_ex", "iris_heap_destroy", "iris_heap_world",
+    "iris_heap_bytes_per_rank", "iris_heap_base", "iris_heap_bases", "iris_malloc", "iris_heap_reset", "iris_translate",
+    "iris_status_check", "iris_put_tile", "iris_get_tile", "iris_atomic_add", "iris_atomic_cas",
+    "iris_atomic_add_contended", "iris_atomic_cas_contended", "iris_flags_fill", "iris_all_store_bench",
+    "iris_gemm_all_scatter_ex", "gemm_all_scatter", "iris_gemm_heap_bytes", "iris_heap_epoch", "iris_num_tiles",
+    "iris_consume_bias", "iris_gemm_all_scatter_host", "iris_gemm_out_offset",
+]
+
+
+class IrisError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"iris error {code}: {msg}")
+        self.code = code
+
+
+class GemmArgs(C.Structure):
+    _fields_ = [
+        ("A", C.c_void_p), ("B_shards", C.POINTER(C.c_void_p)), ("heap", C.c_void_p),
+        ("M", C.c_int), ("N", C.c_int), ("K", C.c_int), ("world", C.c_int), ("mode", C.c_int), ("dtype", C.c_int),
+        ("c_off", C.c_uint64), ("flag_off", C.c_uint64), ("lock_off", C.c_uint64),
+        ("epoch", C.c_int32), ("comm_ctas", C.c_int), ("max_ctas", C.c_int), ("raster_group", C.c_int),
+        ("block_n", C.c_int), ("spin_timeout_ns", C.c_uint64),
+    ]
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load the library (no CUDA call is made by loading it)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2511_12500_b200.build` (needs nvcc); there is no fallback")
+    L = C.CDLL(LIB_PATH)
+    vp, u64, sz, i32, ci = C.c_void_p, C.c_uint64, C.c_size_t, C.c_int32, C.c_int
+    L.iris_last_error.restype = C.c_char_p
+    L.iris_version.restype = C.c_char_p
+    L.iris_heap_create.restype = vp
+    L.iris_heap_create.argtypes = [ci, sz]
+    L.iris_heap_create_ex.argtypes = [ci, sz, vp, C.POINTER(vp)]
+    L.iris_heap_destroy.argtypes = [vp]
+    L.iris_heap_world.argtypes = [vp]
+    L.iris_heap_bytes_per_rank.restype = sz
+    L.iris_heap_bytes_per_rank.argtypes = [vp]
+    L.iris_heap_base.restype = vp
+    L.iris_heap_base.argtypes = [vp, ci]
+    L.iris_heap_bases.argtypes = [vp, C.POINTER(u64)]
+    L.iris_malloc.argtypes = [vp, sz, sz, C.POINTER(u64)]
+    L.iris_heap_reset.argtypes = [vp]
+    L.iris_translate.argtypes = [vp, vp, ci, ci, C.POINTER(vp)]
+    L.iris_status_check.argtypes = [vp, vp, C.POINTER(i32)]
+    for f in (L.iris_put_tile, L.iris_get_tile):
+        f.argtypes = [vp, vp, vp, sz, sz, sz, sz, ci, ci, vp]
+    L.iris_atomic_add.argtypes = [vp, vp, sz, sz, ci, ci, i32, ci, ci, vp, vp]
+    L.iris_atomic_cas.argtypes = [vp, vp, sz, sz, ci, ci, i32, i32, ci, ci, vp, vp]
+    L.iris_atomic_add_contended.argtypes = [vp, vp, sz, ci, ci, i32, ci, ci, vp, vp]
+    L.iris_atomic_cas_contended.argtypes = [vp, vp, sz, ci, ci, i32, i32, ci, ci, vp, vp]
+    L.iris_flags_fill.argtypes = [vp, u64, sz, i32, vp]
+    L.iris_all_store_bench.argtypes = [vp, u64, u64, u64, sz, sz, i32, ci, ci, vp]
+    L.iris_gemm_all_scatter_ex.argtypes = [C.POINTER(GemmArgs), vp]
+    L.gemm_all_scatter.argtypes = [vp, C.POINTER(vp), vp, ci, ci, ci, ci, ci]
+    L.iris_gemm_heap_bytes.restype = sz
+    L.iris_gemm_heap_bytes.argtypes = [ci, ci, ci]
+    L.iris_heap_epoch.restype = i32
+    L.iris_heap_epoch.argtypes = [vp]
+    L.iris_num_tiles.restype = C.c_int64
+    L.iris_num_tiles.argtypes = [ci, ci, ci]
+    L.iris_consume_bias.argtypes = [vp, u64, u64, u64, vp, ci, ci, ci, ci, i32, ci, u64, vp]
+    L.iris_gemm_all_scatter_host.argtypes = [vp, C.POINTER(vp), vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci]
+    L.iris_gemm_out_offset.restype = u64
+    L.iris_gemm_out_offset.argtypes = [ci, ci, ci]
+    _lib = L
+    return L
+
+
+def iris_last_error() -> str:
+    return lib().iris_last_error().decode()
+
+
+def _ck(rc: int) -> int:
+    if rc != IRIS_OK:
+        raise IrisError(rc, iris_last_error())
+    return rc
+
+
+def _ptr(x) -> int | None:
+    """Device/host address of a torch tensor, numpy array, int or None."""
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    if hasattr(x, "ctypes"):
+        return x.ctypes.data
+    raise TypeError(type(x))
+
+
+def _stream(stream) -> int | None:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream or None
+    return stream.cuda_stream
+
+
+# ---------------------------------------------------------------------------------------------- heap
+def iris_heap_create(world: int, bytes_per_rank: int, external_base=None) -> int:
+    h = C.c_void_p()
+    _ck(lib().iris_heap_create_ex(world, bytes_per_rank, _ptr(external_base), C.byref(h)))
+    return h.value
+
+
+def iris_heap_destroy(heap: int):
+    _ck(lib().iris_heap_destroy(heap))
+
+
+def iris_heap_world(heap: int) -> int:
+    return lib().iris_heap_world(heap)
+
+
+def iris_heap_bytes_per_rank(heap: int) -> int:
+    return lib().iris_heap_bytes_per_rank(heap)
+
+
+def iris_heap_base(heap: int, rank: int) -> int:
+    p = lib().iris_heap_base(heap, rank)
+    if not p:
+        raise IrisError(IRIS_ERR_ARG, iris_last_error())
+    return p
+
+
+def iris_heap_bases(heap: int) -> list[int]:
+    out = (C.c_uint64 * IRIS_MAX_WORLD)()
+    _ck(lib().iris_heap_bases(heap, out))
+    return list(out[: iris_heap_world(heap)])
+
+
+def iris_malloc(heap: int, nbytes: int, align: int = 0) -> int:
+    off = C.c_uint64()
+    _ck(lib().iris_malloc(heap, nbytes, align, C.byref(off)))
+    return off.value
+
+
+def iris_heap_reset(heap: int):
+    _ck(lib().iris_heap_reset(heap))
+
+
+def iris_translate(heap: int, ptr: int, from_rank: int, to_rank: int) -> int:
+    out = C.c_void_p()
+    _ck(lib().iris_translate(heap, ptr, from_rank, to_rank, C.byref(out)))
+    return out.value
+
+
+def iris_status_check(heap: int, stream=None):
+    """Synchronise and raise IrisError(IRIS_ERR_TIMEOUT) if a device-side wait expired."""
+    detail = (C.c_int32 * 8)()
+    rc = lib().iris_status_check(heap, _stream(stream), detail)
+    if rc != IRIS_OK:
+        e = IrisError(rc, iris_last_error())
+        e.detail = list(detail)
+        raise e
+
+
+# ---------------------------------------------------------------------------------------- tile ops
+def iris_put_tile(heap, src, dst, rows, row_bytes, src_pitch, dst_pitch, from_rank, to_rank, stream=None):
+    _ck(lib().iris_put_tile(heap, src, dst, rows, row_bytes, src_pitch, dst_pitch, from_rank, to_rank, _stream(stream)))
+
+
+def iris_get_tile(heap, src, dst, rows, row_bytes, src_pitch, dst_pitch, from_rank, to_rank, stream=None):
+    _ck(lib().iris_get_tile(heap, src, dst, rows, row_bytes, src_pitch, dst_pitch, from_rank, to_rank, _stream(stream)))
+
+
+def iris_atomic_add(heap, ptr, count, stride_bytes, from_rank, to_rank, value, sem=IRIS_SEM_RELAXED,
+                    scope=IRIS_SCOPE_GPU, old_out=None, stream=None):
+    _ck(lib().iris_atomic_add(heap, ptr, count, stride_bytes, from_rank, to_rank, value, sem, scope, _ptr(old_out), _stream(stream)))
+
+
+def iris_atomic_cas(heap, ptr, count, stride_bytes, from_rank, to_rank, compare, value, sem=IRIS_SEM_RELAXED,
+                    scope=IRIS_SCOPE_GPU, old_out=None, stream=None):
+    _ck(lib().iris_atomic_cas(heap, ptr, count, stride_bytes, from_rank, to_rank, compare, value, sem, scope, _ptr(old_out), _stream(stream)))
+
+
+def iris_atomic_add_contended(heap, ptr, threads, from_rank, to_rank, value, sem=IRIS_SEM_RELAXED, scope=IRIS_SCOPE_GPU,
+                              old_out=None, stream=None):
+    _ck(lib().iris_atomic_add_contended(heap, ptr, threads, from_rank, to_rank, value, sem, scope, _ptr(old_out), _stream(stream)))
+
+
+def iris_atomic_cas_contended(heap, ptr, threads, from_rank, to_rank, compare, value_base, sem=IRIS_SEM_RELAXED,
+                              scope=IRIS_SCOPE_GPU, old_out=None, stream=None):
+    _ck(lib().iris_atomic_cas_contended(heap, ptr, threads, from_rank, to_rank, compare, value_base, sem, scope, _ptr(old_out), _stream(stream)))
+
+
+def iris_flags_fill(heap, off, count, value, stream=None):
+    _ck(lib().iris_flags_fill(heap, off, count, value, _stream(stream)))
+
+
+def iris_all_store_bench(heap, payload_off, recv_off, flag_off, S, tile_bytes, epoch, ctas=0, pull=0, stream=None):
+    _ck(lib().iris_all_store_bench(heap, payload_off, recv_off, flag_off, S, tile_bytes, epoch, ctas, pull, _stream(stream)))
+
+
+# ------------------------------------------------------------------------------- GEMM + all-scatter
+def iris_num_tiles(M: int, N: int, world: int) -> int:
+    n = lib().iris_num_tiles(M, N, world)
+    if n < 0:
+        raise IrisError(int(n), iris_last_error())
+    return int(n)
+
+
+def iris_gemm_heap_bytes(M: int, N: int, world: int) -> int:
+    return lib().iris_gemm_heap_bytes(M, N, world)
+
+
+def iris_heap_epoch(heap: int) -> int:
+    return lib().iris_heap_epoch(heap)
+
+
+def _shards(B_shards):
+    arr = (C.c_void_p * len(B_shards))(*[_ptr(b) for b in B_shards])
+    return arr
+
+
+def iris_gemm_all_scatter_ex(heap, A, B_shards, M, N, K, world, mode, dtype, c_off, flag_off, lock_off=0, epoch=1,
+                             comm_ctas=0, max_ctas=0, raster_group=0, block_n=0, spin_timeout_ns=0, stream=None):
+    arr = _shards(B_shards)
+    a = GemmArgs(_ptr(A), C.cast(arr, C.POINTER(C.c_void_p)), heap, M, N, K, world, mode, dtype, c_off, flag_off, lock_off,
+                 epoch, comm_ctas, max_ctas, raster_group, block_n, spin_timeout_ns)
+    _ck(lib().iris_gemm_all_scatter_ex(C.byref(a), _stream(stream)))
+
+
+def gemm_all_scatter(A, B_shards, heap, M, N, K, world, mode):
+    """The short form: bf16, C at offset 0, default stream (see the header)."""
+    arr = _shards(B_shards)
+    _ck(lib().gemm_all_scatter(_ptr(A), C.cast(arr, C.POINTER(C.c_void_p)), heap, M, N, K, world, mode))
+
+
+def iris_consume_bias(heap, c_off, out_off, flag_off, bias, M, N, world, dtype, epoch, ctas=0, timeout_ns=0, stream=None):
+    _ck(lib().iris_consume_bias(heap, c_off, out_off, flag_off, _ptr(bias), M, N, world, dtype, epoch, ctas, timeout_ns, _stream(stream)))
+
+
+def iris_gemm_out_offset(M: int, N: int, world: int) -> int:
+    return lib().iris_gemm_out_offset(M, N, world)
+
+
+def iris_gemm_all_scatter_host(A_host, B_shards_host, C_host, flags_host, bias_host, OUT_host, heap, M, N, K, world, mode, dtype,
+                               out_slot=0):
+    arr = _shards(B_shards_host)
+    _ck(lib().iris_gemm_all_scatter_host(_ptr(A_host), C.cast(arr, C.POINTER(C.c_void_p)), _ptr(C_host), _ptr(flags_host),
+                                         _ptr(bias_host), _ptr(OUT_host), heap, M, N, K, world, mode, dtype, out_slot))

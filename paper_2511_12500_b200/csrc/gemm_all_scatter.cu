@@ -1,0 +1,723 @@
+// GEMM + all-scatter over the emulated symmetric heap, three schedules (Section 4, Listings 2-5).
+//
+// One persistent, warp-specialised kernel computes C tiles with tcgen05 MMAs:
+//   warp 0      TMA producer  (cp.async.bulk.tensor -> 128B-swizzled shared-memory stages, mbarrier ring)
+//   warp 1      MMA issuer    (one thread; tcgen05.mma into a double-buffered TMEM accumulator)
+//   warps 2..5  epilogue      (tcgen05.ld -> fp32 -> fp16/bf16 -> 16-byte global stores -> flags)
+// The tile loop is the paper's `for tile_id in range(pid, total_tiles, NUM_SMS)` (Listings 3-5).
+// What happens to a finished tile depends on the schedule:
+//   bulk_synchronous       store to the owner rank's slot; a second kernel scatters and publishes
+//   fused_sequential       store to all W slots from registers, then publish W ready flags
+//   workgroup_specialized  store to the owner slot, cas(lock, 0->1, release); reserved communication
+//                          CTAs poll the locks (acquire), copy the tile to the other W-1 slots with
+//                          TMA and publish the flags
+// Because the TMEM accumulator is double buffered, the epilogue of tile i (including the W-way
+// scatter) overlaps the main loop of tile i+1 inside one CTA.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include <algorithm>
+#include <cstring>
+
+#include "iris_device.cuh"
+#include "sm100_ptx.cuh"
+
+namespace iris {
+
+constexpr int BM = 128;           // rows of a compute tile = rows of a publication tile
+constexpr int BK = 64;            // 64 x 16-bit = 128 bytes = one swizzle row
+constexpr int UMMA_K = 16;        // K of one tcgen05.mma for 16-bit inputs
+constexpr int kGemmThreads = 192;
+constexpr int kEpiThreads = 128;
+constexpr int kRing = 6;          // communication CTA: 32 KB tile buffers in flight
+constexpr int kRingLag = 4;       // store groups allowed in flight before the oldest is retired
+constexpr int kTileBytes = IRIS_TILE * IRIS_TILE * 2;
+constexpr int kSmemPayload = 192 * 1024;
+constexpr int kSmemCtrl = 1024;
+constexpr int kSmemTotal = kSmemPayload + kSmemCtrl + 1024;  // + slack to align the base to 1024
+
+template <int BN>
+struct TileCfg {
+  static constexpr int kStageBytes = BM * BK * 2 + BN * BK * 2;
+  static constexpr int kStages = kSmemPayload / kStageBytes;  // 4 for BN=256, 6 for BN=128
+  static constexpr int kTmemCols = 2 * BN;                    // two accumulators
+};
+
+struct alignas(64) GemmParams {
+  CUtensorMap tmA;                    // A [M, K], box 64 x 128, 128B swizzle
+  CUtensorMap tmB[IRIS_MAX_WORLD];    // B_r [N_local, K], box 64 x BN, 128B swizzle
+  CUtensorMap tmC[IRIS_MAX_WORLD];    // C of slot s viewed as [W][M][N_local], box 128 x 128 x 1, no swizzle
+  HeapTable tab;
+  uint64_t c_off, flag_off, lock_off;
+  uint64_t timeout_ns;
+  int32_t* status;
+  int M, N, K, n_local;
+  int tiles_m;          // ceil(M / 128)
+  int ctiles_per_rank;  // compute tiles per rank along N: ceil(N_local / BN)
+  int ptiles_per_rank;  // publication tiles per rank along N: ceil(N_local / 128)
+  int total_ctiles;     // tiles_m * W * ctiles_per_rank
+  int total_ptiles;     // tiles_m * W * ptiles_per_rank
+  int kblocks;          // ceil(K / 64)
+  int gemm_ctas, comm_ctas;
+  int raster_group;
+  int mode;
+  int32_t epoch;
+};
+
+struct CtrlBlock {  // lives in shared memory after the payload area
+  uint64_t full[8];
+  uint64_t empty[8];
+  uint64_t tmem_full[2];
+  uint64_t tmem_empty[2];
+  uint64_t ring_full[kRing];
+  uint64_t ring_free[kRing];
+  int32_t ring_tile[kRing];
+  uint32_t tmem_base;
+  volatile int abort;
+};
+
+struct TileCoord { int tm, rank, jn; };
+
+// Tile id -> coordinates, grouped like Triton's GROUP_SIZE_M swizzle (Section 3.4): ids run down
+// `raster_group` tile rows before moving to the next tile column, so CTAs that run at the same
+// time share A row panels and B column panels in L2.
+__device__ __forceinline__ TileCoord decode_ctile(int id, const GemmParams& p) {
+  const int tiles_n = p.tab.world * p.ctiles_per_rank;
+  const int per_group = p.raster_group * tiles_n;
+  const int g = id / per_group;
+  const int first_m = g * p.raster_group;
+  const int gsz = min(p.raster_group, p.tiles_m - first_m);
+  const int in = id - g * per_group;
+  const int tn = in / gsz;
+  TileCoord c;
+  c.tm = first_m + in % gsz;
+  c.rank = tn / p.ctiles_per_rank;
+  c.jn = tn % p.ctiles_per_rank;
+  return c;
+}
+
+// Bounded mbarrier wait.  Returns false when the deadline passed (recorded in the status block) or
+// when another thread of the CTA already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const GemmParams& p, CtrlBlock* ctrl, int tile) {
+  if (ptx::mbar_try_wait(bar, parity)) return true;
+  const uint64_t start = globaltimer_ns();
+  uint32_t spins = 0;
+  while (!ptx::mbar_try_wait(bar, parity)) {
+    if ((++spins & 63u) == 0) {
+      if (ctrl->abort) return false;
+      if (globaltimer_ns() - start > p.timeout_ns) {
+        report_timeout(p.status, KID_GEMM, tile, -1, (int)parity, (int)(bar & 0xFFFF));
+        ctrl->abort = 1;
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+template <bool BF16>
+__device__ __forceinline__ uint32_t pack2(uint32_t lo_bits, uint32_t hi_bits) {
+  const float lo = __uint_as_float(lo_bits), hi = __uint_as_float(hi_bits);
+  if (BF16) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);  // .x = lo (lower address), .y = hi
+    return *reinterpret_cast<uint32_t*>(&v);
+  } else {
+    __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Communication CTA (workgroup-specialised mode), Listing 5's `else` branch.
+//   warp 0: all 32 lanes watch 32 pending tiles' locks at once (one acquire-ordered load each);
+//           a ballot collects the ready set, shuffles hand each ready tile id to lane 0, which takes
+//           the lock (cas 1->0, acquire) and issues the TMA load of the owner's tile into a ring buffer.
+//   warp 1: waits for each buffer, issues the W-1 TMA stores (iris.put to every other rank), and once a
+//           store group has completed publishes the W ready flags.
+// ------------------------------------------------------------------------------------------------
+__device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload, int warp, int lane) {
+  const int c = (int)blockIdx.x - p.gemm_ctas;
+  const int W = p.tab.world;
+  const int n_my = (p.total_ptiles - c + p.comm_ctas - 1) / p.comm_ctas;  // tiles c, c+COMM, ...
+  const int pt_n = W * p.ptiles_per_rank;
+  if (warp == 0) {
+    int widx = lane < n_my ? lane : -1;  // index into my tile list that this lane watches
+    int next = n_my < 32 ? n_my : 32;
+    int issued = 0;
+    uint64_t last_progress = globaltimer_ns();
+    uint32_t spins = 0;
+    bool ok = true;
+    while (ok && __any_sync(0xFFFFFFFFu, widx >= 0)) {
+      int t = -1, rank = 0;
+      bool ready = false;
+      if (widx >= 0) {
+        t = c + widx * p.comm_ctas;
+        rank = (t % pt_n) / p.ptiles_per_rank;
+        const int32_t* lock = reinterpret_cast<const int32_t*>(p.tab.base[rank] + p.lock_off) + t;
+        ready = ld_acquire_gpu(lock) == 1;
+      }
+      uint32_t mask = __ballot_sync(0xFFFFFFFFu, ready);
+      if (mask == 0) {
+        if ((++spins & 15u) == 0) {
+          bool expired = false;
+          if (lane == 0) {
+            expired = ctrl->abort != 0;
+            if (!expired && globaltimer_ns() - last_progress > p.timeout_ns) {
+              report_timeout(p.status, KID_GEMM, t, -2, 0, 1);
+              ctrl->abort = 1;
+              expired = true;
+            }
+          }
+          if (__any_sync(0xFFFFFFFFu, expired)) ok = false;
+        }
+        continue;
+      }
+      const uint32_t ready_mask = mask;
+      while (mask) {
+        const int src = __ffs(mask) - 1;
+        mask &= mask - 1;
+        const int rt = __shfl_sync(0xFFFFFFFFu, t, src);
+        const int rrank = __shfl_sync(0xFFFFFFFFu, rank, src);
+        bool fail = false;
+        if (lane == 0) {
+          const int slot = issued % kRing;
+          const uint32_t par = ((issued / kRing) & 1) ^ 1;
+          if (!mbar_wait(ptx::smem_u32(&ctrl->ring_free[slot]), par, p, ctrl, rt)) {
+            fail = true;
+          } else {
+            int32_t* lock = reinterpret_cast<int32_t*>(p.tab.base[rrank] + p.lock_off) + rt;
+            (void)cas_acquire_gpu(lock, 1, 0);  // take the tile; the lock is ready for the next call
+            fence_proxy_async();                // producer's generic-proxy stores -> our async-proxy read
+            const int tm = rt / pt_n, pj = (rt % pt_n) % p.ptiles_per_rank;
+            ctrl->ring_tile[slot] = rt;
+            const uint32_t bar = ptx::smem_u32(&ctrl->ring_full[slot]);
+            ptx::mbar_arrive_expect_tx(bar, kTileBytes);
+            ptx::tma_load_3d(ptx::smem_u32(payload + slot * kTileBytes), &p.tmC[rrank], pj * IRIS_TILE, tm * IRIS_TILE, rrank, bar);
+          }
+        }
+        ++issued;
+        if (__any_sync(0xFFFFFFFFu, fail)) { ok = false; break; }
+      }
+      // lanes whose tile was taken move on to the next unwatched tiles, in lane order
+      const int rank_in_mask = __popc(ready_mask & ((1u << lane) - 1u));
+      if (ready_mask & (1u << lane)) {
+        const int cand = next + rank_in_mask;
+        widx = cand < n_my ? cand : -1;
+      }
+      next = min(n_my, next + __popc(ready_mask));
+      last_progress = globaltimer_ns();
+    }
+  } else if (warp == 1) {
+    int done = 0;  // tiles whose flags have been published
+    bool ok = true;
+    auto publish = [&](int i) {
+      const int slot = i % kRing;
+      const int rt = ctrl->ring_tile[slot];
+      __syncwarp();
+      if (lane < W) st_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[lane] + p.flag_off) + rt, p.epoch);
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->ring_free[slot]));
+    };
+    for (int i = 0; i < n_my && ok; ++i) {
+      const int slot = i % kRing;
+      bool fail = false;
+      if (lane == 0) {
+        if (!mbar_wait(ptx::smem_u32(&ctrl->ring_full[slot]), (i / kRing) & 1, p, ctrl, -3)) {
+          fail = true;
+        } else {
+          const int rt = ctrl->ring_tile[slot];
+          const int tm = rt / pt_n, rrank = (rt % pt_n) / p.ptiles_per_rank, pj = (rt % pt_n) % p.ptiles_per_rank;
+          for (int s = 0; s < W; ++s)
+            if (s != rrank) ptx::tma_store_3d(&p.tmC[s], pj * IRIS_TILE, tm * IRIS_TILE, rrank, ptx::smem_u32(payload + slot * kTileBytes));
+          ptx::bulk_commit_group();
+          if (i >= kRingLag) ptx::bulk_wait_group<kRingLag>();
+        }
+      }
+      if (__any_sync(0xFFFFFFFFu, fail)) { ok = false; break; }
+      if (i >= kRingLag) { publish(done); ++done; }
+    }
+    if (lane == 0) ptx::bulk_wait_group<0>();  // also on the failure path: no copy of ours stays in flight
+    __syncwarp();
+    if (ok) while (done < n_my) { publish(done); ++done; }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// The GEMM + scatter kernel.
+// ------------------------------------------------------------------------------------------------
+template <int BN, bool BF16>
+__global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const __grid_constant__ GemmParams p) {
+  using Cfg = TileCfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* payload = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  CtrlBlock* ctrl = reinterpret_cast<CtrlBlock*>(payload + kSmemPayload);
+  const int warp = (int)threadIdx.x / 32, lane = (int)threadIdx.x % 32;
+  const bool is_comm = (int)blockIdx.x >= p.gemm_ctas;
+  const int W = p.tab.world;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < Cfg::kStages; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->empty[i]), 1); }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i]), 4); }
+    for (int i = 0; i < kRing; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->ring_full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->ring_free[i]), 1); }
+    ctrl->abort = 0;
+    ptx::fence_mbar_init();
+    fence_proxy_async();
+    if (p.kblocks > 0 && !is_comm) {
+      ptx::prefetch_tensormap(&p.tmA);
+      for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmB[r]);
+    }
+    if (is_comm)
+      for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmC[r]);
+  }
+  if (warp == 1 && !is_comm) {
+    ptx::tmem_alloc(ptx::smem_u32(&ctrl->tmem_base), Cfg::kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+
+  if (is_comm) {
+    comm_cta(p, ctrl, payload, warp, lane);
+  } else if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.total_ctiles && ok; tile += p.gemm_ctas) {
+        const TileCoord tc = decode_ctile(tile, p);
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!mbar_wait(ptx::smem_u32(&ctrl->empty[stage]), phase ^ 1, p, ctrl, tile)) { ok = false; break; }
+          const uint32_t bar = ptx::smem_u32(&ctrl->full[stage]);
+          uint8_t* sa = payload + stage * Cfg::kStageBytes;
+          ptx::mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
+          ptx::tma_load_2d(ptx::smem_u32(sa), &p.tmA, kb * BK, tc.tm * BM, bar);
+          ptx::tma_load_2d(ptx::smem_u32(sa + BM * BK * 2), &p.tmB[tc.rank], kb * BK, tc.jn * BN, bar);
+          if (++stage == Cfg::kStages) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::idesc_f16(BM, BN, BF16 ? 1 : 0);
+      const uint32_t tmem_base = ctrl->tmem_base;
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < p.total_ctiles && ok; tile += p.gemm_ctas) {
+        if (!mbar_wait(ptx::smem_u32(&ctrl->tmem_empty[acc]), acc_phase ^ 1, p, ctrl, tile)) break;
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!mbar_wait(ptx::smem_u32(&ctrl->full[stage]), phase, p, ctrl, tile)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t sa = ptx::smem_u32(payload + stage * Cfg::kStageBytes);
+          const uint64_t adesc = ptx::smem_desc_k_sw128(sa);
+          const uint64_t bdesc = ptx::smem_desc_k_sw128(sa + BM * BK * 2);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)  // +32 bytes per K step: +2 in the (>>4) address field
+            ptx::mma_f16_ss(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+          ptx::mma_commit(ptx::smem_u32(&ctrl->empty[stage]));  // stage reusable once these MMAs have read it
+          if (++stage == Cfg::kStages) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        ptx::mma_commit(ptx::smem_u32(&ctrl->tmem_full[acc]));  // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      }
+    }
+  } else {
+    // ---------------- epilogue: warps 2..5, lane quadrant = warp % 4 ----------------
+    const int quad = warp & 3;
+    const int et = (int)threadIdx.x - 64;  // 0..127
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    const uint32_t tmem_base = ctrl->tmem_base;
+    for (int tile = blockIdx.x; tile < p.total_ctiles; tile += p.gemm_ctas) {
+      const TileCoord tc = decode_ctile(tile, p);
+      const bool ok = mbar_wait(ptx::smem_u32(&ctrl->tmem_full[acc]), acc_phase, p, ctrl, tile);
+      if (ptx::bar_red_or(1, kEpiThreads, !ok)) break;  // uniform decision for all four warps
+      ptx::tc_fence_after();
+      const int row = tc.tm * BM + quad * 32 + lane;
+      const int col_in_shard = tc.jn * BN;
+      const uint64_t row_off = p.c_off + ((uint64_t)row * p.N + (uint64_t)tc.rank * p.n_local) * 2;
+#pragma unroll 1
+      for (int ch = 0; ch < BN / 32; ++ch) {
+        uint32_t v[32];
+        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + ch * 32), v);
+        ptx::tmem_wait_ld();
+        uint4 q[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          if (p.kblocks == 0) {
+            q[i] = make_uint4(0, 0, 0, 0);  // K == 0: the sum is empty
+          } else {
+            q[i].x = pack2<BF16>(v[8 * i + 0], v[8 * i + 1]);
+            q[i].y = pack2<BF16>(v[8 * i + 2], v[8 * i + 3]);
+            q[i].z = pack2<BF16>(v[8 * i + 4], v[8 * i + 5]);
+            q[i].w = pack2<BF16>(v[8 * i + 6], v[8 * i + 7]);
+          }
+        }
+        if (row < p.M) {
+          const int c0 = col_in_shard + ch * 32;
+          if (p.mode == IRIS_MODE_FUSED_SEQUENTIAL) {
+            // Listing 4: for remote_rank in range(world_size): iris.store(C + offset, c, cur_rank, remote_rank)
+            for (int s = 0; s < W; ++s) {
+              const uint64_t dst = p.tab.base[s] + row_off + (uint64_t)c0 * 2;  // translate(C + offset, rank -> s)
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                if (c0 + 8 * i < p.n_local) st_global_v4(reinterpret_cast<void*>(dst + 16 * i), q[i]);
+            }
+          } else {
+            // Listings 3 and 5: store to the local (owner) rank's memory
+            const uint64_t dst = p.tab.base[tc.rank] + row_off + (uint64_t)c0 * 2;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              if (c0 + 8 * i < p.n_local) st_global_v4(reinterpret_cast<void*>(dst + 16 * i), q[i]);
+          }
+        }
+      }
+      // accumulator drained: hand it back to the MMA warp
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[acc]));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      if (p.mode != IRIS_MODE_BULK_SYNCHRONOUS) {
+        // every epilogue thread's stores happen-before the barrier; the release below is cumulative
+        asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
+        const int subs = BN / IRIS_TILE;
+        const int pt_n = W * p.ptiles_per_rank;
+        if (p.mode == IRIS_MODE_FUSED_SEQUENTIAL) {
+          if (et < subs * W) {
+            const int sub = et / W, s = et % W;
+            const int pj = tc.jn * subs + sub;
+            if (pj < p.ptiles_per_rank) {
+              const int t = tc.tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
+              st_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[s] + p.flag_off) + t, p.epoch);
+            }
+          }
+        } else if (et < subs) {
+          const int pj = tc.jn * subs + et;
+          if (pj < p.ptiles_per_rank) {
+            const int t = tc.tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
+            // Listing 5: tl.atomic_cas(locks + tile_id, 0, 1, sem="release", scope="gpu")
+            (void)cas_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[tc.rank] + p.lock_off) + t, 0, 1);
+          }
+        }
+      }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1 && !is_comm) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(ctrl->tmem_base, Cfg::kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Bulk-synchronous second kernel (Listing 3, all_scatter): per publication tile, iris.put the owner's
+// tile to every other rank, then publish the W ready flags.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) all_scatter_kernel(const __grid_constant__ HeapTable tab, uint64_t c_off, uint64_t flag_off, int M, int N, int n_local,
+                                                          int tiles_m, int ptiles_per_rank, int32_t epoch) {
+  const int W = tab.world;
+  const int pt_n = W * ptiles_per_rank;
+  const int total = tiles_m * pt_n;
+  for (int t = blockIdx.x; t < total; t += gridDim.x) {
+    const int tm = t / pt_n, rank = (t % pt_n) / ptiles_per_rank, pj = (t % pt_n) % ptiles_per_rank;
+    const int rows = min(IRIS_TILE, M - tm * IRIS_TILE);
+    const int cols = min(IRIS_TILE, n_local - pj * IRIS_TILE);
+    const int cpr = cols / 8;  // 16-byte chunks per row
+    const uint64_t local = tab.base[rank] + c_off + ((uint64_t)(tm * IRIS_TILE) * N + (uint64_t)rank * n_local + (uint64_t)pj * IRIS_TILE) * 2;
+    for (int i0 = threadIdx.x; i0 < rows * cpr; i0 += 256 * 4) {
+      uint4 v[4];
+      uint64_t off[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i = i0 + u * 256;
+        if (i < rows * cpr) {
+          off[u] = ((uint64_t)(i / cpr) * N + (uint64_t)(i % cpr) * 8) * 2;
+          v[u] = ld_global_v4(reinterpret_cast<const void*>(local + off[u]));
+        }
+      }
+      for (int s = 0; s < W; ++s) {
+        if (s == rank) continue;
+        const uint64_t remote = translate(local, rank, s, tab);
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+          if (i0 + u * 256 < rows * cpr) st_global_v4(reinterpret_cast<void*>(remote + off[u]), v[u]);
+      }
+    }
+    __syncthreads();
+    if ((int)threadIdx.x < W) st_release_gpu(reinterpret_cast<int32_t*>(tab.base[threadIdx.x] + flag_off) + t, epoch);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+  }
+  return fn;
+}
+
+static int make_map(CUtensorMap* m, int dtype, int rank, void* base, const cuuint64_t* dims, const cuuint64_t* strides, const cuuint32_t* box,
+                    CUtensorMapSwizzle swz, const char* what) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return fail(IRIS_ERR_CUDA, "cuTensorMapEncodeTiled entry point not available");
+  const cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(m, dtype == IRIS_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, (cuuint32_t)rank, base, dims, strides, box,
+                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(IRIS_ERR_CUDA, "cuTensorMapEncodeTiled(%s) failed with CUresult %d", what, (int)r);
+  return IRIS_OK;
+}
+
+template <int BN, bool BF16>
+static int launch_gemm(const GemmParams& p, int grid, bool cooperative, cudaStream_t st) {
+  auto kern = gemm_all_scatter_kernel<BN, BF16>;
+  static bool configured = false;
+  if (!configured) {
+    IRIS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal));
+    configured = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = kSmemTotal;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;  // CTAs that wait on one another must be co-resident
+  attr[0].val.cooperative = cooperative ? 1 : 0;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  IRIS_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, p));
+  return IRIS_OK;
+}
+
+int64_t num_tiles(int M, int N, int world) {
+  if (M < 0 || N < 0 || world < 1 || world > IRIS_MAX_WORLD || N % world != 0) return -1;
+  const int64_t nl = N / world;
+  return (int64_t)((M + IRIS_TILE - 1) / IRIS_TILE) * world * ((nl + IRIS_TILE - 1) / IRIS_TILE);
+}
+
+}  // namespace iris
+
+using namespace iris;
+
+extern "C" {
+
+int64_t iris_num_tiles(int M, int N, int world) {
+  const int64_t n = num_tiles(M, N, world);
+  return n < 0 ? fail(IRIS_ERR_ARG, "iris_num_tiles: bad arguments") : n;
+}
+
+size_t iris_gemm_heap_bytes(int M, int N, int world) {
+  const int64_t nt = num_tiles(M, N, world);
+  if (nt < 0) return 0;
+  return (size_t)(align_up((uint64_t)M * N * 2, 256) + 2 * align_up((uint64_t)nt * 4, 256) + 256);
+}
+
+int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
+  if (!a) return fail(IRIS_ERR_ARG, "gemm_all_scatter: NULL args");
+  iris_heap* h = a->heap;
+  if (!heap_ok(h)) return fail(IRIS_ERR_STATE, "gemm_all_scatter: bad heap handle");
+  const int W = a->world;
+  if (W != h->world) return fail(IRIS_ERR_ARG, "gemm_all_scatter: world=%d differs from the heap's world=%d", W, h->world);
+  if (a->mode < IRIS_MODE_BULK_SYNCHRONOUS || a->mode > IRIS_MODE_WORKGROUP_SPECIALIZED) return fail(IRIS_ERR_ARG, "gemm_all_scatter: unknown mode %d", a->mode);
+  if (a->dtype != IRIS_F16 && a->dtype != IRIS_BF16) return fail(IRIS_ERR_ARG, "gemm_all_scatter: unknown dtype %d", a->dtype);
+  if (a->M < 0 || a->N < 0 || a->K < 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: negative dimension");
+  if (a->N % W != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: N=%d is not a multiple of world=%d", a->N, W);
+  const int nl = a->N / W;
+  if (nl % 8 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: N/world=%d must be a multiple of 8 (16-byte stores)", nl);
+  if (a->K % 8 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: K=%d must be a multiple of 8 (16-byte row pitch)", a->K);
+  if (a->block_n != 0 && a->block_n != 128 && a->block_n != 256) return fail(IRIS_ERR_ARG, "gemm_all_scatter: block_n must be 0, 128 or 256");
+  if (a->epoch < 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: epoch must be >= 1");
+  if (a->c_off % 256 != 0 || a->flag_off % 4 != 0 || a->lock_off % 4 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: misaligned heap offsets");
+  if (a->comm_ctas < 0 || a->max_ctas < 0 || a->raster_group < 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: negative tuning parameter");
+  const int64_t nt = num_tiles(a->M, a->N, W);
+  const uint64_t bpr = h->bytes_per_rank;
+  const uint64_t c_bytes = (uint64_t)a->M * a->N * 2;
+  if (a->c_off > bpr || c_bytes > bpr - a->c_off) return fail(IRIS_ERR_RANGE, "gemm_all_scatter: C leaves the slot");
+  if (a->flag_off > bpr || (uint64_t)nt * 4 > bpr - a->flag_off) return fail(IRIS_ERR_RANGE, "gemm_all_scatter: flags leave the slot");
+  const bool wg = a->mode == IRIS_MODE_WORKGROUP_SPECIALIZED;
+  if (wg && (a->lock_off > bpr || (uint64_t)nt * 4 > bpr - a->lock_off)) return fail(IRIS_ERR_RANGE, "gemm_all_scatter: locks leave the slot");
+  auto overlaps = [](uint64_t o1, uint64_t n1, uint64_t o2, uint64_t n2) { return n1 && n2 && o1 < o2 + n2 && o2 < o1 + n1; };
+  if (overlaps(a->c_off, c_bytes, a->flag_off, (uint64_t)nt * 4) || (wg && (overlaps(a->c_off, c_bytes, a->lock_off, (uint64_t)nt * 4) || overlaps(a->flag_off, (uint64_t)nt * 4, a->lock_off, (uint64_t)nt * 4))))
+    return fail(IRIS_ERR_ARG, "gemm_all_scatter: C, flag and lock regions overlap");
+  if (a->M == 0 || a->N == 0) return IRIS_OK;  // empty output: nothing to compute, nothing to publish
+  if (!a->A && a->K > 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: A is NULL");
+  if (!a->B_shards) return fail(IRIS_ERR_ARG, "gemm_all_scatter: B_shards is NULL");
+  if ((uint64_t)a->A % 16 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: A must be 16-byte aligned");
+  for (int r = 0; r < W; ++r)
+    if (a->K > 0 && (!a->B_shards[r] || (uint64_t)a->B_shards[r] % 16 != 0)) return fail(IRIS_ERR_ARG, "gemm_all_scatter: B_shards[%d] is NULL or not 16-byte aligned", r);
+
+  GemmParams p;
+  std::memset(&p, 0, sizeof(p));
+  int bn = a->block_n;
+  if (bn == 0) bn = (nl % 256 == 0 || nl > 1024) ? 256 : 128;
+  if (nl <= 128) bn = 128;
+  p.tab = h->table();
+  p.c_off = a->c_off;
+  p.flag_off = a->flag_off;
+  p.lock_off = a->lock_off;
+  p.timeout_ns = a->spin_timeout_ns ? a->spin_timeout_ns : kDefaultTimeoutNs;
+  p.status = h->status;
+  p.M = a->M; p.N = a->N; p.K = a->K; p.n_local = nl;
+  p.tiles_m = (a->M + BM - 1) / BM;
+  p.ctiles_per_rank = (nl + bn - 1) / bn;
+  p.ptiles_per_rank = (nl + IRIS_TILE - 1) / IRIS_TILE;
+  p.total_ctiles = p.tiles_m * W * p.ctiles_per_rank;
+  p.total_ptiles = p.tiles_m * W * p.ptiles_per_rank;
+  p.kblocks = (a->K + BK - 1) / BK;
+  p.raster_group = a->raster_group ? a->raster_group : 16;
+  p.mode = a->mode;
+  p.epoch = a->epoch;
+  int grid = a->max_ctas ? std::min(a->max_ctas, h->sm_count) : h->sm_count;
+  if (wg) {
+    if (grid < 2) return fail(IRIS_ERR_ARG, "gemm_all_scatter: workgroup_specialized needs at least 2 CTAs");
+    int comm = a->comm_ctas ? a->comm_ctas : 8;
+    comm = std::min(comm, std::min(grid - 1, p.total_ptiles));
+    p.comm_ctas = comm;
+    p.gemm_ctas = std::min(grid - comm, p.total_ctiles);
+  } else {
+    p.comm_ctas = 0;
+    p.gemm_ctas = std::min(grid, p.total_ctiles);
+  }
+  grid = p.gemm_ctas + p.comm_ctas;
+
+  // Tensor maps.  K == 0 has no operand to describe; the kernel then never issues a load.
+  if (a->K > 0) {
+    const cuuint64_t dimsA[2] = {(cuuint64_t)a->K, (cuuint64_t)a->M};
+    const cuuint64_t strA[1] = {(cuuint64_t)a->K * 2};
+    const cuuint32_t boxA[2] = {BK, BM};
+    int rc = make_map(&p.tmA, a->dtype, 2, const_cast<void*>(a->A), dimsA, strA, boxA, CU_TENSOR_MAP_SWIZZLE_128B, "A");
+    if (rc != IRIS_OK) return rc;
+    for (int r = 0; r < W; ++r) {
+      const cuuint64_t dimsB[2] = {(cuuint64_t)a->K, (cuuint64_t)nl};
+      const cuuint32_t boxB[2] = {BK, (cuuint32_t)bn};
+      rc = make_map(&p.tmB[r], a->dtype, 2, const_cast<void*>(a->B_shards[r]), dimsB, strA, boxB, CU_TENSOR_MAP_SWIZZLE_128B, "B");
+      if (rc != IRIS_OK) return rc;
+    }
+  }
+  if (wg) {
+    for (int s = 0; s < W; ++s) {
+      const cuuint64_t dimsC[3] = {(cuuint64_t)nl, (cuuint64_t)a->M, (cuuint64_t)W};
+      const cuuint64_t strC[2] = {(cuuint64_t)a->N * 2, (cuuint64_t)nl * 2};
+      const cuuint32_t boxC[3] = {IRIS_TILE, IRIS_TILE, 1};
+      int rc = make_map(&p.tmC[s], a->dtype, 3, h->base + (size_t)s * bpr + a->c_off, dimsC, strC, boxC, CU_TENSOR_MAP_SWIZZLE_NONE, "C");
+      if (rc != IRIS_OK) return rc;
+    }
+  }
+
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc;
+  const bool bf = a->dtype == IRIS_BF16;
+  if (bn == 256) rc = bf ? launch_gemm<256, true>(p, grid, wg, st) : launch_gemm<256, false>(p, grid, wg, st);
+  else           rc = bf ? launch_gemm<128, true>(p, grid, wg, st) : launch_gemm<128, false>(p, grid, wg, st);
+  if (rc != IRIS_OK) return rc;
+  if (a->mode == IRIS_MODE_BULK_SYNCHRONOUS) {
+    // Listing 3: the second kernel on the same stream; the kernel boundary is the synchronisation.
+    const int g2 = std::min(p.total_ptiles, h->sm_count * 8);
+    all_scatter_kernel<<<g2, 256, 0, st>>>(p.tab, a->c_off, a->flag_off, a->M, a->N, nl, p.tiles_m, p.ptiles_per_rank, a->epoch);
+    IRIS_CUDA_TRY(cudaGetLastError());
+  }
+  return IRIS_OK;
+}
+
+static void short_form_layout(int M, int N, int world, uint64_t* flag_off, uint64_t* lock_off) {
+  const int64_t nt = num_tiles(M, N, world);
+  *flag_off = align_up((uint64_t)M * N * 2, 256);
+  *lock_off = *flag_off + align_up((uint64_t)(nt > 0 ? nt : 0) * 4, 256);
+}
+
+static int short_form(const void* A, const void* const* B_shards, iris_heap* heap, int M, int N, int K, int world, int mode, int dtype, void* stream) {
+  if (!heap_ok(heap)) return fail(IRIS_ERR_STATE, "gemm_all_scatter: bad heap handle");
+  if (num_tiles(M, N, world) < 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: bad M/N/world");
+  iris_gemm_args a;
+  std::memset(&a, 0, sizeof(a));
+  a.A = A; a.B_shards = B_shards; a.heap = heap;
+  a.M = M; a.N = N; a.K = K; a.world = world; a.mode = mode; a.dtype = dtype;
+  a.c_off = 0;
+  short_form_layout(M, N, world, &a.flag_off, &a.lock_off);
+  a.epoch = heap->epoch + 1;
+  const int rc = iris_gemm_all_scatter_ex(&a, stream);
+  if (rc == IRIS_OK) heap->epoch = a.epoch;
+  return rc;
+}
+
+int gemm_all_scatter(const void* A, const void* const* B_shards, iris_heap* heap, int M, int N, int K, int world, int mode) {
+  return short_form(A, B_shards, heap, M, N, K, world, mode, IRIS_BF16, nullptr);
+}
+
+uint64_t iris_gemm_out_offset(int M, int N, int world) {
+  if (num_tiles(M, N, world) < 0) return 0;
+  uint64_t flag_off, lock_off;
+  short_form_layout(M, N, world, &flag_off, &lock_off);
+  return lock_off + (lock_off - flag_off);
+}
+
+int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_host, void* C_host, int32_t* flags_host, const void* bias_host,
+                               void* OUT_host, iris_heap* heap, int M, int N, int K, int world, int mode, int dtype, int out_slot) {
+  if (!heap_ok(heap)) return fail(IRIS_ERR_STATE, "gemm_all_scatter_host: bad heap handle");
+  if (world != heap->world || out_slot < 0 || out_slot >= world) return fail(IRIS_ERR_ARG, "gemm_all_scatter_host: bad world or out_slot");
+  const int64_t nt = num_tiles(M, N, world);
+  if (nt < 0 || K < 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter_host: bad M/N/K/world");
+  if ((M > 0 && N > 0) && (!A_host || !B_shards_host || !C_host)) return fail(IRIS_ERR_ARG, "gemm_all_scatter_host: NULL buffer");
+  if ((bias_host == nullptr) != (OUT_host == nullptr)) return fail(IRIS_ERR_ARG, "gemm_all_scatter_host: bias_host and OUT_host go together");
+  const size_t c_bytes = (size_t)M * N * 2;
+  const uint64_t out_off = iris_gemm_out_offset(M, N, world);
+  if (bias_host && out_off + c_bytes > heap->bytes_per_rank) return fail(IRIS_ERR_RANGE, "gemm_all_scatter_host: heap slot too small for OUT");
+  const size_t a_bytes = (size_t)M * K * 2, b_bytes = (size_t)N * K * 2, shard_bytes = world ? b_bytes / world : 0;
+  const size_t stage_b_need = b_bytes + (bias_host ? align_up((uint64_t)N * 2, 256) : 0);
+  if (a_bytes > heap->stage_a_bytes) {
+    if (heap->stage_a) cudaFree(heap->stage_a);
+    heap->stage_a = nullptr; heap->stage_a_bytes = 0;
+    if (cudaMalloc(&heap->stage_a, a_bytes) != cudaSuccess) { cudaGetLastError(); return fail(IRIS_ERR_NOMEM, "gemm_all_scatter_host: staging for A"); }
+    heap->stage_a_bytes = a_bytes;
+  }
+  if (stage_b_need > heap->stage_b_bytes) {
+    if (heap->stage_b) cudaFree(heap->stage_b);
+    heap->stage_b = nullptr; heap->stage_b_bytes = 0;
+    if (cudaMalloc(&heap->stage_b, stage_b_need) != cudaSuccess) { cudaGetLastError(); return fail(IRIS_ERR_NOMEM, "gemm_all_scatter_host: staging for B"); }
+    heap->stage_b_bytes = stage_b_need;
+  }
+  cudaStream_t st = nullptr;
+  const void* dB[IRIS_MAX_WORLD] = {nullptr};
+  if (a_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(heap->stage_a, A_host, a_bytes, cudaMemcpyHostToDevice, st));
+  for (int r = 0; r < world; ++r) {
+    dB[r] = static_cast<char*>(heap->stage_b) + (size_t)r * shard_bytes;
+    if (shard_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(dB[r]), B_shards_host[r], shard_bytes, cudaMemcpyHostToDevice, st));
+  }
+  void* dbias = static_cast<char*>(heap->stage_b) + b_bytes;
+  if (bias_host && N > 0) IRIS_CUDA_TRY(cudaMemcpyAsync(dbias, bias_host, (size_t)N * 2, cudaMemcpyHostToDevice, st));
+  int rc = short_form(heap->stage_a, dB, heap, M, N, K, world, mode, dtype, st);
+  if (rc != IRIS_OK) return rc;
+  uint64_t flag_off, lock_off;
+  short_form_layout(M, N, world, &flag_off, &lock_off);
+  char* slot = heap->base + (size_t)out_slot * heap->bytes_per_rank;
+  if (bias_host) {
+    rc = iris_consume_bias(heap, 0, out_off, flag_off, dbias, M, N, world, dtype, heap->epoch, 0, 0, st);
+    if (rc != IRIS_OK) return rc;
+  }
+  if (c_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(C_host, slot, c_bytes, cudaMemcpyDeviceToHost, st));
+  if (bias_host && c_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(OUT_host, slot + out_off, c_bytes, cudaMemcpyDeviceToHost, st));
+  if (flags_host && nt > 0)
+    for (int s = 0; s < world; ++s)
+      IRIS_CUDA_TRY(cudaMemcpyAsync(flags_host + (size_t)s * nt, heap->base + (size_t)s * heap->bytes_per_rank + flag_off, (size_t)nt * 4, cudaMemcpyDeviceToHost, st));
+  return iris_status_check(heap, st, nullptr);
+}
+
+}  // extern "C"

@@ -19,6 +19,9 @@ round-to-nearest-even library casts; the resulting uint16 bit patterns *are* the
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 import torch
 
@@ -107,9 +110,18 @@ def matrix(seed: int, stream: int, rows: int, cols: int, dist: str, dtype: str,
     n = (row_end - row_begin) * cols
     out = np.empty(n, dtype=np.uint16)
     base = row_begin * cols
-    for off in range(0, n, _CHUNK):
+
+    def fill(off: int):
         cnt = min(_CHUNK, n - off)
         out[off:off + cnt] = to16(_values(seed, stream, base + off, cnt, dist), dtype)
+
+    offsets = range(0, n, _CHUNK)
+    if len(offsets) > 1:       # chunks are independent (counter-based): generate them on several host threads
+        with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as pool:
+            list(pool.map(fill, offsets))
+    else:
+        for off in offsets:
+            fill(off)
     return out.reshape(row_end - row_begin, cols)
 
 

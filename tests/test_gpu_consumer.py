@@ -1,0 +1,115 @@
+"""GPU parity for the flag-gated consumer (OUT = C + bias after acquiring each tile's flag) and for the
+bounded device-side waits: a wait that can never be satisfied returns an error status, and the GPU
+stays usable (nothing traps, nothing spins forever)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2511_12500_b200 as iris
+from paper_2511_12500_b200 import inputs
+from gpu_util import SENTINEL, GpuHeap, dev16, first_diff, gemm_layout
+
+pytestmark = pytest.mark.gpu
+
+MODES = [iris.IRIS_MODE_BULK_SYNCHRONOUS, iris.IRIS_MODE_FUSED_SEQUENTIAL, iris.IRIS_MODE_WORKGROUP_SPECIALIZED]
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "fp16"])
+@pytest.mark.parametrize("W,M,nl", [(2, 256, 128), (4, 130, 136), (8, 384, 256)])
+def test_consumer_matches_oracle_on_seeded_C(dtype, W, M, nl):
+    """C, bias and flags are written directly; the consumer's output must equal the oracle's bit for bit."""
+    N = W * nl
+    c_off, flag_off, lock_off, out_off, bpr = gemm_layout(M, N, W, with_out=True)
+    C = inputs.matrix(51, 0, M, N, "uniform", dtype)
+    bias = inputs.vector(51, inputs.STREAM_BIAS, N, "uniform", dtype)
+    nt = oracle.num_tiles(M, N, W)
+    with GpuHeap(W, bpr) as g:
+        img = g.image()
+        for s in range(W):
+            g.write(s, c_off, C)
+            img.view(s, c_off, M * N * 2, np.uint16)[:] = C.reshape(-1)
+        iris.iris_flags_fill(g.h, flag_off, nt, 9)
+        img.publish_flags(flag_off, nt, 9)
+        iris.iris_consume_bias(g.h, c_off, out_off, flag_off, dev16(bias), M, N, W, iris.DTYPES[dtype], 9)   # flag == epoch
+        iris.iris_status_check(g.h)
+        img.consume_bias(dtype, c_off, out_off, M, N, bias)
+        host = g.to_host()
+        assert np.array_equal(host, img.mem), first_diff(host, img.mem)
+        iris.iris_consume_bias(g.h, c_off, out_off, flag_off, dev16(bias), M, N, W, iris.DTYPES[dtype], 5)   # flag > epoch passes too
+        iris.iris_status_check(g.h)
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_producer_then_consumer_on_poisoned_heap(mode):
+    """The heap starts as NaN patterns (0xFFFF); a consumer that read a tile before its flag would emit NaNs.
+    OUT must equal the consumer definition applied to the GPU's own C, bit for bit (fp32 add + one rounding
+    is deterministic), and C must be within tolerance of the oracle."""
+    W, M, nl, K, dtype = 4, 512, 256, 512, "bf16"
+    N = W * nl
+    A, Bs = inputs.gemm_inputs(inputs.SEED0 + 4, W, M, N, K, "uniform", dtype)
+    bias = inputs.vector(inputs.SEED0 + 4, inputs.STREAM_BIAS, N, "uniform", dtype)
+    c_off, flag_off, lock_off, out_off, bpr = gemm_layout(M, N, W, with_out=True)
+    nt = oracle.num_tiles(M, N, W)
+    with GpuHeap(W, bpr, fill=0xFF) as g:
+        iris.iris_flags_fill(g.h, flag_off, nt, 0)
+        iris.iris_flags_fill(g.h, lock_off, nt, 0)
+        dA, dB, dbias = dev16(A), [dev16(b) for b in Bs], dev16(bias)
+        for epoch in (1, 2):
+            iris.iris_gemm_all_scatter_ex(g.h, dA, dB, M, N, K, W, mode, iris.IRIS_BF16, c_off, flag_off, lock_off, epoch)
+            iris.iris_consume_bias(g.h, c_off, out_off, flag_off, dbias, M, N, W, iris.IRIS_BF16, epoch)
+            iris.iris_status_check(g.h)
+        host = g.to_host()
+        c0 = host[c_off:c_off + M * N * 2].view(np.uint16).reshape(M, N)
+        exp_out = oracle.consume_bias_rows(c0, bias, dtype)
+        for s in range(W):
+            out = host[s * bpr + out_off: s * bpr + out_off + M * N * 2].view(np.uint16).reshape(M, N)
+            assert np.array_equal(out, exp_out)
+        assert not np.isnan(oracle.decode(exp_out, dtype)).any()
+
+
+def test_consumer_wait_that_cannot_be_satisfied_times_out_cleanly():
+    W, M, nl = 2, 256, 128
+    N = W * nl
+    c_off, flag_off, lock_off, out_off, bpr = gemm_layout(M, N, W, with_out=True)
+    with GpuHeap(W, bpr) as g:
+        nt = oracle.num_tiles(M, N, W)
+        iris.iris_flags_fill(g.h, flag_off, nt, 0)                      # nothing will ever publish epoch 1
+        bias = torch.zeros(N, dtype=torch.int16, device="cuda")
+        iris.iris_consume_bias(g.h, c_off, out_off, flag_off, bias, M, N, W, iris.IRIS_BF16, 1, 0, 2_000_000)   # 2 ms deadline
+        with pytest.raises(iris.IrisError) as e:
+            iris.iris_status_check(g.h)
+        assert e.value.code == iris.IRIS_ERR_TIMEOUT
+        assert e.value.detail[1] == 3 and e.value.detail[5] == 0 and e.value.detail[6] == 1   # consumer, seen 0, wanted 1
+        out = g.view(0, out_off, M * N * 2)
+        assert bool(torch.all(out == SENTINEL))                         # no tile was touched
+        iris.iris_status_check(g.h)                                     # status cleared; context still healthy
+        iris.iris_flags_fill(g.h, flag_off, nt, 1)
+        iris.iris_consume_bias(g.h, c_off, out_off, flag_off, bias, M, N, W, iris.IRIS_BF16, 1)
+        iris.iris_status_check(g.h)
+
+
+def test_communication_ctas_give_up_when_a_lock_is_never_released():
+    """Workgroup-specialised mode with the lock array pre-set to a value the handshake never produces for the
+    communicators (2): producers' cas(0->1) misses, communicators never see 1, and their bounded wait expires."""
+    W, M, nl, K = 2, 256, 128, 64
+    N = W * nl
+    A, Bs = inputs.gemm_inputs(3, W, M, N, K, "uniform", "bf16")
+    c_off, flag_off, lock_off, out_off, bpr = gemm_layout(M, N, W, with_out=True)
+    with GpuHeap(W, bpr) as g:
+        nt = oracle.num_tiles(M, N, W)
+        iris.iris_flags_fill(g.h, lock_off, nt, 2)
+        iris.iris_flags_fill(g.h, flag_off, nt, 0)
+        iris.iris_gemm_all_scatter_ex(g.h, dev16(A), [dev16(b) for b in Bs], M, N, K, W, iris.IRIS_MODE_WORKGROUP_SPECIALIZED,
+                                      iris.IRIS_BF16, c_off, flag_off, lock_off, 1, spin_timeout_ns=3_000_000)
+        with pytest.raises(iris.IrisError) as e:
+            iris.iris_status_check(g.h)
+        assert e.value.code == iris.IRIS_ERR_TIMEOUT and e.value.detail[1] == 1
+        flags = g.view(0, flag_off, nt * 4, torch.int32)
+        assert bool(torch.all(flags == 0))                              # nothing was published
+        # the device is still usable: a correct run right after succeeds
+        iris.iris_flags_fill(g.h, lock_off, nt, 0)
+        iris.iris_gemm_all_scatter_ex(g.h, dev16(A), [dev16(b) for b in Bs], M, N, K, W, iris.IRIS_MODE_WORKGROUP_SPECIALIZED,
+                                      iris.IRIS_BF16, c_off, flag_off, lock_off, 1)
+        iris.iris_status_check(g.h)
+        assert bool(torch.all(flags == 1))

@@ -1,0 +1,278 @@
+"""GPU parity for gemm_all_scatter in its three schedules, against the CPU oracle.
+
+Layout, replication, flags and locks are compared bit-exactly (whole heap image); values are compared
+bit-exactly where the arithmetic is exact (integer-valued inputs) and within the stated tolerance
+otherwise: max |gpu - ref| <= 1e-2 (|ref| + 1) elementwise, relative Frobenius error <= 2e-3.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2511_12500_b200 as iris
+from paper_2511_12500_b200 import inputs
+from gpu_util import SENTINEL, GpuHeap, check_tolerance, dev16, first_diff, gemm_layout
+
+pytestmark = pytest.mark.gpu
+
+MODES = [iris.IRIS_MODE_BULK_SYNCHRONOUS, iris.IRIS_MODE_FUSED_SEQUENTIAL, iris.IRIS_MODE_WORKGROUP_SPECIALIZED]
+MODE_IDS = ["bulk_synchronous", "fused_sequential", "workgroup_specialized"]
+
+
+def run_gemm(g, A, Bs, dtype, mode, epoch=1, with_locks_zeroed=True, **kw):
+    M, K = A.shape
+    W, nl = len(Bs), Bs[0].shape[0]
+    N = W * nl
+    c_off, flag_off, lock_off, out_off, _ = gemm_layout(M, N, W, with_out=True)
+    dA, dB = dev16(A), [dev16(b) for b in Bs]
+    nt = oracle.num_tiles(M, N, W) if M and N else 0
+    if with_locks_zeroed and nt:
+        iris.iris_flags_fill(g.h, lock_off, nt, 0)
+    iris.iris_gemm_all_scatter_ex(g.h, dA, dB, M, N, K, W, mode, iris.DTYPES[dtype], c_off, flag_off, lock_off, epoch, **kw)
+    iris.iris_status_check(g.h)
+    return c_off, flag_off, lock_off, out_off, nt
+
+
+def expected_image(g, A, Bs, dtype, mode, epoch=1, c_full=None):
+    M = A.shape[0]
+    W, nl = len(Bs), Bs[0].shape[0]
+    N = W * nl
+    c_off, flag_off, lock_off, out_off, _ = gemm_layout(M, N, W, with_out=True)
+    img = g.image()
+    nt = oracle.num_tiles(M, N, W) if M and N else 0
+    for s in range(W):                       # the caller zeroes the lock array in every slot
+        img.view(s, lock_off, nt * 4, np.int32)[:] = 0
+    if M and N:
+        if c_full is None:
+            c_full = oracle.gemm_block(A, Bs, dtype)
+        img.all_scatter(c_off, c_full)
+        img.publish_flags(flag_off, nt, epoch)
+        if mode == iris.IRIS_MODE_WORKGROUP_SPECIALIZED:
+            img.consume_locks(lock_off, M, N)
+    return img, c_full
+
+
+def c_slot(host, g, s, c_off, M, N):
+    return host[s * g.bpr + c_off: s * g.bpr + c_off + M * N * 2].view(np.uint16).reshape(M, N)
+
+
+# ------------------------------------------------------------------------------------------------
+# Config 1 of the benchmark definition: W=2, M=N=K=256, fp16 uniform[-1,1], 128x128 tiles.
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+def test_config1_all_modes(mode):
+    W, M, N, K, dtype = 2, 256, 256, 256, "fp16"
+    A, Bs = inputs.gemm_inputs(inputs.SEED0 + 0, W, M, N, K, "uniform", dtype)
+    bpr = gemm_layout(M, N, W, True)[4]
+    with GpuHeap(W, bpr) as g:
+        c_off, flag_off, lock_off, _, nt = run_gemm(g, A, Bs, dtype, mode)
+        host = g.to_host()
+        img, c_ref = expected_image(g, A, Bs, dtype, mode)
+        # values: within tolerance in slot 0 ...
+        check_tolerance(c_slot(host, g, 0, c_off, M, N), c_ref, dtype)
+        # ... layout / replication / flags / locks / sentinel: bit-exact once the oracle image carries the GPU's values
+        img2, _ = expected_image(g, A, Bs, dtype, mode, c_full=c_slot(host, g, 0, c_off, M, N).copy())
+        assert np.array_equal(host, img2.mem), first_diff(host, img2.mem)
+        assert nt == 4
+
+
+# ------------------------------------------------------------------------------------------------
+# Exact-arithmetic inputs: every dot product is a small integer, so any correct fp32-accumulating GEMM
+# equals the oracle byte for byte.  This pins tile placement, rank offsets, replication, flags and locks.
+# ------------------------------------------------------------------------------------------------
+EXACT_SHAPES = [
+    # W, M, N_local, K
+    (1, 128, 128, 64),
+    (2, 256, 128, 256),
+    (2, 384, 256, 192),        # BN=256 path, 3 tile rows
+    (4, 130, 136, 72),         # ragged M, ragged N_local (not a multiple of 128), ragged K (not a multiple of 64)
+    (8, 128, 512, 128),
+    (3, 520, 392, 328),        # odd world, everything ragged, several tiles
+    (8, 1, 8, 8),              # smallest legal problem
+    (2, 300, 640, 64),         # N_local > 512 and not a multiple of 256
+]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("dtype", ["bf16", "fp16"])
+@pytest.mark.parametrize("W,M,nl,K", EXACT_SHAPES)
+def test_exact_integer_gemm_full_heap_image(mode, dtype, W, M, nl, K):
+    N = W * nl
+    A = inputs.matrix(41, inputs.STREAM_A, M, K, "ternary:0.5", dtype)
+    Bs = [inputs.matrix(41, inputs.STREAM_B0 + r, nl, K, "smallint:2", dtype) for r in range(W)]
+    bpr = gemm_layout(M, N, W, True)[4]
+    with GpuHeap(W, bpr) as g:
+        run_gemm(g, A, Bs, dtype, mode)
+        host = g.to_host()
+        img, _ = expected_image(g, A, Bs, dtype, mode)
+        assert np.array_equal(host, img.mem), first_diff(host, img.mem)
+
+
+@pytest.mark.parametrize("block_n", [128, 256])
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+def test_exact_integer_gemm_tile_width_and_grid_knobs(block_n, mode):
+    W, M, nl, K, dtype = 4, 640, 512, 320, "bf16"
+    N = W * nl
+    A = inputs.matrix(43, inputs.STREAM_A, M, K, "smallint:2", dtype)
+    Bs = [inputs.matrix(43, inputs.STREAM_B0 + r, nl, K, "ternary:0.5", dtype) for r in range(W)]
+    bpr = gemm_layout(M, N, W, True)[4]
+    with GpuHeap(W, bpr) as g:
+        img = None
+        for kw in (dict(), dict(max_ctas=7, comm_ctas=3, raster_group=2), dict(max_ctas=148, comm_ctas=32, raster_group=1)):
+            g.mem.fill_(SENTINEL)
+            run_gemm(g, A, Bs, dtype, mode, block_n=block_n, **kw)
+            host = g.to_host()
+            if img is None:
+                img, _ = expected_image(g, A, Bs, dtype, mode)
+            assert np.array_equal(host, img.mem), (kw, first_diff(host, img.mem))
+
+
+# ------------------------------------------------------------------------------------------------
+# Real-valued inputs: tolerance vs the oracle; all W copies byte-identical; the three schedules agree
+# bit for bit (they share one main loop).
+# ------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,dist", [("bf16", "normal002"), ("bf16", "uniform"), ("fp16", "uniform")])
+def test_real_valued_tolerance_replication_and_cross_mode_equality(dtype, dist):
+    W, M, nl, K = 4, 384, 256, 1024
+    N = W * nl
+    A, Bs = inputs.gemm_inputs(inputs.SEED0 + 2, W, M, N, K, dist, dtype)
+    c_ref = oracle.gemm_block(A, Bs, dtype)
+    bpr = gemm_layout(M, N, W, True)[4]
+    results = []
+    with GpuHeap(W, bpr) as g:
+        for mode in MODES:
+            g.mem.fill_(SENTINEL)
+            c_off, flag_off, lock_off, _, nt = run_gemm(g, A, Bs, dtype, mode)
+            host = g.to_host()
+            c0 = c_slot(host, g, 0, c_off, M, N).copy()
+            check_tolerance(c0, c_ref, dtype)
+            for s in range(1, W):
+                assert np.array_equal(c_slot(host, g, s, c_off, M, N), c0)
+            img, _ = expected_image(g, A, Bs, dtype, mode, c_full=c0)
+            assert np.array_equal(host, img.mem), first_diff(host, img.mem)
+            results.append(c0)
+    assert np.array_equal(results[0], results[1]) and np.array_equal(results[0], results[2])
+
+
+def test_identity_B_reproduces_A_and_zero_A_gives_zero():
+    W, M, K, dtype = 2, 256, 256, "bf16"
+    A = inputs.matrix(5, 0, M, K, "uniform", dtype)
+    A[A == 0x8000] = 0
+    eye = oracle.encode(np.eye(K), dtype)
+    Bs = [np.ascontiguousarray(eye[r * 128:(r + 1) * 128]) for r in range(W)]
+    bpr = gemm_layout(M, K, W, True)[4]
+    with GpuHeap(W, bpr) as g:
+        c_off = run_gemm(g, A, Bs, dtype, iris.IRIS_MODE_FUSED_SEQUENTIAL)[0]
+        host = g.to_host()
+        for s in range(W):
+            assert np.array_equal(c_slot(host, g, s, c_off, M, K), A)
+        c_off = run_gemm(g, np.zeros_like(A), Bs, dtype, iris.IRIS_MODE_WORKGROUP_SPECIALIZED, epoch=2)[0]
+        host = g.to_host()
+        for s in range(W):
+            assert not c_slot(host, g, s, c_off, M, K).any()
+
+
+def test_epochs_advance_without_resets_and_runs_are_deterministic():
+    W, M, nl, K, dtype = 2, 256, 256, 512, "bf16"
+    N = W * nl
+    A, Bs = inputs.gemm_inputs(77, W, M, N, K, "uniform", dtype)
+    bpr = gemm_layout(M, N, W, True)[4]
+    with GpuHeap(W, bpr) as g:
+        first = None
+        for epoch in range(1, 6):
+            mode = MODES[epoch % 3]
+            c_off, flag_off, lock_off, _, nt = run_gemm(g, A, Bs, dtype, mode, epoch=epoch, with_locks_zeroed=(epoch == 1))
+            host = g.to_host()
+            for s in range(W):
+                f = host[s * g.bpr + flag_off: s * g.bpr + flag_off + nt * 4].view(np.int32)
+                assert np.all(f == epoch)
+                lk = host[s * g.bpr + lock_off: s * g.bpr + lock_off + nt * 4].view(np.int32)
+                assert np.all(lk == 0)                      # locks reset themselves (cas 1 -> 0)
+            c0 = c_slot(host, g, 0, c_off, M, N).copy()
+            if first is None:
+                first = c0
+            assert np.array_equal(first, c0)
+
+
+def test_empty_problems_and_K_zero():
+    with GpuHeap(2, 1 << 20) as g:
+        dummy = torch.zeros(64, dtype=torch.int16, device="cuda")
+        for (M, N, K) in [(0, 256, 64), (128, 0, 64)]:
+            iris.iris_gemm_all_scatter_ex(g.h, dummy, [dummy, dummy], M, N, K, 2, 1, iris.IRIS_BF16, 0, 65536, 0, 1)
+        iris.iris_status_check(g.h)
+        assert bool(torch.all(g.mem == SENTINEL))           # nothing written, nothing published
+        # K = 0: the empty sum, C = +0 everywhere, flags published
+        M, N = 128, 256
+        c_off, flag_off, lock_off, _, _ = gemm_layout(M, N, 2, True)
+        for mode in MODES:
+            g.mem.fill_(SENTINEL)
+            iris.iris_flags_fill(g.h, lock_off, 2, 0)
+            iris.iris_gemm_all_scatter_ex(g.h, None, [None, None], M, N, 0, 2, mode, iris.IRIS_BF16, c_off, flag_off, lock_off, 3)
+            iris.iris_status_check(g.h)
+            host = g.to_host()
+            img = g.image()
+            for s in range(2):
+                img.view(s, lock_off, 8, np.int32)[:] = 0
+            img.all_scatter(c_off, np.zeros((M, N), dtype=np.uint16))
+            img.publish_flags(flag_off, 2, 3)
+            assert np.array_equal(host, img.mem), first_diff(host, img.mem)
+
+
+def test_argument_errors_are_reported_before_any_launch():
+    with GpuHeap(2, 1 << 20) as g:
+        d = torch.zeros(1 << 16, dtype=torch.int16, device="cuda")
+        ok = dict(M=128, N=256, K=64, world=2, mode=1, dtype=iris.IRIS_BF16, c_off=0, flag_off=65536, lock_off=66560, epoch=1)
+        cases = [
+            (dict(N=250), iris.IRIS_ERR_ARG), (dict(N=264, K=64), iris.IRIS_ERR_ARG), (dict(K=60), iris.IRIS_ERR_ARG),
+            (dict(mode=3), iris.IRIS_ERR_ARG), (dict(dtype=2), iris.IRIS_ERR_ARG), (dict(world=4), iris.IRIS_ERR_ARG),
+            (dict(epoch=0), iris.IRIS_ERR_ARG), (dict(c_off=128), iris.IRIS_ERR_ARG), (dict(block_n=64), iris.IRIS_ERR_ARG),
+            (dict(M=4096, N=256), iris.IRIS_ERR_RANGE), (dict(flag_off=(1 << 20) - 4), iris.IRIS_ERR_RANGE),
+            (dict(flag_off=1024), iris.IRIS_ERR_ARG),                   # flags inside C
+            (dict(mode=2, lock_off=65536), iris.IRIS_ERR_ARG),          # locks on top of flags
+        ]
+        for delta, code in cases:
+            kw = {**ok, **delta}
+            with pytest.raises(iris.IrisError) as e:
+                iris.iris_gemm_all_scatter_ex(g.h, d, [d, d], kw["M"], kw["N"], kw["K"], kw["world"], kw["mode"], kw["dtype"],
+                                              kw["c_off"], kw["flag_off"], kw["lock_off"], kw["epoch"], block_n=kw.get("block_n", 0))
+            assert e.value.code == code, (delta, e.value)
+        torch.cuda.synchronize()
+        assert bool(torch.all(g.mem == SENTINEL))
+
+
+def test_short_form_and_host_entry_point():
+    W, M, N, K = 2, 256, 512, 256
+    A, Bs = inputs.gemm_inputs(9, W, M, N, K, "smallint:2", "bf16")
+    c_ref = oracle.gemm_block(A, Bs, "bf16")
+    nt = oracle.num_tiles(M, N, W)
+    bpr = iris.iris_gemm_heap_bytes(M, N, W)
+    flag_off = (M * N * 2 + 255) // 256 * 256
+    lock_off = flag_off + (nt * 4 + 255) // 256 * 256
+    assert bpr == lock_off + (nt * 4 + 255) // 256 * 256 + 256
+    with GpuHeap(W, bpr) as g:
+        dA, dB = dev16(A), [dev16(b) for b in Bs]
+        iris.iris_flags_fill(g.h, lock_off, nt, 0)
+        for i, mode in enumerate(MODES):
+            iris.gemm_all_scatter(dA, dB, g.h, M, N, K, W, mode)       # default stream
+            iris.iris_status_check(g.h, 0)
+            assert iris.iris_heap_epoch(g.h) == i + 1
+            host = g.to_host()
+            for s in range(W):
+                assert np.array_equal(c_slot(host, g, s, 0, M, N), c_ref)
+                assert np.all(host[s * bpr + flag_off: s * bpr + flag_off + nt * 4].view(np.int32) == i + 1)
+        # host buffers in, host buffers out
+        C_host = np.empty((M, N), dtype=np.uint16)
+        flags = np.empty((W, nt), dtype=np.int32)
+        iris.iris_gemm_all_scatter_host(A, Bs, C_host, flags, None, None, g.h, M, N, K, W, iris.IRIS_MODE_WORKGROUP_SPECIALIZED,
+                                        iris.IRIS_BF16, 1)
+        assert np.array_equal(C_host, c_ref) and np.all(flags == 4)
+    # with the consumer: OUT comes back too
+    out_off = iris.iris_gemm_out_offset(M, N, W)
+    assert out_off == bpr - 256
+    bias = inputs.vector(9, inputs.STREAM_BIAS, N, "smallint:2", "bf16")
+    with GpuHeap(W, out_off + M * N * 2) as g:
+        iris.iris_flags_fill(g.h, lock_off, nt, 0)
+        C_host, OUT_host = np.empty((M, N), dtype=np.uint16), np.empty((M, N), dtype=np.uint16)
+        iris.iris_gemm_all_scatter_host(A, Bs, C_host, None, bias, OUT_host, g.h, M, N, K, W, iris.IRIS_MODE_FUSED_SEQUENTIAL,
+                                        iris.IRIS_BF16, 0)
+        assert np.array_equal(C_host, c_ref) and np.array_equal(OUT_host, oracle.consume_bias_rows(c_ref, bias, "bf16"))
