@@ -1,0 +1,407 @@
+#!/usr/bin/env python
+"""Benchmark of the GEMM + all-scatter hot path on B200 (one JSON line on stdout).
+
+A step = one pass of the whole path on one batch of synthetic input:
+    gemm_all_scatter (workgroup_specialized)  ->  flag-gated consumer (OUT = C + bias)
+on the workload the target is quoted on: W=8 emulated ranks, M=8192, N=K=16384, bf16 uniform[-1,1).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W]            # the CUDA path
+  python bench.py --impl reference [--steps K] [--warmup W]      # the CPU oracle on a bounded sample
+
+`value` is TFLOP/s of the step (2*M*N*K flops per step) with inputs resident in HBM; `e2e` is the same
+metric through the host-buffer entry point (H2D of A, B, bias and D2H of C, OUT, flags inside the timed
+region); `roofline` describes the dominant kernel (the GEMM + scatter kernel) against the measured
+tensor peak; `cpu_baseline` is the oracle timed on this machine's host cores on a sample of the same workload.
+With --gpus N > 1 every rank runs an independent replica (the path is emulated inside one GPU and has no
+cross-GPU exchange step); the value is the sum over ranks, timed as the max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+WORKLOADS = {
+    # name: (W, M, N, K, dist, dtype)
+    "cfg5_w8_m8192_n16384_k16384": (8, 8192, 16384, 16384, "uniform", "bf16"),
+    "cfg5_w8_m1024_n16384_k16384": (8, 1024, 16384, 16384, "uniform", "bf16"),
+    "cfg3_w8_m4096_n8192_k8192": (8, 4096, 8192, 8192, "normal002", "bf16"),
+    "cfg4_w8_m128_n28672_k8192": (8, 128, 28672, 8192, "normal002", "bf16"),
+    "cfg1_w2_256": (2, 256, 256, 256, "uniform", "fp16"),
+}
+DEFAULT_WORKLOAD = "cfg5_w8_m8192_n16384_k16384"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+METRIC = "gemm_all_scatter_tflops"
+UNIT = "TFLOP/s"
+# DRAM traffic of one workgroup_specialized launch on the default workload (bytes), from the ncu capture
+# summarised in profiles/; None until a capture exists.
+NCU_TRAFFIC_BYTES = None
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def align(x, a=256):
+    return (x + a - 1) // a * a
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 100 ms while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        os.unlink(self.path)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), power_w_max=float(max(pw)), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+def sample_strips(M: int, W: int, count: int, seed: int = 1):
+    """Seeded sample of (tile row, rank) strips: 128 rows x one rank's whole column shard."""
+    rng = np.random.default_rng(seed)
+    tiles_m = -(-M // 128)
+    total = tiles_m * W
+    picks = rng.choice(total, size=min(count, total), replace=False)
+    return [(int(p) // W, int(p) % W) for p in picks]
+
+
+def oracle_strip_sample(workload, seed, strips, threads=None):
+    """Oracle (as it stands: fp64 accumulation, one rounding) on the given strips: (seconds, flops, cores).
+    Only the oracle call is timed; drawing the strip's input rows is not."""
+    import oracle
+    from paper_2511_12500_b200 import inputs
+    W, M, N, K, dist, dtype = workload
+    nl = N // W
+    secs, flops = 0.0, 0.0
+    cores = threads or oracle.hw_threads()
+    for tm, r in strips:
+        m0, m1 = tm * 128, min(M, tm * 128 + 128)
+        A = inputs.matrix(seed, inputs.STREAM_A, M, K, dist, dtype, m0, m1)
+        B = inputs.matrix(seed, inputs.STREAM_B0 + r, nl, K, dist, dtype)
+        t0 = time.perf_counter()
+        oracle.gemm_block(A, [B], dtype, threads=cores)
+        secs += time.perf_counter() - t0
+        flops += 2.0 * (m1 - m0) * nl * K
+    return secs, flops, cores
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    workload = WORKLOADS[args.workload]
+    W, M, N, K, dist, dtype = workload
+    seed = 251112500 + 4
+    strips = sample_strips(M, W, args.steps + args.warmup, seed=7)
+    while len(strips) < args.steps + args.warmup:
+        strips += strips
+    for i in range(args.warmup):
+        oracle_strip_sample(workload, seed, strips[i:i + 1])
+    secs, flops, cores = 0.0, 0.0, 0
+    for i in range(args.warmup, args.warmup + args.steps):
+        s, f, cores = oracle_strip_sample(workload, seed, strips[i:i + 1])
+        secs += s
+        flops += f
+    value = flops / secs / 1e12
+    sample = f"one strip (128 rows x one rank's {N // W}-column shard, K={K}) of {args.workload} per step, fp64 accumulation"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": secs / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "world": W, "M": M, "N": N, "K": K, "mode": "oracle", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import torch
+    import paper_2511_12500_b200 as iris
+    from paper_2511_12500_b200 import inputs
+
+    world_size = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    dist_on = world_size > 1
+    if dist_on:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    pk, pk_kind = peaks()
+
+    workload = WORKLOADS[args.workload]
+    W, M, N, K, dist_name, dtype = workload
+    seed = 251112500 + 4 + rank                     # independent batch per replica
+    nl = N // W
+    nt = iris.iris_num_tiles(M, N, W)
+    flag_off = align(M * N * 2)
+    lock_off = flag_off + align(nt * 4)
+    out_off = iris.iris_gemm_out_offset(M, N, W)
+    bpr = align(out_off + M * N * 2)
+    mode = iris.MODES[args.mode]
+    dt = iris.DTYPES[dtype]
+
+    A, Bs = inputs.gemm_inputs(seed, W, M, N, K, dist_name, dtype)
+    bias = inputs.vector(seed, inputs.STREAM_BIAS, N, "uniform", dtype)
+    dA = torch.from_numpy(A.view(np.int16)).cuda()
+    dB = [torch.from_numpy(b.view(np.int16)).cuda() for b in Bs]
+    dbias = torch.from_numpy(bias.view(np.int16)).cuda()
+    heap_mem = torch.zeros(W * bpr, dtype=torch.uint8, device="cuda")
+    h = iris.iris_heap_create(W, bpr, external_base=heap_mem.data_ptr())
+    stream = torch.cuda.current_stream()
+    flops = 2.0 * M * N * K
+    store_bytes = float(W) * M * N * 2
+
+    def gemm(epoch, m=mode, **kw):
+        iris.iris_gemm_all_scatter_ex(h, dA, dB, M, N, K, W, m, dt, 0, flag_off, lock_off, epoch, comm_ctas=args.comm_ctas,
+                                      raster_group=args.raster_group, block_n=args.block_n, **kw)
+
+    def consume(epoch):
+        iris.iris_consume_bias(h, 0, out_off, flag_off, dbias, M, N, W, dt, epoch)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist_on:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    epoch = 0
+    for _ in range(args.warmup):
+        epoch += 1
+        gemm(epoch)
+        consume(epoch)
+    iris.iris_status_check(h)
+
+    # ---------------- timed region: exactly K steps ----------------
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    barrier()
+    sampler.start()
+    for i in range(args.steps):
+        epoch += 1
+        ev[i][0].record(stream)
+        gemm(epoch)
+        ev[i][1].record(stream)
+        consume(epoch)
+        ev[i][2].record(stream)
+    barrier()
+    clocks = sampler.stop()
+    iris.iris_status_check(h)
+    total_ms = ev[0][0].elapsed_time(ev[-1][2])
+    gemm_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+    cons_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+    if dist_on:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world_size * flops / (ms_per_step * 1e-3) / 1e12
+
+    result = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world_size, "steps": args.steps, "warmup": args.warmup,
+              "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if dtype == "bf16" else "f16",
+              "data": "synthetic",
+              "config": {"workload": args.workload, "world": W, "M": M, "N": N, "K": K, "mode": args.mode, "comm_ctas": args.comm_ctas or 8,
+                         "step": "gemm_all_scatter + flag-gated consumer (OUT = C + bias)", "accumulate": "fp32",
+                         "l2": "inputs (0.8 GB) and outputs (4.3 GB) far exceed the 126 MB L2; no explicit flush",
+                         "multi_gpu": "replicas only (ranks are emulated inside one GPU)"},
+              "clocks": clocks, "gpu_launches": 2 * args.steps}
+
+    if rank == 0:
+        # ---------------- roofline of the dominant kernel ----------------
+        t_tensor = flops / (pk["bf16_tflops"] * 1e12) * 1e3
+        t_store = store_bytes / (pk["hbm_gbs"] * 1e9) * 1e3
+        achieved = flops / (gemm_ms * 1e-3) / 1e12
+        result["roofline"] = {"kernel": f"gemm_all_scatter_kernel<256,bf16> ({args.mode})", "bound": "tensor", "achieved": achieved,
+                              "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / pk["bf16_tflops"],
+                              "peak_kind": f"{pk_kind} burst (of {pk_kind})", "peak_sustained": pk["bf16_tflops_sustained"],
+                              "frac_sustained": achieved / pk["bf16_tflops_sustained"], "traffic": NCU_TRAFFIC_BYTES,
+                              "kernel_ms": gemm_ms, "combined_roofline_ms": max(t_tensor, t_store),
+                              "frac_of_combined_roofline": max(t_tensor, t_store) / gemm_ms,
+                              "replicated_store_gbs": store_bytes / (gemm_ms * 1e-3) / 1e9}
+        cons_bytes = 2.0 * store_bytes + N * 2
+        result["consumer"] = {"kernel_ms": cons_ms, "gbs": cons_bytes / (cons_ms * 1e-3) / 1e9,
+                              "frac_of_hbm_peak": cons_bytes / (cons_ms * 1e-3) / 1e9 / pk["hbm_gbs"], "bytes": cons_bytes}
+
+        # ---------------- the three schedules on the same workload (context for the headline) ----------------
+        modes = {}
+        for name, m in (iris.MODES.items() if args.mode_iters > 0 else ()):
+            ts = []
+            for _ in range(1 + args.mode_iters):
+                epoch += 1
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                gemm(epoch, m)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            ms = float(np.median(ts[1:]))
+            modes[name] = {"ms": ms, "tflops": flops / ms / 1e9, "store_gbs": store_bytes / ms / 1e6,
+                           "frac_of_combined_roofline": max(t_tensor, t_store) / ms}
+        iris.iris_status_check(h)
+        result["modes"] = modes
+
+        # ---------------- end to end through the host-buffer entry point ----------------
+        try:
+            if args.e2e_steps <= 0:
+                raise RuntimeError("skipped (--e2e-steps 0)")
+            pin = lambda a: torch.from_numpy(a.view(np.int16)).pin_memory()  # noqa: E731
+            hA, hB, hbias = pin(A), [pin(b) for b in Bs], pin(bias)
+            hC = torch.empty(M * N, dtype=torch.int16).pin_memory()
+            hOUT = torch.empty(M * N, dtype=torch.int16).pin_memory()
+            hflags = torch.empty(W * nt, dtype=torch.int32).pin_memory()
+            iris.iris_flags_fill(h, flag_off, nt, 0)
+            torch.cuda.synchronize()
+            e2e_t = []
+            for i in range(1 + args.e2e_steps):
+                t0 = time.perf_counter()
+                iris.iris_gemm_all_scatter_host(hA, hB, hC, hflags, hbias, hOUT, h, M, N, K, W, mode, dt, 0)
+                e2e_t.append(time.perf_counter() - t0)
+            e2e_s = float(np.mean(e2e_t[1:]))
+            h2d = (M * K + N * K + N) * 2
+            d2h = 2 * M * N * 2 + W * nt * 4
+            result["e2e"] = {"value": flops / e2e_s / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                             "ms_per_step": e2e_s * 1e3, "api": "iris_gemm_all_scatter_host (pinned host buffers, default stream)"}
+            del hA, hB, hC, hOUT
+        except Exception as exc:  # pragma: no cover
+            result["e2e"] = {"value": None, "unit": UNIT, "error": str(exc)}
+
+        # ---------------- all-store microbenchmark (replicated-store GB/s vs HBM peak) ----------------
+        if args.sweep != "none":
+            result["all_store"] = all_store_sweep(iris, pk, args.sweep)
+
+        # ---------------- CPU oracle on a bounded sample of the same workload ----------------
+        if not args.no_cpu_baseline:
+            strips = sample_strips(M, W, args.cpu_strips, seed=3)
+            secs, fl, cores = oracle_strip_sample(workload, seed, strips)
+            result["cpu_baseline"] = {"value": fl / secs / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle", "seconds": secs,
+                                      "sample": f"{len(strips)} strips (128 rows x one rank's {nl}-column shard, K={K}) of {args.workload}, "
+                                                f"{fl / flops:.4f} of one step's flops, fp64 accumulation",
+                                      "extrapolated_full_step_seconds": flops / (fl / secs)}
+        print(json.dumps(result))
+    iris.iris_heap_destroy(h)
+    if dist_on:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def all_store_sweep(iris, pk, kind):
+    """W=8 all-store: message sizes 1 KiB .. (64 MiB | 1 GiB) in powers of 4; GB/s counts W*S read + W*W*S written."""
+    import torch
+    W = 8
+    top = 15 if kind == "full" else 13
+    out = []
+    for e in range(5, top + 1):
+        S = 4 ** e
+        tile = min(S, 32768)
+        T = -(-S // tile)
+        payload_off, recv_off = 0, align(S)
+        flag_off = recv_off + align(W * S)
+        bpr = align(flag_off + W * T * 4)
+        free, _ = torch.cuda.mem_get_info()
+        if W * bpr + (2 << 30) > free:
+            out.append({"S": S, "skipped": "insufficient free HBM"})
+            continue
+        mem = torch.empty(W * bpr, dtype=torch.uint8, device="cuda")
+        mem[: 1 << 20].zero_()
+        h = iris.iris_heap_create(W, bpr, external_base=mem.data_ptr())
+        iris.iris_flags_fill(h, flag_off, W * T, 0)
+        stream = torch.cuda.current_stream()
+        iters = 20 if S <= (1 << 24) else 5
+        iris.iris_all_store_bench(h, payload_off, recv_off, flag_off, S, tile, 1)
+        iris.iris_all_store_bench(h, payload_off, recv_off, flag_off, S, tile, 2)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for i in range(iters):
+            iris.iris_all_store_bench(h, payload_off, recv_off, flag_off, S, tile, 3 + i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        iris.iris_status_check(h)
+        ms = e0.elapsed_time(e1) / iters
+        moved = float(W * S + W * W * S)
+        out.append({"S": S, "ms": ms, "gbs": moved / ms / 1e6, "frac_of_hbm_peak": moved / ms / 1e6 / pk["hbm_gbs"],
+                    "l2": "warm (working set below L2)" if W * W * S < (100 << 20) else "exceeds L2"})
+        iris.iris_heap_destroy(h)
+        del mem
+        torch.cuda.empty_cache()
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
+    ap.add_argument("--mode", default="workgroup_specialized", choices=["bulk_synchronous", "fused_sequential", "workgroup_specialized"])
+    ap.add_argument("--comm-ctas", type=int, default=0)
+    ap.add_argument("--raster-group", type=int, default=0)
+    ap.add_argument("--block-n", type=int, default=0)
+    ap.add_argument("--mode-iters", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-strips", type=int, default=16)
+    ap.add_argument("--sweep", default="short", choices=["none", "short", "full"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3                       # timing hygiene: at least three warm-up steps
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
