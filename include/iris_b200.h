@@ -235,6 +235,45 @@ int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_h
 /* Offset of OUT in the short form's layout: right after the lock array (256-byte aligned). */
 uint64_t iris_gemm_out_offset(int M, int N, int world);
 
+/* ------------------------------------------------------------------------------------------ */
+/* An entry point that allocates nothing                                                       */
+/* ------------------------------------------------------------------------------------------ */
+
+/* (The paper has no counterpart to this call; it exists for deployment reasons only.)
+ *
+ * Some callers of this library are not in a position to allocate device memory: a serving process
+ * whose framework reserved all of HBM for its own pool at start-up, so that a cudaMalloc from a
+ * plug-in would fail or eat into somebody else's budget; a latency-critical loop that cannot afford
+ * the device-wide synchronisation an allocation or a free implies; code that runs under a memory
+ * budget fixed in advance and audited.  Every other GEMM entry point needs an iris_heap handle, and
+ * creating one allocates (the status block, and the heap itself unless a base is supplied), and the
+ * workgroup-specialised schedule needs a zeroed lock array on top.  This call needs none of that:
+ *
+ *   - it takes the W slot base addresses directly (slot_bases: HOST array of `world` DEVICE
+ *     addresses, each 256-byte aligned, each the start of bytes_per_rank bytes the caller owns);
+ *     inputs A, B_shards and the outputs (C at c_off and int32 flags at flag_off in every slot)
+ *     are the caller's, exactly as for iris_gemm_all_scatter_ex;
+ *   - it runs the workgroup-specialised schedule; the per-tile locks and the status block live in
+ *     a fixed array inside the library image (static __device__, 65 792 bytes, held by every GPU
+ *     that loads the library until the process exits);
+ *   - it calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ * Limit: at most 16 384 publication tiles, i.e. ceil(M/128) * world * ceil((N/world)/128) <= 16384
+ * (the W=8, 8192 x 16384 output of the largest benchmark configuration has 8192).  Larger problems
+ * are refused with IRIS_ERR_UNSUPPORTED and a message naming the limit; nothing is launched.
+ *
+ * The first call on a device looks up the device address of that array (with that device current)
+ * and remembers it; make this first call outside any stream capture.  Every call clears the words
+ * it is going to use (the array keeps the previous call's contents) on `stream`, launches on
+ * `stream`, then WAITS for the stream and returns IRIS_OK or IRIS_ERR_TIMEOUT (a bounded device-side
+ * wait ran out).  All calls share the one array: two calls whose GPU work overlaps (different
+ * streams, different host threads) race on it and must be serialised by the caller.
+ * Other arguments, checks, layout and results are those of iris_gemm_all_scatter_ex in
+ * IRIS_MODE_WORKGROUP_SPECIALIZED with default tuning; the results are bit-identical to it. */
+int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, const uint64_t* slot_bases,
+                                  size_t bytes_per_rank, int M, int N, int K, int world, int dtype, uint64_t c_off,
+                                  uint64_t flag_off, int32_t epoch, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

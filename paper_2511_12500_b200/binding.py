@@ -30,6 +30,7 @@ EXPORTS = [
     "iris_atomic_add_contended", "iris_atomic_cas_contended", "iris_flags_fill", "iris_all_store_bench",
     "iris_gemm_all_scatter_ex", "gemm_all_scatter", "iris_gemm_heap_bytes", "iris_heap_epoch", "iris_num_tiles",
     "iris_consume_bias", "iris_gemm_all_scatter_host", "iris_gemm_out_offset",
+    "iris_gemm_all_scatter_noalloc",
 ]
 
 
@@ -97,6 +98,7 @@ def lib() -> C.CDLL:
     L.iris_gemm_all_scatter_host.argtypes = [vp, C.POINTER(vp), vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci]
     L.iris_gemm_out_offset.restype = u64
     L.iris_gemm_out_offset.argtypes = [ci, ci, ci]
+    L.iris_gemm_all_scatter_noalloc.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), sz, ci, ci, ci, ci, ci, u64, u64, i32, vp]
     _lib = L
     return L
 
@@ -276,3 +278,13 @@ def iris_gemm_all_scatter_host(A_host, B_shards_host, C_host, flags_host, bias_h
     arr = _shards(B_shards_host)
     _ck(lib().iris_gemm_all_scatter_host(_ptr(A_host), C.cast(arr, C.POINTER(C.c_void_p)), _ptr(C_host), _ptr(flags_host),
                                          _ptr(bias_host), _ptr(OUT_host), heap, M, N, K, world, mode, dtype, out_slot))
+
+
+def iris_gemm_all_scatter_noalloc(A, B_shards, slot_bases, bytes_per_rank, M, N, K, world, dtype, c_off, flag_off, epoch, stream=None):
+    """Workgroup-specialised gemm_all_scatter for callers that must not allocate device memory: no heap handle, the
+    locks and the status block sit in a fixed array inside the library (at most 16384 publication tiles).  Blocks
+    until the work on `stream` has finished.  Calls that overlap on the GPU race on that array."""
+    arr = _shards(B_shards)
+    bases = (C.c_uint64 * len(slot_bases))(*slot_bases)
+    _ck(lib().iris_gemm_all_scatter_noalloc(_ptr(A), C.cast(arr, C.POINTER(C.c_void_p)), bases, bytes_per_rank, M, N, K, world, dtype,
+                                            c_off, flag_off, epoch, _stream(stream)))

@@ -128,6 +128,25 @@ __device__ __forceinline__ uint32_t pack2(uint32_t lo_bits, uint32_t hi_bits) {
   }
 }
 
+}  // namespace iris
+
+// Scratch of iris_gemm_all_scatter_noalloc(): a status block (first 64 words) followed by one lock per
+// publication tile.  It lives in the library image, so every GPU that loads the library holds these
+// 65 792 bytes until the process exits.  Device code names the array directly; host code must not use
+// the name as an address (it is only a host-side stand-in) and asks cudaGetSymbolAddress() instead.
+constexpr int kNoAllocStatusWords = 64;
+constexpr int kNoAllocMaxTiles = 16384;
+static __device__ __align__(256) int32_t g_noalloc_scratch[kNoAllocStatusWords + kNoAllocMaxTiles];
+
+namespace iris {
+
+// Address of lock[t]: in the owner rank's heap slot, or (STATIC_LOCKS) in the library's static scratch.
+template <bool STATIC_LOCKS>
+__device__ __forceinline__ int32_t* lock_addr(const GemmParams& p, int rank, int t) {
+  if (STATIC_LOCKS) return &g_noalloc_scratch[kNoAllocStatusWords + t];
+  return reinterpret_cast<int32_t*>(p.tab.base[rank] + p.lock_off) + t;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Communication CTA (workgroup-specialised mode), Listing 5's `else` branch.
 //   warp 0: all 32 lanes watch 32 pending tiles' locks at once (one acquire-ordered load each);
@@ -136,6 +155,7 @@ __device__ __forceinline__ uint32_t pack2(uint32_t lo_bits, uint32_t hi_bits) {
 //   warp 1: waits for each buffer, issues the W-1 TMA stores (iris.put to every other rank), and once a
 //           store group has completed publishes the W ready flags.
 // ------------------------------------------------------------------------------------------------
+template <bool STATIC_LOCKS>
 __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload, int warp, int lane) {
   const int c = (int)blockIdx.x - p.gemm_ctas;
   const int W = p.tab.world;
@@ -154,7 +174,7 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
       if (widx >= 0) {
         t = c + widx * p.comm_ctas;
         rank = (t % pt_n) / p.ptiles_per_rank;
-        const int32_t* lock = reinterpret_cast<const int32_t*>(p.tab.base[rank] + p.lock_off) + t;
+        const int32_t* lock = lock_addr<STATIC_LOCKS>(p, rank, t);
         ready = ld_acquire_gpu(lock) == 1;
       }
       uint32_t mask = __ballot_sync(0xFFFFFFFFu, ready);
@@ -186,7 +206,7 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
           if (!mbar_wait(ptx::smem_u32(&ctrl->ring_free[slot]), par, p, ctrl, rt)) {
             fail = true;
           } else {
-            int32_t* lock = reinterpret_cast<int32_t*>(p.tab.base[rrank] + p.lock_off) + rt;
+            int32_t* lock = lock_addr<STATIC_LOCKS>(p, rrank, rt);
             (void)cas_acquire_gpu(lock, 1, 0);  // take the tile; the lock is ready for the next call
             fence_proxy_async();                // producer's generic-proxy stores -> our async-proxy read
             const int tm = rt / pt_n, pj = (rt % pt_n) % p.ptiles_per_rank;
@@ -246,7 +266,7 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
 // ------------------------------------------------------------------------------------------------
 // The GEMM + scatter kernel.
 // ------------------------------------------------------------------------------------------------
-template <int BN, bool BF16>
+template <int BN, bool BF16, bool STATIC_LOCKS = false>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const __grid_constant__ GemmParams p) {
   using Cfg = TileCfg<BN>;
   extern __shared__ uint8_t smem_raw[];
@@ -279,7 +299,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
   ptx::tc_fence_after();
 
   if (is_comm) {
-    comm_cta(p, ctrl, payload, warp, lane);
+    comm_cta<STATIC_LOCKS>(p, ctrl, payload, warp, lane);
   } else if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
@@ -403,7 +423,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
           if (pj < p.ptiles_per_rank) {
             const int t = tc.tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
             // Listing 5: tl.atomic_cas(locks + tile_id, 0, 1, sem="release", scope="gpu")
-            (void)cas_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[tc.rank] + p.lock_off) + t, 0, 1);
+            (void)cas_release_gpu(lock_addr<STATIC_LOCKS>(p, tc.rank, t), 0, 1);
           }
         }
       }
@@ -485,9 +505,9 @@ static int make_map(CUtensorMap* m, int dtype, int rank, void* base, const cuuin
   return IRIS_OK;
 }
 
-template <int BN, bool BF16>
+template <int BN, bool BF16, bool STATIC_LOCKS = false>
 static int launch_gemm(const GemmParams& p, int grid, bool cooperative, cudaStream_t st) {
-  auto kern = gemm_all_scatter_kernel<BN, BF16>;
+  auto kern = gemm_all_scatter_kernel<BN, BF16, STATIC_LOCKS>;
   static bool configured = false;
   if (!configured) {
     IRIS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal));
@@ -719,5 +739,108 @@ int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_h
       IRIS_CUDA_TRY(cudaMemcpyAsync(flags_host + (size_t)s * nt, heap->base + (size_t)s * heap->bytes_per_rank + flag_off, (size_t)nt * 4, cudaMemcpyDeviceToHost, st));
   return iris_status_check(heap, st, nullptr);
 }
+
+// The one entry point that allocates nothing (see the header).  Workgroup-specialised schedule with the
+// locks and the status block in g_noalloc_scratch.
+int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, const uint64_t* slot_bases, size_t bytes_per_rank, int M, int N,
+                                  int K, int world, int dtype, uint64_t c_off, uint64_t flag_off, int32_t epoch, void* stream) {
+  if (world < 1 || world > IRIS_MAX_WORLD) return fail(IRIS_ERR_ARG, "gemm_all_scatter_noalloc: world=%d not in [1,%d]", world, IRIS_MAX_WORLD);
+  if (!slot_bases) return fail(IRIS_ERR_ARG, "gemm_all_scatter_noalloc: slot_bases is NULL");
+  if (dtype != IRIS_F16 && dtype != IRIS_BF16) return fail(IRIS_ERR_ARG, "gemm_all_scatter_noalloc: unknown dtype %d", dtype);
+  if (M < 0 || N < 0 || K < 0 || N % world != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter_noalloc: bad M/N/K (N must be a multiple of world)");
+  const int nl = N / world;
+  if (nl % 8 != 0 || K % 8 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter_noalloc: N/world and K must be multiples of 8");
+  if (epoch < 1 || c_off % 256 != 0 || flag_off % 4 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter_noalloc: epoch must be >= 1, c_off %% 256 == 0, flag_off %% 4 == 0");
+  const int64_t nt = num_tiles(M, N, world);
+  if (nt > kNoAllocMaxTiles)
+    return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter_noalloc: %lld publication tiles exceed the static scratch limit of %d (use iris_gemm_all_scatter_ex with locks in the heap)",
+                (long long)nt, kNoAllocMaxTiles);
+  const uint64_t c_bytes = (uint64_t)M * N * 2;
+  if (c_off > bytes_per_rank || c_bytes > bytes_per_rank - c_off || flag_off > bytes_per_rank || (uint64_t)nt * 4 > bytes_per_rank - flag_off)
+    return fail(IRIS_ERR_RANGE, "gemm_all_scatter_noalloc: C or the flags leave the slot");
+  if (c_bytes && nt && c_off < flag_off + (uint64_t)nt * 4 && flag_off < c_off + c_bytes) return fail(IRIS_ERR_ARG, "gemm_all_scatter_noalloc: C and flag regions overlap");
+  for (int r = 0; r < world; ++r)
+    if (slot_bases[r] == 0 || slot_bases[r] % 256 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter_noalloc: slot_bases[%d] is NULL or not 256-byte aligned", r);
+  if (M == 0 || N == 0) return IRIS_OK;
+  if (K > 0) {
+    if (!A || (uint64_t)A % 16 != 0 || !B_shards) return fail(IRIS_ERR_ARG, "gemm_all_scatter_noalloc: A/B_shards NULL or A not 16-byte aligned");
+    for (int r = 0; r < world; ++r)
+      if (!B_shards[r] || (uint64_t)B_shards[r] % 16 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter_noalloc: B_shards[%d] is NULL or not 16-byte aligned", r);
+  }
+
+  // Set-up, once per device, with that device current: the device address of the static scratch.
+  static int32_t* scratch_of_device[64] = {nullptr};
+  int dev = -1, sms = 0;
+  IRIS_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter_noalloc: device ordinal %d not supported", dev);
+  if (!scratch_of_device[dev]) {
+    void* sym = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(&sym, g_noalloc_scratch);
+    if (e != cudaSuccess || !sym) return fail(IRIS_ERR_CUDA, "gemm_all_scatter_noalloc: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+    scratch_of_device[dev] = static_cast<int32_t*>(sym);
+  }
+  int32_t* scratch = scratch_of_device[dev];
+  IRIS_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+  if (sms < 2) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter_noalloc: needs at least 2 SMs");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // The array keeps the previous call's contents: the status block and the locks in use must start at zero.
+  IRIS_CUDA_TRY(cudaMemsetAsync(scratch, 0, (size_t)(kNoAllocStatusWords + nt) * 4, st));
+
+  GemmParams p;
+  std::memset(&p, 0, sizeof(p));
+  const int bn = (nl <= 128) ? 128 : ((nl % 256 == 0 || nl > 1024) ? 256 : 128);
+  for (int r = 0; r < world; ++r) p.tab.base[r] = slot_bases[r];
+  p.tab.bytes_per_rank = bytes_per_rank;
+  p.tab.world = world;
+  p.c_off = c_off;
+  p.flag_off = flag_off;
+  p.timeout_ns = kDefaultTimeoutNs;
+  p.status = scratch;
+  p.M = M; p.N = N; p.K = K; p.n_local = nl;
+  p.tiles_m = (M + BM - 1) / BM;
+  p.ctiles_per_rank = (nl + bn - 1) / bn;
+  p.ptiles_per_rank = (nl + IRIS_TILE - 1) / IRIS_TILE;
+  p.total_ctiles = p.tiles_m * world * p.ctiles_per_rank;
+  p.total_ptiles = p.tiles_m * world * p.ptiles_per_rank;
+  p.kblocks = (K + BK - 1) / BK;
+  p.raster_group = 16;
+  p.mode = IRIS_MODE_WORKGROUP_SPECIALIZED;
+  p.epoch = epoch;
+  p.comm_ctas = std::min(8, std::min(sms - 1, p.total_ptiles));
+  p.gemm_ctas = std::min(sms - p.comm_ctas, p.total_ctiles);
+  if (K > 0) {
+    const cuuint64_t dimsA[2] = {(cuuint64_t)K, (cuuint64_t)M};
+    const cuuint64_t strA[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t boxA[2] = {BK, BM};
+    int rc = make_map(&p.tmA, dtype, 2, const_cast<void*>(A), dimsA, strA, boxA, CU_TENSOR_MAP_SWIZZLE_128B, "A");
+    if (rc != IRIS_OK) return rc;
+    for (int r = 0; r < world; ++r) {
+      const cuuint64_t dimsB[2] = {(cuuint64_t)K, (cuuint64_t)nl};
+      const cuuint32_t boxB[2] = {BK, (cuuint32_t)bn};
+      rc = make_map(&p.tmB[r], dtype, 2, const_cast<void*>(B_shards[r]), dimsB, strA, boxB, CU_TENSOR_MAP_SWIZZLE_128B, "B");
+      if (rc != IRIS_OK) return rc;
+    }
+  }
+  for (int s = 0; s < world; ++s) {
+    const cuuint64_t dimsC[3] = {(cuuint64_t)nl, (cuuint64_t)M, (cuuint64_t)world};
+    const cuuint64_t strC[2] = {(cuuint64_t)N * 2, (cuuint64_t)nl * 2};
+    const cuuint32_t boxC[3] = {IRIS_TILE, IRIS_TILE, 1};
+    int rc = make_map(&p.tmC[s], dtype, 3, reinterpret_cast<void*>(slot_bases[s] + c_off), dimsC, strC, boxC, CU_TENSOR_MAP_SWIZZLE_NONE, "C");
+    if (rc != IRIS_OK) return rc;
+  }
+  const int grid = p.gemm_ctas + p.comm_ctas;
+  const bool bf = dtype == IRIS_BF16;
+  int rc;
+  if (bn == 256) rc = bf ? launch_gemm<256, true, true>(p, grid, true, st) : launch_gemm<256, false, true>(p, grid, true, st);
+  else           rc = bf ? launch_gemm<128, true, true>(p, grid, true, st) : launch_gemm<128, false, true>(p, grid, true, st);
+  if (rc != IRIS_OK) return rc;
+  IRIS_CUDA_TRY(cudaStreamSynchronize(st));
+  int32_t host_status[kStatusWords];
+  IRIS_CUDA_TRY(cudaMemcpy(host_status, scratch, sizeof(host_status), cudaMemcpyDeviceToHost));
+  if (host_status[0] != 0)
+    return fail(host_status[0], "gemm_all_scatter_noalloc: device-side wait expired: block=%d tile=%d", host_status[2], host_status[3]);
+  return IRIS_OK;
+}
+
 
 }  // extern "C"
