@@ -251,7 +251,7 @@ def run_ours(args):
     result = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world_size, "steps": args.steps, "warmup": args.warmup,
               "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if dtype == "bf16" else "f16",
               "data": "synthetic",
-              "config": {"workload": args.workload, "world": W, "M": M, "N": N, "K": K, "mode": args.mode, "comm_ctas": args.comm_ctas or 8,
+              "config": {"workload": args.workload, "world": W, "M": M, "N": N, "K": K, "mode": args.mode, "comm_ctas": args.comm_ctas or "auto",
                          "step": "gemm_all_scatter + flag-gated consumer (OUT = C + bias)", "accumulate": "fp32",
                          "l2": "inputs (0.8 GB) and outputs (4.3 GB) far exceed the 126 MB L2; no explicit flush",
                          "multi_gpu": "replicas only (ranks are emulated inside one GPU)"},

@@ -18,6 +18,7 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
+#include <cmath>
 #include <cstring>
 
 #include "iris_device.cuh"
@@ -30,8 +31,7 @@ constexpr int BK = 64;            // 64 x 16-bit = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;        // K of one tcgen05.mma for 16-bit inputs
 constexpr int kGemmThreads = 192;
 constexpr int kEpiThreads = 128;
-constexpr int kRing = 6;          // communication CTA: 32 KB tile buffers in flight
-constexpr int kRingLag = 4;       // store groups allowed in flight before the oldest is retired
+constexpr int kCommWarps = 6;     // communication CTA: every warp is a communicator with a 32 KB tile buffer
 constexpr int kTileBytes = IRIS_TILE * IRIS_TILE * 2;
 constexpr int kSmemPayload = 192 * 1024;
 constexpr int kSmemCtrl = 1024;
@@ -70,9 +70,7 @@ struct CtrlBlock {  // lives in shared memory after the payload area
   uint64_t empty[8];
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
-  uint64_t ring_full[kRing];
-  uint64_t ring_free[kRing];
-  int32_t ring_tile[kRing];
+  uint64_t comm_full[kCommWarps];
   uint32_t tmem_base;
   volatile int abort;
 };
@@ -149,117 +147,135 @@ __device__ __forceinline__ int32_t* lock_addr(const GemmParams& p, int rank, int
 
 // ------------------------------------------------------------------------------------------------
 // Communication CTA (workgroup-specialised mode), Listing 5's `else` branch.
-//   warp 0: all 32 lanes watch 32 pending tiles' locks at once (one acquire-ordered load each);
-//           a ballot collects the ready set, shuffles hand each ready tile id to lane 0, which takes
-//           the lock (cas 1->0, acquire) and issues the TMA load of the owner's tile into a ring buffer.
-//   warp 1: waits for each buffer, issues the W-1 TMA stores (iris.put to every other rank), and once a
-//           store group has completed publishes the W ready flags.
+// Each of the CTA's six warps is an independent communicator with its own 32 KB tile buffer and its own
+// mbarrier.  Work items are publication tiles numbered in the producers' raster order (item k = sub-tile
+// k % SUBS of compute tile k / SUBS), dealt round-robin to the communicator warps, so a warp sees its
+// tiles become ready roughly first-in first-out.
+//   poll     all 32 lanes watch 32 of the warp's pending items at once: one acquire-ordered load of
+//            lock[t] per lane; a ballot collects the ready set
+//   claim    the ready lanes take their locks together: cas(lock, 1 -> 0, acquire, gpu)
+//   copy     per ready tile (ids handed over by shuffles): lane 0 issues one TMA load of the owner's tile
+//            and, once it has landed, W-1 TMA stores from the same buffer (iris.put to every other rank),
+//            then waits until the stores have been performed
+//   publish  lanes 0..W-1 write the tile's ready flag in slot `lane` with release semantics
 // ------------------------------------------------------------------------------------------------
-template <bool STATIC_LOCKS>
+#ifdef IRIS_COMM_TRACE
+// Debug build only: per communicator warp {tiles, ns in: load, store issue, store wait, publish, idle poll, claim}.
+__device__ unsigned long long g_comm_trace[64 * 6 * 8];
+#define IRIS_TR(var) const uint64_t var = globaltimer_ns()
+#else
+#define IRIS_TR(var)
+#endif
+
+template <bool STATIC_LOCKS, int SUBS>
 __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload, int warp, int lane) {
-  const int c = (int)blockIdx.x - p.gemm_ctas;
+  constexpr uint32_t kFull = 0xFFFFFFFFu;
   const int W = p.tab.world;
-  const int n_my = (p.total_ptiles - c + p.comm_ctas - 1) / p.comm_ctas;  // tiles c, c+COMM, ...
+  const int ncw = p.comm_ctas * kCommWarps;
+  const int cw = ((int)blockIdx.x - p.gemm_ctas) * kCommWarps + warp;
+  const int items = p.total_ctiles * SUBS;
+  const int n_my = cw < items ? (items - cw + ncw - 1) / ncw : 0;  // items cw, cw + ncw, ...
   const int pt_n = W * p.ptiles_per_rank;
-  if (warp == 0) {
-    int widx = lane < n_my ? lane : -1;  // index into my tile list that this lane watches
-    int next = n_my < 32 ? n_my : 32;
-    int issued = 0;
-    uint64_t last_progress = globaltimer_ns();
-    uint32_t spins = 0;
-    bool ok = true;
-    while (ok && __any_sync(0xFFFFFFFFu, widx >= 0)) {
-      int t = -1, rank = 0;
-      bool ready = false;
-      if (widx >= 0) {
-        t = c + widx * p.comm_ctas;
-        rank = (t % pt_n) / p.ptiles_per_rank;
-        const int32_t* lock = lock_addr<STATIC_LOCKS>(p, rank, t);
-        ready = ld_acquire_gpu(lock) == 1;
-      }
-      uint32_t mask = __ballot_sync(0xFFFFFFFFu, ready);
-      if (mask == 0) {
-        if ((++spins & 15u) == 0) {
-          bool expired = false;
-          if (lane == 0) {
-            expired = ctrl->abort != 0;
-            if (!expired && globaltimer_ns() - last_progress > p.timeout_ns) {
-              report_timeout(p.status, KID_GEMM, t, -2, 0, 1);
-              ctrl->abort = 1;
-              expired = true;
-            }
-          }
-          if (__any_sync(0xFFFFFFFFu, expired)) ok = false;
-        }
-        continue;
-      }
-      const uint32_t ready_mask = mask;
-      while (mask) {
-        const int src = __ffs(mask) - 1;
-        mask &= mask - 1;
-        const int rt = __shfl_sync(0xFFFFFFFFu, t, src);
-        const int rrank = __shfl_sync(0xFFFFFFFFu, rank, src);
-        bool fail = false;
+  const uint32_t buf = ptx::smem_u32(payload + warp * kTileBytes);
+  const uint32_t bar = ptx::smem_u32(&ctrl->comm_full[warp]);
+  uint32_t bar_phase = 0;
+  int widx = lane < n_my ? lane : -1;  // index into this warp's item list that this lane watches
+  int next = n_my < 32 ? n_my : 32;
+  uint64_t last_progress = globaltimer_ns();
+#ifdef IRIS_COMM_TRACE
+  uint64_t last_poll = last_progress;
+#endif
+  uint32_t spins = 0;
+  bool ok = true;
+  // item -> publication tile, recomputed only when the lane moves to a new item
+  // (t < 0 with widx >= 0: the compute tile has no such sub-tile; nothing to do)
+  int t = -1, rank = 0;
+  auto assign = [&]() {
+    t = -1;
+    if (widx < 0) return;
+    const int k = cw + widx * ncw;
+    const TileCoord tc = decode_ctile(k / SUBS, p);
+    const int pj = tc.jn * SUBS + k % SUBS;
+    rank = tc.rank;
+    if (pj < p.ptiles_per_rank) t = tc.tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
+  };
+  assign();
+  while (ok && __any_sync(kFull, widx >= 0)) {
+    bool ready = false;
+    if (widx >= 0) ready = t < 0 || ld_acquire_gpu(lock_addr<STATIC_LOCKS>(p, rank, t)) == 1;
+    const uint32_t mask = __ballot_sync(kFull, ready);
+#ifdef IRIS_COMM_TRACE
+    unsigned long long* tr = &g_comm_trace[(size_t)cw * 8];
+    if (lane == 0 && mask == 0) { const uint64_t now = globaltimer_ns(); tr[5] += now - last_poll; last_poll = now; }
+#endif
+    if (mask == 0) {
+      if ((++spins & 15u) == 0) {
+        bool expired = false;
         if (lane == 0) {
-          const int slot = issued % kRing;
-          const uint32_t par = ((issued / kRing) & 1) ^ 1;
-          if (!mbar_wait(ptx::smem_u32(&ctrl->ring_free[slot]), par, p, ctrl, rt)) {
-            fail = true;
-          } else {
-            int32_t* lock = lock_addr<STATIC_LOCKS>(p, rrank, rt);
-            (void)cas_acquire_gpu(lock, 1, 0);  // take the tile; the lock is ready for the next call
-            fence_proxy_async();                // producer's generic-proxy stores -> our async-proxy read
-            const int tm = rt / pt_n, pj = (rt % pt_n) % p.ptiles_per_rank;
-            ctrl->ring_tile[slot] = rt;
-            const uint32_t bar = ptx::smem_u32(&ctrl->ring_full[slot]);
-            ptx::mbar_arrive_expect_tx(bar, kTileBytes);
-            ptx::tma_load_3d(ptx::smem_u32(payload + slot * kTileBytes), &p.tmC[rrank], pj * IRIS_TILE, tm * IRIS_TILE, rrank, bar);
+          expired = ctrl->abort != 0;
+          if (!expired && globaltimer_ns() - last_progress > p.timeout_ns) {
+            report_timeout(p.status, KID_GEMM, t, -2, 0, 1);
+            ctrl->abort = 1;
+            expired = true;
           }
         }
-        ++issued;
-        if (__any_sync(0xFFFFFFFFu, fail)) { ok = false; break; }
+        if (__any_sync(kFull, expired)) ok = false;
       }
-      // lanes whose tile was taken move on to the next unwatched tiles, in lane order
-      const int rank_in_mask = __popc(ready_mask & ((1u << lane) - 1u));
-      if (ready_mask & (1u << lane)) {
-        const int cand = next + rank_in_mask;
-        widx = cand < n_my ? cand : -1;
-      }
-      next = min(n_my, next + __popc(ready_mask));
-      last_progress = globaltimer_ns();
+      continue;
     }
-  } else if (warp == 1) {
-    int done = 0;  // tiles whose flags have been published
-    bool ok = true;
-    auto publish = [&](int i) {
-      const int slot = i % kRing;
-      const int rt = ctrl->ring_tile[slot];
-      __syncwarp();
-      if (lane < W) st_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[lane] + p.flag_off) + rt, p.epoch);
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->ring_free[slot]));
-    };
-    for (int i = 0; i < n_my && ok; ++i) {
-      const int slot = i % kRing;
+    // Listing 5: tl.atomic_cas(locks + tile_id, 1, 0, sem="acquire", scope="gpu"); all ready lanes at once.
+    IRIS_TR(tc0);
+    if (ready && t >= 0) (void)cas_acquire_gpu(lock_addr<STATIC_LOCKS>(p, rank, t), 1, 0);
+    __syncwarp();
+#ifdef IRIS_COMM_TRACE
+    if (lane == 0) tr[6] += globaltimer_ns() - tc0;
+#endif
+    uint32_t todo = mask;
+    while (todo) {
+      const int src = __ffs(todo) - 1;
+      todo &= todo - 1;
+      const int rt = __shfl_sync(kFull, t, src);
+      const int rrank = __shfl_sync(kFull, rank, src);
+      if (rt < 0) continue;
+      const int tm = rt / pt_n, pj = (rt % pt_n) % p.ptiles_per_rank;
       bool fail = false;
+      IRIS_TR(t0);
       if (lane == 0) {
-        if (!mbar_wait(ptx::smem_u32(&ctrl->ring_full[slot]), (i / kRing) & 1, p, ctrl, -3)) {
+        fence_proxy_async();  // producers' generic-proxy stores (acquired above) -> our async-proxy read
+        ptx::mbar_arrive_expect_tx(bar, kTileBytes);
+        ptx::tma_load_3d(buf, &p.tmC[rrank], pj * IRIS_TILE, tm * IRIS_TILE, rrank, bar);
+        if (!mbar_wait(bar, bar_phase, p, ctrl, rt)) {
           fail = true;
         } else {
-          const int rt = ctrl->ring_tile[slot];
-          const int tm = rt / pt_n, rrank = (rt % pt_n) / p.ptiles_per_rank, pj = (rt % pt_n) % p.ptiles_per_rank;
+          IRIS_TR(t1);
           for (int s = 0; s < W; ++s)
-            if (s != rrank) ptx::tma_store_3d(&p.tmC[s], pj * IRIS_TILE, tm * IRIS_TILE, rrank, ptx::smem_u32(payload + slot * kTileBytes));
+            if (s != rrank) ptx::tma_store_3d(&p.tmC[s], pj * IRIS_TILE, tm * IRIS_TILE, rrank, buf);
           ptx::bulk_commit_group();
-          if (i >= kRingLag) ptx::bulk_wait_group<kRingLag>();
+          IRIS_TR(t2);
+          ptx::bulk_wait_group<0>();  // stores performed: the buffer is free and the tile may be published
+#ifdef IRIS_COMM_TRACE
+          const uint64_t t3 = globaltimer_ns();
+          tr[0] += 1; tr[1] += t1 - t0; tr[2] += t2 - t1; tr[3] += t3 - t2;
+#endif
         }
       }
-      if (__any_sync(0xFFFFFFFFu, fail)) { ok = false; break; }
-      if (i >= kRingLag) { publish(done); ++done; }
+      bar_phase ^= 1;
+      if (__any_sync(kFull, fail)) { ok = false; break; }
+      IRIS_TR(t4);
+      if (lane < W) st_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[lane] + p.flag_off) + rt, p.epoch);
+      __syncwarp();
+#ifdef IRIS_COMM_TRACE
+      if (lane == 0) { tr[4] += globaltimer_ns() - t4; last_poll = globaltimer_ns(); }
+#endif
     }
-    if (lane == 0) ptx::bulk_wait_group<0>();  // also on the failure path: no copy of ours stays in flight
-    __syncwarp();
-    if (ok) while (done < n_my) { publish(done); ++done; }
+    // lanes whose item was handled move on to the next unwatched items, in lane order
+    if (mask & (1u << lane)) {
+      const int cand = next + __popc(mask & ((1u << lane) - 1u));
+      widx = cand < n_my ? cand : -1;
+      assign();
+    }
+    next = min(n_my, next + __popc(mask));
+    last_progress = globaltimer_ns();
   }
 }
 
@@ -279,7 +295,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
   if (threadIdx.x == 0) {
     for (int i = 0; i < Cfg::kStages; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->empty[i]), 1); }
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i]), 4); }
-    for (int i = 0; i < kRing; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->ring_full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->ring_free[i]), 1); }
+    for (int i = 0; i < kCommWarps; ++i) ptx::mbar_init(ptx::smem_u32(&ctrl->comm_full[i]), 1);
     ctrl->abort = 0;
     ptx::fence_mbar_init();
     fence_proxy_async();
@@ -299,7 +315,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
   ptx::tc_fence_after();
 
   if (is_comm) {
-    comm_cta<STATIC_LOCKS>(p, ctrl, payload, warp, lane);
+    comm_cta<STATIC_LOCKS, BN / IRIS_TILE>(p, ctrl, payload, warp, lane);
   } else if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
@@ -527,6 +543,20 @@ static int launch_gemm(const GemmParams& p, int grid, bool cooperative, cudaStre
   return IRIS_OK;
 }
 
+// How many CTAs to reserve for communication when the caller does not say.  A communication CTA moves
+// one tile read plus W-1 tile writes per publication tile; one SM sustains about 55 GB/s of such TMA
+// traffic while the other SMs run the GEMM (measured with per-phase %globaltimer stamps in the
+// communicator warps).  The split c : (S - c) that lets both sides finish together solves
+// c / (S - c) = x with x = (communication SM-seconds) / (GEMM SM-seconds); a 35 % margin covers the
+// tail, where the last tiles become ready only when the GEMM ends.
+static int auto_comm_ctas(int M, int N, int K, int W, int sms) {
+  const double bytes = (double)W * M * N * 2.0;
+  const double t_gemm = std::max(2.0 * M * N * (double)K / 1.45e15, ((double)M * K + (double)N * K) * 2.0 / 6.0e12);
+  const double x = 1.35 * (bytes / 55e9) / (t_gemm * sms + 1e-12);
+  int c = (int)std::ceil(sms * x / (1.0 + x));
+  return std::max(4, std::min(c, sms / 3));
+}
+
 int64_t num_tiles(int M, int N, int world) {
   if (M < 0 || N < 0 || world < 1 || world > IRIS_MAX_WORLD || N % world != 0) return -1;
   const int64_t nl = N / world;
@@ -608,7 +638,7 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   int grid = a->max_ctas ? std::min(a->max_ctas, h->sm_count) : h->sm_count;
   if (wg) {
     if (grid < 2) return fail(IRIS_ERR_ARG, "gemm_all_scatter: workgroup_specialized needs at least 2 CTAs");
-    int comm = a->comm_ctas ? a->comm_ctas : 8;
+    int comm = a->comm_ctas ? a->comm_ctas : auto_comm_ctas(a->M, a->N, a->K, W, grid);
     comm = std::min(comm, std::min(grid - 1, p.total_ptiles));
     p.comm_ctas = comm;
     p.gemm_ctas = std::min(grid - comm, p.total_ctiles);
@@ -806,7 +836,7 @@ int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, co
   p.raster_group = 16;
   p.mode = IRIS_MODE_WORKGROUP_SPECIALIZED;
   p.epoch = epoch;
-  p.comm_ctas = std::min(8, std::min(sms - 1, p.total_ptiles));
+  p.comm_ctas = std::min(auto_comm_ctas(M, N, K, world, sms), std::min(sms - 1, p.total_ptiles));
   p.gemm_ctas = std::min(sms - p.comm_ctas, p.total_ctiles);
   if (K > 0) {
     const cuuint64_t dimsA[2] = {(cuuint64_t)K, (cuuint64_t)M};
@@ -842,5 +872,14 @@ int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, co
   return IRIS_OK;
 }
 
+
+#ifdef IRIS_COMM_TRACE
+int iris_debug_comm_trace(unsigned long long* host_out, int clear) {
+  cudaDeviceSynchronize();
+  if (host_out) cudaMemcpyFromSymbol(host_out, g_comm_trace, sizeof(g_comm_trace));
+  if (clear) { static unsigned long long z[64 * 6 * 8]; cudaMemcpyToSymbol(g_comm_trace, z, sizeof(z)); }
+  return 0;
+}
+#endif
 
 }  // extern "C"

@@ -1,0 +1,86 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times.
+
+The oracle cannot finish a 4.4 TFLOP fp64 GEMM, so values are checked on a seeded sample of publication tiles
+(each computed by the oracle from the same seeded inputs), while replication (all W copies byte-identical),
+flags, locks and the consumer's output are checked at full size on the device (they are memcmp / scans).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2511_12500_b200 as iris
+from paper_2511_12500_b200 import inputs
+from gpu_util import check_tolerance
+
+pytestmark = pytest.mark.gpu
+
+
+def align(x, a=256):
+    return (x + a - 1) // a * a
+
+
+def _run_fullsize(W, M, N, K, dist, dtype, mode, seed, n_sample, comm_ctas=0, with_consumer=True):
+    nl = N // W
+    nt = iris.iris_num_tiles(M, N, W)
+    flag_off = align(M * N * 2)
+    lock_off = flag_off + align(nt * 4)
+    out_off = iris.iris_gemm_out_offset(M, N, W)
+    bpr = align(out_off + M * N * 2)
+    A, Bs = inputs.gemm_inputs(seed, W, M, N, K, dist, dtype)
+    bias = inputs.vector(seed, inputs.STREAM_BIAS, N, "uniform", dtype)
+    dA = torch.from_numpy(A.view(np.int16)).cuda()
+    dB = [torch.from_numpy(b.view(np.int16)).cuda() for b in Bs]
+    dbias = torch.from_numpy(bias.view(np.int16)).cuda()
+    mem = torch.full((W * bpr,), 0xFF, dtype=torch.uint8, device="cuda")      # NaN poison
+    h = iris.iris_heap_create(W, bpr, external_base=mem.data_ptr())
+    try:
+        iris.iris_flags_fill(h, flag_off, nt, 0)
+        iris.iris_flags_fill(h, lock_off, nt, 0)
+        for epoch in (1, 2):           # the second pass runs over the first one's data, as the timed loop does
+            iris.iris_gemm_all_scatter_ex(h, dA, dB, M, N, K, W, iris.MODES[mode], iris.DTYPES[dtype], 0, flag_off, lock_off, epoch,
+                                          comm_ctas=comm_ctas)
+            if with_consumer:
+                iris.iris_consume_bias(h, 0, out_off, flag_off, dbias, M, N, W, iris.DTYPES[dtype], epoch)
+            iris.iris_status_check(h)
+        slots = mem.view(W, bpr)
+        c0 = slots[0, : M * N * 2]
+        for s in range(1, W):                                       # replication: all W copies byte-identical
+            assert torch.equal(slots[s, : M * N * 2], c0), f"slot {s} differs from slot 0"
+            if with_consumer:
+                assert torch.equal(slots[s, out_off: out_off + M * N * 2], slots[0, out_off: out_off + M * N * 2])
+        for s in range(W):                                          # flags == epoch, locks consumed, everywhere
+            assert bool(torch.all(slots[s, flag_off: flag_off + nt * 4].view(torch.int32) == 2))
+            assert bool(torch.all(slots[s, lock_off: lock_off + nt * 4].view(torch.int32) == 0))
+        c_host = c0.view(torch.int16).view(M, N)
+        out_host = slots[0, out_off: out_off + M * N * 2].view(torch.int16).view(M, N)
+        rng = np.random.default_rng(seed)
+        tiles = sorted(set([0, nt - 1] + [int(t) for t in rng.choice(nt, size=min(n_sample, nt), replace=False)]))
+        for t in tiles:
+            m0, m1, n0, n1 = oracle.tile_rect(t, M, N, W)
+            r = n0 // nl
+            ref = oracle.gemm_block(A[m0:m1], [Bs[r][n0 - r * nl: n1 - r * nl]], dtype)
+            got = c_host[m0:m1, n0:n1].cpu().numpy().view(np.uint16)
+            check_tolerance(got, ref, dtype)
+            if with_consumer:                                       # consumer: bit-exact on the GPU's own C
+                exp = oracle.consume_bias_rows(np.ascontiguousarray(got), bias[n0:n1], dtype)
+                assert np.array_equal(out_host[m0:m1, n0:n1].cpu().numpy().view(np.uint16), exp)
+    finally:
+        iris.iris_heap_destroy(h)
+
+
+def test_bench_workload_workgroup_specialized_sampled_tiles():
+    """W=8, M=8192, N=K=16384, bf16 uniform[-1,1): the workload and schedule bench.py reports."""
+    _run_fullsize(8, 8192, 16384, 16384, "uniform", "bf16", "workgroup_specialized", inputs.SEED0 + 4, n_sample=10)
+
+
+@pytest.mark.parametrize("mode", ["bulk_synchronous", "fused_sequential"])
+def test_config3_sampled_tiles(mode):
+    """W=8, M=4096, N=8192, K=8192, bf16 normal(0, 0.02)."""
+    _run_fullsize(8, 4096, 8192, 8192, "normal002", "bf16", mode, inputs.SEED0 + 2, n_sample=8)
+
+
+@pytest.mark.parametrize("comm_ctas", [8, 32])
+def test_config4_skinny_workgroup_specialized(comm_ctas):
+    """W=8, M=128, N=28672, K=8192, bf16 normal(0, 0.02): the memory-bound decode-like shape."""
+    _run_fullsize(8, 128, 28672, 8192, "normal002", "bf16", "workgroup_specialized", inputs.SEED0 + 3, n_sample=12, comm_ctas=comm_ctas)
