@@ -205,7 +205,7 @@ def run_ours(args):
 
     def gemm(epoch, m=mode, **kw):
         iris.iris_gemm_all_scatter_ex(h, dA, dB, M, N, K, W, m, dt, 0, flag_off, lock_off, epoch, comm_ctas=args.comm_ctas,
-                                      raster_group=args.raster_group, block_n=args.block_n, **kw)
+                                      raster_group=args.raster_group, block_n=args.block_n, cta_pair=args.cta_pair, **kw)
 
     def consume(epoch):
         iris.iris_consume_bias(h, 0, out_off, flag_off, dbias, M, N, W, dt, epoch)
@@ -389,6 +389,7 @@ def main():
     ap.add_argument("--comm-ctas", type=int, default=0)
     ap.add_argument("--raster-group", type=int, default=0)
     ap.add_argument("--block-n", type=int, default=0)
+    ap.add_argument("--cta-pair", type=int, default=0)
     ap.add_argument("--mode-iters", type=int, default=3)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-strips", type=int, default=16)

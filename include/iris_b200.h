@@ -197,6 +197,9 @@ typedef struct iris_gemm_args {
   int raster_group;            /* tile rows per raster group for L2 reuse (0 = 16)               */
   int block_n;                 /* compute-tile width: 0 = auto, 128 or 256                       */
   uint64_t spin_timeout_ns;    /* deadline of every device-side wait (0 = 2 s)                   */
+  int cta_pair;                /* 0 = use 256 x 256 CTA-pair tiles (tcgen05 cta_group::2) when
+                                  (N/world) % 256 == 0 and M > 128; 1 = require them
+                                  (IRIS_ERR_UNSUPPORTED otherwise); -1 = single-CTA tiles only   */
 } iris_gemm_args;
 
 /* Enqueue the whole operation on `stream` (bulk-synchronous: two kernels; otherwise one).
@@ -270,7 +273,8 @@ uint64_t iris_gemm_out_offset(int M, int N, int world);
  * wait ran out).  All calls share the one array: two calls whose GPU work overlaps (different
  * streams, different host threads) race on it and must be serialised by the caller.
  * Other arguments, checks, layout and results are those of iris_gemm_all_scatter_ex in
- * IRIS_MODE_WORKGROUP_SPECIALIZED with default tuning; the results are bit-identical to it. */
+ * IRIS_MODE_WORKGROUP_SPECIALIZED with single-CTA tiles (cta_pair = -1) and default tuning; the
+ * results are bit-identical to that call's. */
 int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, const uint64_t* slot_bases,
                                   size_t bytes_per_rank, int M, int N, int K, int world, int dtype, uint64_t c_off,
                                   uint64_t flag_off, int32_t epoch, void* stream);

@@ -59,6 +59,7 @@ struct alignas(64) GemmParams {
   int total_ctiles;     // tiles_m * W * ctiles_per_rank
   int total_ptiles;     // tiles_m * W * ptiles_per_rank
   int kblocks;          // ceil(K / 64)
+  int ptiles_m;         // publication tile rows: ceil(M / 128)
   int gemm_ctas, comm_ctas;
   int raster_group;
   int mode;
@@ -149,7 +150,7 @@ __device__ __forceinline__ int32_t* lock_addr(const GemmParams& p, int rank, int
 // Communication CTA (workgroup-specialised mode), Listing 5's `else` branch.
 // Each of the CTA's six warps is an independent communicator with its own 32 KB tile buffer and its own
 // mbarrier.  Work items are publication tiles numbered in the producers' raster order (item k = sub-tile
-// k % SUBS of compute tile k / SUBS), dealt round-robin to the communicator warps, so a warp sees its
+// k % SUBS of compute tile k / SUBS; a CTA pair's 256-row tile has SUBS_M = 2 rows of them), dealt round-robin to the communicator warps, so a warp sees its
 // tiles become ready roughly first-in first-out.
 //   poll     all 32 lanes watch 32 of the warp's pending items at once: one acquire-ordered load of
 //            lock[t] per lane; a ballot collects the ready set
@@ -167,13 +168,13 @@ __device__ unsigned long long g_comm_trace[64 * 6 * 8];
 #define IRIS_TR(var)
 #endif
 
-template <bool STATIC_LOCKS, int SUBS>
+template <bool STATIC_LOCKS, int SUBS, int SUBS_M = 1>
 __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload, int warp, int lane) {
   constexpr uint32_t kFull = 0xFFFFFFFFu;
   const int W = p.tab.world;
   const int ncw = p.comm_ctas * kCommWarps;
   const int cw = ((int)blockIdx.x - p.gemm_ctas) * kCommWarps + warp;
-  const int items = p.total_ctiles * SUBS;
+  const int items = p.total_ctiles * SUBS * SUBS_M;
   const int n_my = cw < items ? (items - cw + ncw - 1) / ncw : 0;  // items cw, cw + ncw, ...
   const int pt_n = W * p.ptiles_per_rank;
   const uint32_t buf = ptx::smem_u32(payload + warp * kTileBytes);
@@ -194,10 +195,12 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
     t = -1;
     if (widx < 0) return;
     const int k = cw + widx * ncw;
-    const TileCoord tc = decode_ctile(k / SUBS, p);
-    const int pj = tc.jn * SUBS + k % SUBS;
+    const TileCoord tc = decode_ctile(k / (SUBS * SUBS_M), p);
+    const int sub = k % (SUBS * SUBS_M);
+    const int pj = tc.jn * SUBS + sub % SUBS;
+    const int tm = tc.tm * SUBS_M + sub / SUBS;  // publication tile row
     rank = tc.rank;
-    if (pj < p.ptiles_per_rank) t = tc.tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
+    if (pj < p.ptiles_per_rank && tm < p.ptiles_m) t = tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
   };
   assign();
   while (ok && __any_sync(kFull, widx >= 0)) {
@@ -455,6 +458,190 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
 }
 
 // ------------------------------------------------------------------------------------------------
+// CTA-pair variant: a cluster of two CTAs (one TPC) computes a 256 x 256 tile with tcgen05 cta_group::2.
+// CTA r of the pair owns rows [128 r, 128 r + 128) of the tile: it TMA-loads its own 128 x 64 slice of A
+// and its own half (128 of the 256 columns) of the B tile -- no multicast, every CTA fetches only what
+// it keeps -- and the leader's MMA thread issues one 256 x 256 x 16 instruction for both: each SM's
+// tensor core reads its A slice locally and both B halves.  Per CTA and k-step 32 KB are staged instead
+// of 48 KB for the same flops per SM, which is what the single-CTA kernel's shared-memory port cannot
+// afford.  Accumulators: 2 x 256 columns of TMEM in each CTA (rows of its own half).
+//   full[s]        leader only; the leader's producer expects 64 KB, all four loads (two per CTA) complete on it
+//   empty[s]       both CTAs; the leader's tcgen05.commit multicasts the arrival to the pair
+//   tmem_full[a]   both CTAs; multicast commit after a tile's last MMA
+//   tmem_empty[a]  leader only; 8 arrivals = 4 epilogue warps x 2 CTAs (the peer's arrive remotely)
+// ------------------------------------------------------------------------------------------------
+constexpr int kPairStageBytes = 2 * BM * BK * 2;            // 32 KB: A slice + B half
+constexpr int kPairStages = kSmemPayload / kPairStageBytes;  // 6
+constexpr int kPairBN = 256;
+
+template <bool BF16, bool STATIC_LOCKS = false>
+__global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_pair_kernel(const __grid_constant__ GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* payload = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  CtrlBlock* ctrl = reinterpret_cast<CtrlBlock*>(payload + kSmemPayload);
+  const int warp = (int)threadIdx.x / 32, lane = (int)threadIdx.x % 32;
+  const int cta_rank = (int)ptx::cluster_ctarank();
+  const bool leader = cta_rank == 0;
+  const bool is_comm = (int)blockIdx.x >= p.gemm_ctas;   // gemm_ctas is even: a pair is never split
+  const int pair_id = (int)blockIdx.x >> 1, gemm_pairs = p.gemm_ctas >> 1;
+  const int W = p.tab.world;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kPairStages; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->empty[i]), 1); }
+    for (int i = 0; i < 2; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i]), 8); }
+    for (int i = 0; i < kCommWarps; ++i) ptx::mbar_init(ptx::smem_u32(&ctrl->comm_full[i]), 1);
+    ctrl->abort = 0;
+    ptx::fence_mbar_init();
+    fence_proxy_async();
+    if (p.kblocks > 0 && !is_comm) {
+      ptx::prefetch_tensormap(&p.tmA);
+      for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmB[r]);
+    }
+    if (is_comm)
+      for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmC[r]);
+  }
+  if (warp == 1 && !is_comm) {
+    ptx::tmem_alloc_pair(ptx::smem_u32(&ctrl->tmem_base), 2 * kPairBN);
+    ptx::tmem_relinquish_pair();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync();   // the peer's barriers exist before anything of ours can signal them
+  ptx::tc_fence_after();
+
+  if (is_comm) {
+    comm_cta<STATIC_LOCKS, kPairBN / IRIS_TILE, 2>(p, ctrl, payload, warp, lane);
+  } else if (warp == 0) {
+    // ---------------- TMA producer (both CTAs) ----------------
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = pair_id; tile < p.total_ctiles && ok; tile += gemm_pairs) {
+        const TileCoord tc = decode_ctile(tile, p);
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!mbar_wait(ptx::smem_u32(&ctrl->empty[stage]), phase ^ 1, p, ctrl, tile)) { ok = false; break; }
+          const uint32_t full_local = ptx::smem_u32(&ctrl->full[stage]);
+          if (leader) ptx::mbar_arrive_expect_tx(full_local, 2 * kPairStageBytes);
+          const uint32_t full_leader = ptx::mapa(full_local, 0);
+          const uint32_t sa = ptx::smem_u32(payload + stage * kPairStageBytes);
+          ptx::tma_load_2d_pair(sa, &p.tmA, kb * BK, tc.tm * 2 * BM + cta_rank * BM, full_leader);
+          ptx::tma_load_2d_pair(sa + BM * BK * 2, &p.tmB[tc.rank], kb * BK, tc.jn * kPairBN + cta_rank * (kPairBN / 2), full_leader);
+          if (++stage == kPairStages) { stage = 0; phase ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer (leader CTA only) ----------------
+    if (lane == 0 && leader) {
+      constexpr uint32_t idesc = ptx::idesc_f16(2 * BM, kPairBN, BF16 ? 1 : 0);
+      const uint32_t tmem_base = ctrl->tmem_base;
+      int stage = 0, acc = 0;
+      uint32_t phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (int tile = pair_id; tile < p.total_ctiles && ok; tile += gemm_pairs) {
+        if (!mbar_wait(ptx::smem_u32(&ctrl->tmem_empty[acc]), acc_phase ^ 1, p, ctrl, tile)) break;
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kPairBN);
+        for (int kb = 0; kb < p.kblocks; ++kb) {
+          if (!mbar_wait(ptx::smem_u32(&ctrl->full[stage]), phase, p, ctrl, tile)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint32_t sa = ptx::smem_u32(payload + stage * kPairStageBytes);
+          const uint64_t adesc = ptx::smem_desc_k_sw128(sa);
+          const uint64_t bdesc = ptx::smem_desc_k_sw128(sa + BM * BK * 2);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k)
+            ptx::mma_f16_ss_pair(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+          ptx::mma_commit_pair(ptx::smem_u32(&ctrl->empty[stage]), 3);  // both CTAs may refill this stage
+          if (++stage == kPairStages) { stage = 0; phase ^= 1; }
+        }
+        if (!ok) break;
+        ptx::mma_commit_pair(ptx::smem_u32(&ctrl->tmem_full[acc]), 3);  // accumulator complete in both CTAs
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      }
+    }
+  } else {
+    // ---------------- epilogue: warps 2..5 of both CTAs, each CTA drains its own 128 rows ----------------
+    const int quad = warp & 3;
+    const int et = (int)threadIdx.x - 64;
+    int acc = 0;
+    uint32_t acc_phase = 0;
+    const uint32_t tmem_base = ctrl->tmem_base;
+    for (int tile = pair_id; tile < p.total_ctiles; tile += gemm_pairs) {
+      const TileCoord tc = decode_ctile(tile, p);
+      const bool ok = mbar_wait(ptx::smem_u32(&ctrl->tmem_full[acc]), acc_phase, p, ctrl, tile);
+      if (ptx::bar_red_or(1, kEpiThreads, !ok)) break;
+      ptx::tc_fence_after();
+      const int tm = tc.tm * 2 + cta_rank;  // publication tile row of this CTA's half
+      const int row = tm * BM + quad * 32 + lane;
+      const int col_in_shard = tc.jn * kPairBN;
+      const uint64_t row_off = p.c_off + ((uint64_t)row * p.N + (uint64_t)tc.rank * p.n_local) * 2;
+#pragma unroll 1
+      for (int ch = 0; ch < kPairBN / 32; ++ch) {
+        uint32_t v[32];
+        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kPairBN + ch * 32), v);
+        ptx::tmem_wait_ld();
+        uint4 q[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          if (p.kblocks == 0) {
+            q[i] = make_uint4(0, 0, 0, 0);
+          } else {
+            q[i].x = pack2<BF16>(v[8 * i + 0], v[8 * i + 1]);
+            q[i].y = pack2<BF16>(v[8 * i + 2], v[8 * i + 3]);
+            q[i].z = pack2<BF16>(v[8 * i + 4], v[8 * i + 5]);
+            q[i].w = pack2<BF16>(v[8 * i + 6], v[8 * i + 7]);
+          }
+        }
+        if (row < p.M) {
+          const int c0 = col_in_shard + ch * 32;
+          if (p.mode == IRIS_MODE_FUSED_SEQUENTIAL) {
+            for (int s = 0; s < W; ++s) {
+              const uint64_t dst = p.tab.base[s] + row_off + (uint64_t)c0 * 2;
+#pragma unroll
+              for (int i = 0; i < 4; ++i) st_global_v4(reinterpret_cast<void*>(dst + 16 * i), q[i]);
+            }
+          } else {
+            const uint64_t dst = p.tab.base[tc.rank] + row_off + (uint64_t)c0 * 2;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) st_global_v4(reinterpret_cast<void*>(dst + 16 * i), q[i]);
+          }
+        }
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&ctrl->tmem_empty[acc]), 0));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      if (p.mode != IRIS_MODE_BULK_SYNCHRONOUS) {
+        asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
+        constexpr int subs = kPairBN / IRIS_TILE;
+        const int pt_n = W * p.ptiles_per_rank;
+        if (tm < p.ptiles_m) {
+          if (p.mode == IRIS_MODE_FUSED_SEQUENTIAL) {
+            if (et < subs * W) {
+              const int sub = et / W, s = et % W;
+              const int t = tm * pt_n + tc.rank * p.ptiles_per_rank + tc.jn * subs + sub;
+              st_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[s] + p.flag_off) + t, p.epoch);
+            }
+          } else if (et < subs) {
+            const int t = tm * pt_n + tc.rank * p.ptiles_per_rank + tc.jn * subs + et;
+            (void)cas_release_gpu(lock_addr<STATIC_LOCKS>(p, tc.rank, t), 0, 1);
+          }
+        }
+      }
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::cluster_sync();   // the leader's MMAs read the peer's shared memory and both write both TMEMs: leave together
+  if (warp == 1 && !is_comm) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc_pair(ctrl->tmem_base, 2 * kPairBN);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Bulk-synchronous second kernel (Listing 3, all_scatter): per publication tile, iris.put the owner's
 // tile to every other rank, then publish the W ready flags.
 // ------------------------------------------------------------------------------------------------
@@ -543,6 +730,34 @@ static int launch_gemm(const GemmParams& p, int grid, bool cooperative, cudaStre
   return IRIS_OK;
 }
 
+template <bool BF16, bool STATIC_LOCKS = false>
+static int launch_gemm_pair(const GemmParams& p, int grid, cudaStream_t st, int* max_pairs_out) {
+  auto kern = gemm_all_scatter_pair_kernel<BF16, STATIC_LOCKS>;
+  static bool configured = false;
+  if (!configured) {
+    IRIS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal));
+    configured = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)(max_pairs_out ? 2 : grid));
+  cfg.blockDim = dim3(kGemmThreads);
+  cfg.dynamicSmemBytes = kSmemTotal;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (max_pairs_out) {  // query only: how many pairs can be resident at once
+    IRIS_CUDA_TRY(cudaOccupancyMaxActiveClusters(max_pairs_out, kern, &cfg));
+    return IRIS_OK;
+  }
+  IRIS_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, p));
+  return IRIS_OK;
+}
+
 // How many CTAs to reserve for communication when the caller does not say.  A communication CTA moves
 // one tile read plus W-1 tile writes per publication tile; one SM sustains about 55 GB/s of such TMA
 // traffic while the other SMs run the GEMM (measured with per-phase %globaltimer stamps in the
@@ -597,6 +812,7 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   if (a->epoch < 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: epoch must be >= 1");
   if (a->c_off % 256 != 0 || a->flag_off % 4 != 0 || a->lock_off % 4 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: misaligned heap offsets");
   if (a->comm_ctas < 0 || a->max_ctas < 0 || a->raster_group < 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: negative tuning parameter");
+  if (a->cta_pair < -1 || a->cta_pair > 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: cta_pair must be -1, 0 or 1");
   const int64_t nt = num_tiles(a->M, a->N, W);
   const uint64_t bpr = h->bytes_per_rank;
   const uint64_t c_bytes = (uint64_t)a->M * a->N * 2;
@@ -619,6 +835,21 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   int bn = a->block_n;
   if (bn == 0) bn = (nl % 256 == 0 || nl > 1024) ? 256 : 128;
   if (nl <= 128) bn = 128;
+  // CTA pairs (256 x 256 tiles) when the shard is a whole number of 256-column tiles and there are at
+  // least two tile rows; otherwise the single-CTA kernel, which also handles every ragged case.
+  const bool pair_ok = nl % 256 == 0 && a->M > BM && a->block_n != 128 && h->sm_count >= 4;
+  if (a->cta_pair > 0 && !pair_ok) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: cta_pair needs (N/world) %% 256 == 0, M > 128 and block_n != 128");
+  bool pair = a->cta_pair >= 0 && pair_ok;
+  int max_pairs = 0;
+  if (pair) {
+    const int rc = a->dtype == IRIS_BF16 ? launch_gemm_pair<true>(p, 0, nullptr, &max_pairs) : launch_gemm_pair<false>(p, 0, nullptr, &max_pairs);
+    if (rc != IRIS_OK) return rc;
+    if (max_pairs < 2) {
+      if (a->cta_pair > 0) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: no room for CTA pairs on this device");
+      pair = false;
+    }
+  }
+  if (pair) bn = kPairBN;
   p.tab = h->table();
   p.c_off = a->c_off;
   p.flag_off = a->flag_off;
@@ -626,17 +857,30 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   p.timeout_ns = a->spin_timeout_ns ? a->spin_timeout_ns : kDefaultTimeoutNs;
   p.status = h->status;
   p.M = a->M; p.N = a->N; p.K = a->K; p.n_local = nl;
-  p.tiles_m = (a->M + BM - 1) / BM;
+  p.ptiles_m = (a->M + BM - 1) / BM;
+  p.tiles_m = pair ? (a->M + 2 * BM - 1) / (2 * BM) : p.ptiles_m;
   p.ctiles_per_rank = (nl + bn - 1) / bn;
   p.ptiles_per_rank = (nl + IRIS_TILE - 1) / IRIS_TILE;
   p.total_ctiles = p.tiles_m * W * p.ctiles_per_rank;
-  p.total_ptiles = p.tiles_m * W * p.ptiles_per_rank;
+  p.total_ptiles = p.ptiles_m * W * p.ptiles_per_rank;
   p.kblocks = (a->K + BK - 1) / BK;
   p.raster_group = a->raster_group ? a->raster_group : 16;
   p.mode = a->mode;
   p.epoch = a->epoch;
   int grid = a->max_ctas ? std::min(a->max_ctas, h->sm_count) : h->sm_count;
-  if (wg) {
+  if (pair) {
+    grid = std::min(grid & ~1, 2 * max_pairs);
+    if (grid < (wg ? 4 : 2)) return fail(IRIS_ERR_ARG, "gemm_all_scatter: max_ctas too small for CTA pairs");
+    if (wg) {
+      int comm = a->comm_ctas ? a->comm_ctas : auto_comm_ctas(a->M, a->N, a->K, W, grid);
+      comm = std::max(2, std::min((comm + 1) & ~1, grid - 2));   // whole pairs on both sides
+      p.comm_ctas = comm;
+      p.gemm_ctas = 2 * std::min((grid - comm) / 2, p.total_ctiles);
+    } else {
+      p.comm_ctas = 0;
+      p.gemm_ctas = 2 * std::min(grid / 2, p.total_ctiles);
+    }
+  } else if (wg) {
     if (grid < 2) return fail(IRIS_ERR_ARG, "gemm_all_scatter: workgroup_specialized needs at least 2 CTAs");
     int comm = a->comm_ctas ? a->comm_ctas : auto_comm_ctas(a->M, a->N, a->K, W, grid);
     comm = std::min(comm, std::min(grid - 1, p.total_ptiles));
@@ -657,7 +901,7 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     if (rc != IRIS_OK) return rc;
     for (int r = 0; r < W; ++r) {
       const cuuint64_t dimsB[2] = {(cuuint64_t)a->K, (cuuint64_t)nl};
-      const cuuint32_t boxB[2] = {BK, (cuuint32_t)bn};
+      const cuuint32_t boxB[2] = {BK, (cuuint32_t)(pair ? kPairBN / 2 : bn)};   // a pair's CTA loads its half of the tile
       rc = make_map(&p.tmB[r], a->dtype, 2, const_cast<void*>(a->B_shards[r]), dimsB, strA, boxB, CU_TENSOR_MAP_SWIZZLE_128B, "B");
       if (rc != IRIS_OK) return rc;
     }
@@ -675,13 +919,14 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc;
   const bool bf = a->dtype == IRIS_BF16;
-  if (bn == 256) rc = bf ? launch_gemm<256, true>(p, grid, wg, st) : launch_gemm<256, false>(p, grid, wg, st);
-  else           rc = bf ? launch_gemm<128, true>(p, grid, wg, st) : launch_gemm<128, false>(p, grid, wg, st);
+  if (pair)           rc = bf ? launch_gemm_pair<true>(p, grid, st, nullptr) : launch_gemm_pair<false>(p, grid, st, nullptr);
+  else if (bn == 256) rc = bf ? launch_gemm<256, true>(p, grid, wg, st) : launch_gemm<256, false>(p, grid, wg, st);
+  else                rc = bf ? launch_gemm<128, true>(p, grid, wg, st) : launch_gemm<128, false>(p, grid, wg, st);
   if (rc != IRIS_OK) return rc;
   if (a->mode == IRIS_MODE_BULK_SYNCHRONOUS) {
     // Listing 3: the second kernel on the same stream; the kernel boundary is the synchronisation.
     const int g2 = std::min(p.total_ptiles, h->sm_count * 8);
-    all_scatter_kernel<<<g2, 256, 0, st>>>(p.tab, a->c_off, a->flag_off, a->M, a->N, nl, p.tiles_m, p.ptiles_per_rank, a->epoch);
+    all_scatter_kernel<<<g2, 256, 0, st>>>(p.tab, a->c_off, a->flag_off, a->M, a->N, nl, p.ptiles_m, p.ptiles_per_rank, a->epoch);
     IRIS_CUDA_TRY(cudaGetLastError());
   }
   return IRIS_OK;
@@ -828,6 +1073,7 @@ int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, co
   p.status = scratch;
   p.M = M; p.N = N; p.K = K; p.n_local = nl;
   p.tiles_m = (M + BM - 1) / BM;
+  p.ptiles_m = p.tiles_m;
   p.ctiles_per_rank = (nl + bn - 1) / bn;
   p.ptiles_per_rank = (nl + IRIS_TILE - 1) / IRIS_TILE;
   p.total_ctiles = p.tiles_m * world * p.ctiles_per_rank;

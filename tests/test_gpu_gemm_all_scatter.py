@@ -90,6 +90,8 @@ EXACT_SHAPES = [
     (3, 520, 392, 328),        # odd world, everything ragged, several tiles
     (8, 1, 8, 8),              # smallest legal problem
     (2, 300, 640, 64),         # N_local > 512 and not a multiple of 256
+    (2, 1000, 512, 200),       # CTA-pair tiles (256 x 256), ragged M: the last pair's second CTA has no rows
+    (8, 257, 256, 64),         # CTA-pair tiles, one row in the second tile row
 ]
 
 
@@ -118,7 +120,8 @@ def test_exact_integer_gemm_tile_width_and_grid_knobs(block_n, mode):
     bpr = gemm_layout(M, N, W, True)[4]
     with GpuHeap(W, bpr) as g:
         img = None
-        for kw in (dict(), dict(max_ctas=7, comm_ctas=3, raster_group=2), dict(max_ctas=148, comm_ctas=32, raster_group=1)):
+        for kw in (dict(), dict(max_ctas=7, comm_ctas=3, raster_group=2), dict(max_ctas=148, comm_ctas=32, raster_group=1),
+                   dict(cta_pair=-1), dict(cta_pair=-1, max_ctas=5, comm_ctas=2), dict(cta_pair=1 if block_n == 256 else 0, comm_ctas=8)):
             g.mem.fill_(SENTINEL)
             run_gemm(g, A, Bs, dtype, mode, block_n=block_n, **kw)
             host = g.to_host()
@@ -229,12 +232,15 @@ def test_argument_errors_are_reported_before_any_launch():
             (dict(M=4096, N=256), iris.IRIS_ERR_RANGE), (dict(flag_off=(1 << 20) - 4), iris.IRIS_ERR_RANGE),
             (dict(flag_off=1024), iris.IRIS_ERR_ARG),                   # flags inside C
             (dict(mode=2, lock_off=65536), iris.IRIS_ERR_ARG),          # locks on top of flags
+            (dict(cta_pair=1), iris.IRIS_ERR_UNSUPPORTED),              # M = 128: no room for a 256-row pair tile
+            (dict(cta_pair=2), iris.IRIS_ERR_ARG),
         ]
         for delta, code in cases:
             kw = {**ok, **delta}
             with pytest.raises(iris.IrisError) as e:
                 iris.iris_gemm_all_scatter_ex(g.h, d, [d, d], kw["M"], kw["N"], kw["K"], kw["world"], kw["mode"], kw["dtype"],
-                                              kw["c_off"], kw["flag_off"], kw["lock_off"], kw["epoch"], block_n=kw.get("block_n", 0))
+                                              kw["c_off"], kw["flag_off"], kw["lock_off"], kw["epoch"], block_n=kw.get("block_n", 0),
+                                              cta_pair=kw.get("cta_pair", 0))
             assert e.value.code == code, (delta, e.value)
         torch.cuda.synchronize()
         assert bool(torch.all(g.mem == SENTINEL))

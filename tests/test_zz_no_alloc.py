@@ -5,8 +5,8 @@ already handed out to a framework's pool, a loop that cannot take the synchronis
 it takes raw slot addresses instead of a heap handle and keeps its locks and status block in a fixed array
 inside the library.  That array is shared by all calls and keeps its old contents, so the test calls it twice
 in a row, with different inputs, and compares every byte of C and every flag in every slot with what
-iris_gemm_all_scatter_ex (workgroup-specialised) produced for the same inputs.  Both paths run the same main
-loop, so the comparison is bit-exact, which is tighter than the tolerance the other GPU tests use.
+iris_gemm_all_scatter_ex (workgroup-specialised, single-CTA tiles) produced for the same inputs.  Both paths run
+the same main loop, so the comparison is bit-exact, which is tighter than the tolerance the other GPU tests use.
 
 This file is named so that pytest collects it last.
 """
@@ -29,7 +29,7 @@ def _reference_run(W, M, N, K, dtype, A, Bs, epoch):
     with GpuHeap(W, bpr) as g:
         iris.iris_flags_fill(g.h, lock_off, nt, 0)
         iris.iris_gemm_all_scatter_ex(g.h, dev16(A), [dev16(b) for b in Bs], M, N, K, W, iris.IRIS_MODE_WORKGROUP_SPECIALIZED,
-                                      iris.DTYPES[dtype], c_off, flag_off, lock_off, epoch)
+                                      iris.DTYPES[dtype], c_off, flag_off, lock_off, epoch, cta_pair=-1)
         iris.iris_status_check(g.h)
         host = g.to_host().reshape(W, bpr)
         return (host[:, c_off:c_off + M * N * 2].copy(), host[:, flag_off:flag_off + nt * 4].copy())
