@@ -42,9 +42,9 @@ DEFAULT_WORKLOAD = "cfg5_w8_m8192_n16384_k16384"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 METRIC = "gemm_all_scatter_tflops"
 UNIT = "TFLOP/s"
-# DRAM traffic of one workgroup_specialized launch on the default workload (bytes), from the ncu capture
-# summarised in profiles/; None until a capture exists.
-NCU_TRAFFIC_BYTES = None
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one workgroup_specialized launch on the default
+# workload, from the 1-pass ncu capture summarised in profiles/bench_default_launch_list.md: 6.22 GB + 2.10 GB.
+NCU_TRAFFIC_BYTES = {"cfg5_w8_m8192_n16384_k16384": 8.32e9}
 
 
 def peaks():
@@ -60,7 +60,7 @@ def align(x, a=256):
 
 
 class ClockSampler:
-    """nvidia-smi clocks / throttle reasons sampled every 100 ms while the timed region runs."""
+    """nvidia-smi clocks / throttle reasons sampled every 20 ms while the timed region runs."""
 
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -73,7 +73,7 @@ class ClockSampler:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             os.close(fd)
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                                          "-lms", "20"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except Exception:
             self.proc = None
 
@@ -205,7 +205,7 @@ def run_ours(args):
 
     def gemm(epoch, m=mode, **kw):
         iris.iris_gemm_all_scatter_ex(h, dA, dB, M, N, K, W, m, dt, 0, flag_off, lock_off, epoch, comm_ctas=args.comm_ctas,
-                                      raster_group=args.raster_group, block_n=args.block_n, cta_pair=args.cta_pair, **kw)
+                                      raster_group=args.raster_group, block_n=args.block_n, cta_pair=args.cta_pair, static_schedule=args.static_schedule, **kw)
 
     def consume(epoch):
         iris.iris_consume_bias(h, 0, out_off, flag_off, dbias, M, N, W, dt, epoch)
@@ -262,10 +262,11 @@ def run_ours(args):
         t_tensor = flops / (pk["bf16_tflops"] * 1e12) * 1e3
         t_store = store_bytes / (pk["hbm_gbs"] * 1e9) * 1e3
         achieved = flops / (gemm_ms * 1e-3) / 1e12
-        result["roofline"] = {"kernel": f"gemm_all_scatter_kernel<256,bf16> ({args.mode})", "bound": "tensor", "achieved": achieved,
+        result["roofline"] = {"kernel": f"gemm_all_scatter_pair_kernel<bf16> ({args.mode}); single-CTA kernel when --cta-pair -1 or the shape needs it", "bound": "tensor", "achieved": achieved,
                               "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / pk["bf16_tflops"],
                               "peak_kind": f"{pk_kind} burst (of {pk_kind})", "peak_sustained": pk["bf16_tflops_sustained"],
-                              "frac_sustained": achieved / pk["bf16_tflops_sustained"], "traffic": NCU_TRAFFIC_BYTES,
+                              "frac_sustained": achieved / pk["bf16_tflops_sustained"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if args.mode == "workgroup_specialized" else None,
+                              "algorithmic_bytes": (M * K + N * K) * 2.0 + store_bytes,
                               "kernel_ms": gemm_ms, "combined_roofline_ms": max(t_tensor, t_store),
                               "frac_of_combined_roofline": max(t_tensor, t_store) / gemm_ms,
                               "replicated_store_gbs": store_bytes / (gemm_ms * 1e-3) / 1e9}
@@ -290,6 +291,27 @@ def run_ours(args):
                            "frac_of_combined_roofline": max(t_tensor, t_store) / ms}
         iris.iris_status_check(h)
         result["modes"] = modes
+
+        # ---------------- context only: the library GEMM (cuBLAS via torch.matmul) on the same operands ----------------
+        # Not part of the path and not a target: it shows what the same data, clocks and power cap give a plain
+        # GEMM without any scatter, next to the burst / sustained peaks measured on other data.
+        try:
+            tA = dA.view(torch.bfloat16 if dtype == "bf16" else torch.float16).view(M, K)
+            tB = torch.cat([b.view(tA.dtype).view(nl, K) for b in dB], dim=0)
+            for _ in range(3):
+                tC = tA @ tB.t()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for _ in range(args.steps):
+                tC = tA @ tB.t()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / args.steps
+            result["context"] = {"torch_matmul_same_operands": {"ms": ms, "tflops": flops / ms / 1e9, "note": "library GEMM only, no scatter, no flags"}}
+            del tB, tC
+        except Exception as exc:  # pragma: no cover
+            result["context"] = {"error": str(exc)}
 
         # ---------------- end to end through the host-buffer entry point ----------------
         try:
@@ -381,7 +403,7 @@ def all_store_sweep(iris, pk, kind):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(WORKLOADS))
@@ -390,6 +412,7 @@ def main():
     ap.add_argument("--raster-group", type=int, default=0)
     ap.add_argument("--block-n", type=int, default=0)
     ap.add_argument("--cta-pair", type=int, default=0)
+    ap.add_argument("--static-schedule", type=int, default=0)
     ap.add_argument("--mode-iters", type=int, default=3)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-strips", type=int, default=16)

@@ -194,12 +194,16 @@ typedef struct iris_gemm_args {
   int comm_ctas;               /* workgroup-specialised: communication CTAs (0 = chosen from the
                                   ratio of scatter bytes to GEMM time; 16 at the largest config) */
   int max_ctas;                /* cap on the persistent grid (0 = one CTA per SM)                */
-  int raster_group;            /* tile rows per raster group for L2 reuse (0 = 16)               */
+  int raster_group;            /* tile rows per raster group for L2 reuse (0 = 2048 rows)        */
   int block_n;                 /* compute-tile width: 0 = auto, 128 or 256                       */
   uint64_t spin_timeout_ns;    /* deadline of every device-side wait (0 = 2 s)                   */
   int cta_pair;                /* 0 = use 256 x 256 CTA-pair tiles (tcgen05 cta_group::2) when
                                   (N/world) % 256 == 0 and M > 128; 1 = require them
                                   (IRIS_ERR_UNSUPPORTED otherwise); -1 = single-CTA tiles only   */
+  int static_schedule;         /* CTA-pair kernel: 0 = pairs claim tile ids in raster order from
+                                  an atomic counter as they become free; 1 = the listings' static
+                                  loop tile = pid, pid + NUM, ... (the single-CTA kernel always
+                                  uses the static loop)                                          */
 } iris_gemm_args;
 
 /* Enqueue the whole operation on `stream` (bulk-synchronous: two kernels; otherwise one).

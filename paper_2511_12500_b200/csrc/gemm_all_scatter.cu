@@ -31,6 +31,7 @@ constexpr int BK = 64;            // 64 x 16-bit = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;        // K of one tcgen05.mma for 16-bit inputs
 constexpr int kGemmThreads = 192;
 constexpr int kEpiThreads = 128;
+constexpr int kSchedDepth = 4;    // pair kernel: tile ids in flight between the claiming thread and the other roles
 constexpr int kCommWarps = 6;     // communication CTA: every warp is a communicator with a 32 KB tile buffer
 constexpr int kTileBytes = IRIS_TILE * IRIS_TILE * 2;
 constexpr int kSmemPayload = 192 * 1024;
@@ -60,6 +61,8 @@ struct alignas(64) GemmParams {
   int total_ptiles;     // tiles_m * W * ptiles_per_rank
   int kblocks;          // ceil(K / 64)
   int ptiles_m;         // publication tile rows: ceil(M / 128)
+  int dynamic;          // pair kernel: 1 = tiles are claimed from *tile_counter in raster order, 0 = static stride
+  int32_t* tile_counter;
   int gemm_ctas, comm_ctas;
   int raster_group;
   int mode;
@@ -72,6 +75,9 @@ struct CtrlBlock {  // lives in shared memory after the payload area
   uint64_t tmem_full[2];
   uint64_t tmem_empty[2];
   uint64_t comm_full[kCommWarps];
+  uint64_t sched_full[kSchedDepth];
+  uint64_t sched_empty[kSchedDepth];
+  volatile int32_t sched_tile[kSchedDepth];
   uint32_t tmem_base;
   volatile int abort;
 };
@@ -98,11 +104,13 @@ __device__ __forceinline__ TileCoord decode_ctile(int id, const GemmParams& p) {
 
 // Bounded mbarrier wait.  Returns false when the deadline passed (recorded in the status block) or
 // when another thread of the CTA already gave up.
+template <bool CLUSTER_ACQUIRE = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, const GemmParams& p, CtrlBlock* ctrl, int tile) {
-  if (ptx::mbar_try_wait(bar, parity)) return true;
+  auto poll = [&]() { return CLUSTER_ACQUIRE ? ptx::mbar_try_wait_cluster(bar, parity) : ptx::mbar_try_wait(bar, parity); };
+  if (poll()) return true;
   const uint64_t start = globaltimer_ns();
   uint32_t spins = 0;
-  while (!ptx::mbar_try_wait(bar, parity)) {
+  while (!poll()) {
     if ((++spins & 63u) == 0) {
       if (ctrl->abort) return false;
       if (globaltimer_ns() - start > p.timeout_ns) {
@@ -163,6 +171,7 @@ __device__ __forceinline__ int32_t* lock_addr(const GemmParams& p, int rank, int
 #ifdef IRIS_COMM_TRACE
 // Debug build only: per communicator warp {tiles, ns in: load, store issue, store wait, publish, idle poll, claim}.
 __device__ unsigned long long g_comm_trace[64 * 6 * 8];
+__device__ unsigned long long g_tile_trace[2 * 4096];  // {start ns, smid} per compute tile
 #define IRIS_TR(var) const uint64_t var = globaltimer_ns()
 #else
 #define IRIS_TR(var)
@@ -490,6 +499,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_pair_kernel(
     for (int i = 0; i < kPairStages; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->empty[i]), 1); }
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i]), 8); }
     for (int i = 0; i < kCommWarps; ++i) ptx::mbar_init(ptx::smem_u32(&ctrl->comm_full[i]), 1);
+    // tile feed: one publisher; readers = the leader's MMA thread + 4 epilogue warps, the peer's producer + 4 epilogue warps
+    for (int i = 0; i < kSchedDepth; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->sched_full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->sched_empty[i]), 10); }
     ctrl->abort = 0;
     ptx::fence_mbar_init();
     fence_proxy_async();
@@ -509,16 +520,52 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_pair_kernel(
   ptx::cluster_sync();   // the peer's barriers exist before anything of ours can signal them
   ptx::tc_fence_after();
 
+  // Tile feed.  Lane 0 of the leader's producer warp decides which tile the pair computes next -- the next id
+  // of the raster order from a global counter (dynamic), or pair_id + n * gemm_pairs (static, the listings'
+  // loop) -- and publishes it through a small ring in both CTAs' shared memory; every other role takes its
+  // tile ids from the ring.  -1 ends the stream.
+  auto feed_take = [&](int& j, uint32_t& ph, int& slot) -> int {   // -2: the wait expired
+    if (!mbar_wait<true>(ptx::smem_u32(&ctrl->sched_full[j]), ph, p, ctrl, -4)) return -2;
+    const int tile = ctrl->sched_tile[j];
+    slot = j;
+    if (++j == kSchedDepth) { j = 0; ph ^= 1; }
+    return tile;
+  };
+  auto feed_release = [&](int slot) { ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&ctrl->sched_empty[slot]), 0)); };
+
   if (is_comm) {
     comm_cta<STATIC_LOCKS, kPairBN / IRIS_TILE, 2>(p, ctrl, payload, warp, lane);
   } else if (warp == 0) {
-    // ---------------- TMA producer (both CTAs) ----------------
+    // ---------------- TMA producer (both CTAs); the leader's also claims and publishes the tiles ----------------
     if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
-      bool ok = true;
-      for (int tile = pair_id; tile < p.total_ctiles && ok; tile += gemm_pairs) {
+      int stage = 0, fj = 0, fslot = 0;
+      uint32_t phase = 0, fph = 0;
+      int static_next = pair_id;
+      auto claim = [&]() -> int {
+        int t;
+        if (p.dynamic) t = atomicAdd(p.tile_counter, 1);
+        else { t = static_next; static_next += gemm_pairs; }
+        return t;
+      };
+      int claimed = leader ? claim() : 0;
+      for (;;) {
+        int tile;
+        if (leader) {
+          tile = claimed < p.total_ctiles ? claimed : -1;
+          if (!mbar_wait(ptx::smem_u32(&ctrl->sched_empty[fj]), fph ^ 1, p, ctrl, -5)) break;
+          ctrl->sched_tile[fj] = tile;
+          ptx::st_shared_cluster_u32(ptx::mapa(ptx::smem_u32((const void*)&ctrl->sched_tile[fj]), 1), (uint32_t)tile);
+          ptx::mbar_arrive(ptx::smem_u32(&ctrl->sched_full[fj]));
+          ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&ctrl->sched_full[fj]), 1));   // release.cluster: after the remote store
+          if (++fj == kSchedDepth) { fj = 0; fph ^= 1; }
+          if (tile >= 0) claimed = claim();   // the next claim's latency hides behind this tile's loads
+        } else {
+          tile = feed_take(fj, fph, fslot);
+          if (tile != -2) feed_release(fslot);
+        }
+        if (tile < 0) break;
         const TileCoord tc = decode_ctile(tile, p);
+        bool ok = true;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!mbar_wait(ptx::smem_u32(&ctrl->empty[stage]), phase ^ 1, p, ctrl, tile)) { ok = false; break; }
           const uint32_t full_local = ptx::smem_u32(&ctrl->full[stage]);
@@ -529,6 +576,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_pair_kernel(
           ptx::tma_load_2d_pair(sa + BM * BK * 2, &p.tmB[tc.rank], kb * BK, tc.jn * kPairBN + cta_rank * (kPairBN / 2), full_leader);
           if (++stage == kPairStages) { stage = 0; phase ^= 1; }
         }
+        if (!ok) break;
       }
     }
   } else if (warp == 1) {
@@ -536,13 +584,19 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_pair_kernel(
     if (lane == 0 && leader) {
       constexpr uint32_t idesc = ptx::idesc_f16(2 * BM, kPairBN, BF16 ? 1 : 0);
       const uint32_t tmem_base = ctrl->tmem_base;
-      int stage = 0, acc = 0;
-      uint32_t phase = 0, acc_phase = 0;
-      bool ok = true;
-      for (int tile = pair_id; tile < p.total_ctiles && ok; tile += gemm_pairs) {
+      int stage = 0, acc = 0, fj = 0, fslot = 0;
+      uint32_t phase = 0, acc_phase = 0, fph = 0;
+      for (;;) {
+        const int tile = feed_take(fj, fph, fslot);
+        if (tile != -2) feed_release(fslot);
+        if (tile < 0) break;
         if (!mbar_wait(ptx::smem_u32(&ctrl->tmem_empty[acc]), acc_phase ^ 1, p, ctrl, tile)) break;
         ptx::tc_fence_after();
+#ifdef IRIS_COMM_TRACE
+        if (tile < 4096) { g_tile_trace[2 * tile] = globaltimer_ns(); unsigned sm; asm("mov.u32 %0, %%smid;" : "=r"(sm)); g_tile_trace[2 * tile + 1] = sm; }
+#endif
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kPairBN);
+        bool ok = true;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!mbar_wait(ptx::smem_u32(&ctrl->full[stage]), phase, p, ctrl, tile)) { ok = false; break; }
           ptx::tc_fence_after();
@@ -564,13 +618,18 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_pair_kernel(
     // ---------------- epilogue: warps 2..5 of both CTAs, each CTA drains its own 128 rows ----------------
     const int quad = warp & 3;
     const int et = (int)threadIdx.x - 64;
-    int acc = 0;
-    uint32_t acc_phase = 0;
+    int acc = 0, fj = 0, fslot = 0;
+    uint32_t acc_phase = 0, fph = 0;
     const uint32_t tmem_base = ctrl->tmem_base;
-    for (int tile = pair_id; tile < p.total_ctiles; tile += gemm_pairs) {
-      const TileCoord tc = decode_ctile(tile, p);
-      const bool ok = mbar_wait(ptx::smem_u32(&ctrl->tmem_full[acc]), acc_phase, p, ctrl, tile);
+    for (;;) {
+      const int tile = feed_take(fj, fph, fslot);
+      __syncwarp();
+      if (tile != -2 && lane == 0) feed_release(fslot);
+      // uniform decision for all four warps: stop on the end marker or on any failed wait
+      bool ok = tile >= 0;
+      if (ok) ok = mbar_wait(ptx::smem_u32(&ctrl->tmem_full[acc]), acc_phase, p, ctrl, tile);
       if (ptx::bar_red_or(1, kEpiThreads, !ok)) break;
+      const TileCoord tc = decode_ctile(tile, p);
       ptx::tc_fence_after();
       const int tm = tc.tm * 2 + cta_rank;  // publication tile row of this CTA's half
       const int row = tm * BM + quad * 32 + lane;
@@ -864,7 +923,9 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   p.total_ctiles = p.tiles_m * W * p.ctiles_per_rank;
   p.total_ptiles = p.ptiles_m * W * p.ptiles_per_rank;
   p.kblocks = (a->K + BK - 1) / BK;
-  p.raster_group = a->raster_group ? a->raster_group : 16;
+  // 2048 rows per raster group: with tiles claimed in raster order the running tiles then cover about
+  // 8 x 9 pair tiles, the near-square footprint that minimises operand re-reads from HBM (measured).
+  p.raster_group = a->raster_group ? a->raster_group : (pair ? 8 : 16);
   p.mode = a->mode;
   p.epoch = a->epoch;
   int grid = a->max_ctas ? std::min(a->max_ctas, h->sm_count) : h->sm_count;
@@ -919,6 +980,11 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc;
   const bool bf = a->dtype == IRIS_BF16;
+  if (pair) {
+    p.dynamic = a->static_schedule ? 0 : 1;
+    p.tile_counter = h->status + 16;   // a spare word of the status block; every launch starts it at zero
+    if (p.dynamic) IRIS_CUDA_TRY(cudaMemsetAsync(p.tile_counter, 0, sizeof(int32_t), st));
+  }
   if (pair)           rc = bf ? launch_gemm_pair<true>(p, grid, st, nullptr) : launch_gemm_pair<false>(p, grid, st, nullptr);
   else if (bn == 256) rc = bf ? launch_gemm<256, true>(p, grid, wg, st) : launch_gemm<256, false>(p, grid, wg, st);
   else                rc = bf ? launch_gemm<128, true>(p, grid, wg, st) : launch_gemm<128, false>(p, grid, wg, st);
@@ -1124,6 +1190,11 @@ int iris_debug_comm_trace(unsigned long long* host_out, int clear) {
   cudaDeviceSynchronize();
   if (host_out) cudaMemcpyFromSymbol(host_out, g_comm_trace, sizeof(g_comm_trace));
   if (clear) { static unsigned long long z[64 * 6 * 8]; cudaMemcpyToSymbol(g_comm_trace, z, sizeof(z)); }
+  return 0;
+}
+int iris_debug_tile_trace(unsigned long long* host_out) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(host_out, g_tile_trace, sizeof(g_tile_trace));
   return 0;
 }
 #endif

@@ -121,7 +121,7 @@ def test_exact_integer_gemm_tile_width_and_grid_knobs(block_n, mode):
     with GpuHeap(W, bpr) as g:
         img = None
         for kw in (dict(), dict(max_ctas=7, comm_ctas=3, raster_group=2), dict(max_ctas=148, comm_ctas=32, raster_group=1),
-                   dict(cta_pair=-1), dict(cta_pair=-1, max_ctas=5, comm_ctas=2), dict(cta_pair=1 if block_n == 256 else 0, comm_ctas=8)):
+                   dict(cta_pair=-1), dict(cta_pair=-1, max_ctas=5, comm_ctas=2), dict(cta_pair=1 if block_n == 256 else 0, comm_ctas=8), dict(static_schedule=1), dict(static_schedule=1, max_ctas=10, raster_group=3)):
             g.mem.fill_(SENTINEL)
             run_gemm(g, A, Bs, dtype, mode, block_n=block_n, **kw)
             host = g.to_host()
