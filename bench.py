@@ -165,6 +165,22 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def max_over_ranks(value: float, device=None) -> float:
+    """Max of a per-rank scalar over the process group (the job's time is its slowest rank's)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([value], dtype=torch.float64, device=device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(world_size: int, flops_per_rank_step: float, ms_per_step_max: float) -> float:
+    """Whole-job TFLOP/s of `world_size` replicas, each doing flops_per_rank_step per step, timed by the slowest."""
+    return world_size * flops_per_rank_step / (ms_per_step_max * 1e-3) / 1e12
+
+
 def run_ours(args):
     import torch
     import paper_2511_12500_b200 as iris
@@ -203,9 +219,10 @@ def run_ours(args):
     flops = 2.0 * M * N * K
     store_bytes = float(W) * M * N * 2
 
-    def gemm(epoch, m=mode, **kw):
+    def gemm(epoch, m=mode, fused=False, **kw):
         iris.iris_gemm_all_scatter_ex(h, dA, dB, M, N, K, W, m, dt, 0, flag_off, lock_off, epoch, comm_ctas=args.comm_ctas,
-                                      raster_group=args.raster_group, block_n=args.block_n, cta_pair=args.cta_pair, static_schedule=args.static_schedule, **kw)
+                                      raster_group=args.raster_group, block_n=args.block_n, cta_pair=args.cta_pair, static_schedule=args.static_schedule,
+                                      consumer_bias=dbias if fused else None, consumer_out_off=out_off, **kw)
 
     def consume(epoch):
         iris.iris_consume_bias(h, 0, out_off, flag_off, dbias, M, N, W, dt, epoch)
@@ -216,11 +233,28 @@ def run_ours(args):
             dist.barrier()
             torch.cuda.synchronize()
 
+    fused = bool(args.fused_consumer)
+
+    def step(epoch, events=None):
+        """One pass of the path: GEMM + all-scatter + flag publication + flag-gated consumer."""
+        if events:
+            events[0].record(stream)
+        if fused:
+            gemm(epoch, fused=True)          # the consumer's warps acquire the flags inside the same launch
+            if events:
+                events[1].record(stream)
+        else:
+            gemm(epoch)
+            if events:
+                events[1].record(stream)
+            consume(epoch)
+        if events:
+            events[2].record(stream)
+
     epoch = 0
     for _ in range(args.warmup):
         epoch += 1
-        gemm(epoch)
-        consume(epoch)
+        step(epoch)
     iris.iris_status_check(h)
 
     # ---------------- timed region: exactly K steps ----------------
@@ -230,32 +264,25 @@ def run_ours(args):
     sampler.start()
     for i in range(args.steps):
         epoch += 1
-        ev[i][0].record(stream)
-        gemm(epoch)
-        ev[i][1].record(stream)
-        consume(epoch)
-        ev[i][2].record(stream)
+        step(epoch, ev[i])
     barrier()
     clocks = sampler.stop()
     iris.iris_status_check(h)
     total_ms = ev[0][0].elapsed_time(ev[-1][2])
     gemm_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
     cons_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
-    if dist_on:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, device="cuda")
     ms_per_step = total_ms / args.steps
-    value = world_size * flops / (ms_per_step * 1e-3) / 1e12
+    value = job_value(world_size, flops, ms_per_step)
 
     result = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world_size, "steps": args.steps, "warmup": args.warmup,
               "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if dtype == "bf16" else "f16",
               "data": "synthetic",
               "config": {"workload": args.workload, "world": W, "M": M, "N": N, "K": K, "mode": args.mode, "comm_ctas": args.comm_ctas or "auto",
-                         "step": "gemm_all_scatter + flag-gated consumer (OUT = C + bias)", "accumulate": "fp32",
+                         "step": "gemm_all_scatter + flag-gated consumer (OUT = C + bias)" + (", consumer warps inside the GEMM launch" if fused else ", consumer as a second kernel"), "accumulate": "fp32",
                          "l2": "inputs (0.8 GB) and outputs (4.3 GB) far exceed the 126 MB L2; no explicit flush",
                          "multi_gpu": "replicas only (ranks are emulated inside one GPU)"},
-              "clocks": clocks, "gpu_launches": 2 * args.steps}
+              "clocks": clocks, "gpu_launches": (1 if fused else 2) * args.steps}
 
     if rank == 0:
         # ---------------- roofline of the dominant kernel ----------------
@@ -271,8 +298,19 @@ def run_ours(args):
                               "frac_of_combined_roofline": max(t_tensor, t_store) / gemm_ms,
                               "replicated_store_gbs": store_bytes / (gemm_ms * 1e-3) / 1e9}
         cons_bytes = 2.0 * store_bytes + N * 2
+        if fused:   # time the stand-alone consumer kernel too, for its own HBM figure
+            ts = []
+            for _ in range(4):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                consume(epoch)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            cons_ms = float(np.median(ts[1:]))
         result["consumer"] = {"kernel_ms": cons_ms, "gbs": cons_bytes / (cons_ms * 1e-3) / 1e9,
-                              "frac_of_hbm_peak": cons_bytes / (cons_ms * 1e-3) / 1e9 / pk["hbm_gbs"], "bytes": cons_bytes}
+                              "frac_of_hbm_peak": cons_bytes / (cons_ms * 1e-3) / 1e9 / pk["hbm_gbs"], "bytes": cons_bytes,
+                              "note": "stand-alone consumer kernel after the producer" + ("; in the timed step the consumer runs inside the GEMM launch" if fused else "")}
 
         # ---------------- the three schedules on the same workload (context for the headline) ----------------
         modes = {}
@@ -291,6 +329,24 @@ def run_ours(args):
                            "frac_of_combined_roofline": max(t_tensor, t_store) / ms}
         iris.iris_status_check(h)
         result["modes"] = modes
+
+        # ---------------- the same step with the consumer's warps inside the GEMM launch ----------------
+        if not fused and args.mode != "bulk_synchronous":
+            for _ in range(2):
+                epoch += 1
+                gemm(epoch, fused=True)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            e0.record(stream)
+            for _ in range(args.steps):
+                epoch += 1
+                gemm(epoch, fused=True)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            iris.iris_status_check(h)
+            fms = e0.elapsed_time(e1) / args.steps
+            result["fused_consumer_step"] = {"ms_per_step": fms, "value": flops / fms / 1e9, "unit": UNIT, "gpu_launches_per_step": 1,
+                                             "note": "consumer warps acquire each tile's flag inside the GEMM launch (consumer_bias set); same outputs"}
 
         # ---------------- context only: the library GEMM (cuBLAS via torch.matmul) on the same operands ----------------
         # Not part of the path and not a target: it shows what the same data, clocks and power cap give a plain
@@ -413,6 +469,7 @@ def main():
     ap.add_argument("--block-n", type=int, default=0)
     ap.add_argument("--cta-pair", type=int, default=0)
     ap.add_argument("--static-schedule", type=int, default=0)
+    ap.add_argument("--fused-consumer", type=int, default=0)
     ap.add_argument("--mode-iters", type=int, default=3)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-strips", type=int, default=16)

@@ -204,6 +204,13 @@ typedef struct iris_gemm_args {
                                   an atomic counter as they become free; 1 = the listings' static
                                   loop tile = pid, pid + NUM, ... (the single-CTA kernel always
                                   uses the static loop)                                          */
+  const void* consumer_bias;   /* not NULL: also run the flag-gated consumer OUT = C + bias (see
+                                  iris_consume_bias) as part of this call: inside the same launch,
+                                  as extra warps that acquire each tile's flag while the GEMM is
+                                  still running (CTA-pair kernel, fused_sequential and
+                                  workgroup_specialized), or as a following kernel otherwise.
+                                  Device pointer to N elements, 16-byte aligned                  */
+  uint64_t consumer_out_off;   /* offset of OUT [M, N] in every slot (with consumer_bias)        */
 } iris_gemm_args;
 
 /* Enqueue the whole operation on `stream` (bulk-synchronous: two kernels; otherwise one).

@@ -3,27 +3,9 @@
 // producer-consumer handshake (Section 4.1): it "spins on these atomic locks (with acquire
 // semantics)" and touches the data only afterwards.  HBM-bound: 16-byte coalesced accesses, one warp
 // instruction covers 512 contiguous bytes of a row, several CTAs per SM for latency hiding.
-#include <cuda_bf16.h>
-#include <cuda_fp16.h>
-
 #include "iris_device.cuh"
 
 namespace iris {
-
-template <bool BF16>
-__device__ __forceinline__ uint32_t add2(uint32_t c, uint32_t b) {
-  if (BF16) {
-    const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&c));
-    const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b));
-    __nv_bfloat162 r = __floats2bfloat162_rn(x.x + y.x, x.y + y.y);
-    return *reinterpret_cast<uint32_t*>(&r);
-  } else {
-    const float2 x = __half22float2(*reinterpret_cast<const __half2*>(&c));
-    const float2 y = __half22float2(*reinterpret_cast<const __half2*>(&b));
-    __half2 r = __floats2half2_rn(x.x + y.x, x.y + y.y);
-    return *reinterpret_cast<uint32_t*>(&r);
-  }
-}
 
 constexpr int kConsThreads = 256;
 

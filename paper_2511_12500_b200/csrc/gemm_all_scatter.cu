@@ -31,6 +31,10 @@ constexpr int BK = 64;            // 64 x 16-bit = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;        // K of one tcgen05.mma for 16-bit inputs
 constexpr int kGemmThreads = 192;
 constexpr int kEpiThreads = 128;
+constexpr int kConsWarps = 4;     // optional consumer warps appended to every producer CTA of the pair kernel
+constexpr int kGemmThreadsFused = kGemmThreads + 32 * kConsWarps;
+constexpr int kConsUnroll = 16;   // 16-byte loads in flight per consumer lane
+constexpr int kPairBNc = 256;      // pair tile width (also used by the fused consumer's item decode)
 constexpr int kSchedDepth = 4;    // pair kernel: tile ids in flight between the claiming thread and the other roles
 constexpr int kCommWarps = 6;     // communication CTA: every warp is a communicator with a 32 KB tile buffer
 constexpr int kTileBytes = IRIS_TILE * IRIS_TILE * 2;
@@ -63,6 +67,8 @@ struct alignas(64) GemmParams {
   int ptiles_m;         // publication tile rows: ceil(M / 128)
   int dynamic;          // pair kernel: 1 = tiles are claimed from *tile_counter in raster order, 0 = static stride
   int32_t* tile_counter;
+  const uint8_t* bias;  // fused consumer: bias[N] of the element type (NULL = no consumer warps)
+  uint64_t out_off;     // fused consumer: OUT region in every slot
   int gemm_ctas, comm_ctas;
   int raster_group;
   int mode;
@@ -467,6 +473,81 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
 }
 
 // ------------------------------------------------------------------------------------------------
+// Fused consumer warps (optional).  The flag-gated consumer of Section 4.1 running inside the same launch:
+// four extra warps in every producer CTA take (publication tile, slot) items in the producers' raster
+// order, wait -- acquire load of flag[s][t], bounded, with back-off so the spinning does not steal issue
+// slots from the MMA and TMA warps -- and then stream the tile: OUT[s] = C[s] + bias.  The consumer is
+// HBM-bound and the GEMM tensor-bound, so sharing the SMs costs the GEMM little and hides the consumer's
+// 2 x W x M x N x 2 bytes behind it; per SM this is under 10 GB/s.
+// ------------------------------------------------------------------------------------------------
+template <bool BF16>
+__device__ void consumer_warp(const GemmParams& p, CtrlBlock* ctrl, int cwarp, int lane) {
+  constexpr uint32_t kFull = 0xFFFFFFFFu;
+  constexpr int SUBS = kPairBNc / IRIS_TILE, SUBS_M = 2;
+  const int W = p.tab.world;
+  const int ncons = p.gemm_ctas * kConsWarps;
+  const int pt_n = W * p.ptiles_per_rank;
+  const long long items = (long long)p.total_ctiles * SUBS * SUBS_M * W;
+  for (long long q = (long long)blockIdx.x * kConsWarps + cwarp; q < items; q += ncons) {
+    const int k = (int)(q / W), s = (int)(q % W);
+    const TileCoord tc = decode_ctile(k / (SUBS * SUBS_M), p);
+    const int sub = k % (SUBS * SUBS_M);
+    const int pj = tc.jn * SUBS + sub % SUBS;
+    const int tm = tc.tm * SUBS_M + sub / SUBS;
+    if (pj >= p.ptiles_per_rank || tm >= p.ptiles_m) continue;
+    const int t = tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
+    int ok = 1;
+    if (lane == 0) {
+      const int32_t* flag = reinterpret_cast<const int32_t*>(p.tab.base[s] + p.flag_off) + t;
+      int32_t seen = ld_acquire_gpu(flag);
+      if (seen < p.epoch) {
+        const uint64_t start = globaltimer_ns();
+        uint32_t spins = 0;
+        while ((seen = ld_acquire_gpu(flag)) < p.epoch) {
+          __nanosleep(400);
+          if ((++spins & 15u) == 0) {
+            if (ctrl->abort) { ok = 0; break; }
+            if (globaltimer_ns() - start > p.timeout_ns) {
+              report_timeout(p.status, KID_CONSUMER, t, s, seen, p.epoch);
+              ctrl->abort = 1;
+              ok = 0;
+              break;
+            }
+          }
+        }
+      }
+    }
+    ok = __shfl_sync(kFull, ok, 0);  // warp-level synchronisation: lane 0's acquire precedes every lane's reads
+    if (!ok) return;
+    const int rows = min(IRIS_TILE, p.M - tm * IRIS_TILE);
+    const uint64_t col0 = (uint64_t)tc.rank * p.n_local + (uint64_t)pj * IRIS_TILE;
+    const uint64_t tile_off = ((uint64_t)(tm * IRIS_TILE) * p.N + col0) * 2;
+    const uint64_t src = p.tab.base[s] + p.c_off + tile_off;
+    const uint64_t dst = p.tab.base[s] + p.out_off + tile_off;
+    const int ch = lane & 15;  // 16-byte chunk within the 256-byte tile row
+    const uint4 b = *reinterpret_cast<const uint4*>(p.bias + (col0 + (uint64_t)ch * 8) * 2);
+    // 2 rows per pass, kConsUnroll passes (= 8 KB per warp) in flight: at ~2 us of loaded-memory latency that is
+    // ~4 GB/s per warp, several times the 1.3 GB/s each warp must sustain to keep up with the GEMM.
+    for (int r0 = lane >> 4; r0 < rows; r0 += 2 * kConsUnroll) {
+      uint4 v[kConsUnroll];
+#pragma unroll
+      for (int u = 0; u < kConsUnroll; ++u)
+        if (r0 + 2 * u < rows) v[u] = ld_global_v4(reinterpret_cast<const void*>(src + ((uint64_t)(r0 + 2 * u) * p.N + (uint64_t)ch * 8) * 2));
+#pragma unroll
+      for (int u = 0; u < kConsUnroll; ++u)
+        if (r0 + 2 * u < rows) {
+          uint4 o;
+          o.x = add2<BF16>(v[u].x, b.x);
+          o.y = add2<BF16>(v[u].y, b.y);
+          o.z = add2<BF16>(v[u].z, b.z);
+          o.w = add2<BF16>(v[u].w, b.w);
+          st_global_v4(reinterpret_cast<void*>(dst + ((uint64_t)(r0 + 2 * u) * p.N + (uint64_t)ch * 8) * 2), o);
+        }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // CTA-pair variant: a cluster of two CTAs (one TPC) computes a 256 x 256 tile with tcgen05 cta_group::2.
 // CTA r of the pair owns rows [128 r, 128 r + 128) of the tile: it TMA-loads its own 128 x 64 slice of A
 // and its own half (128 of the 256 columns) of the B tile -- no multicast, every CTA fetches only what
@@ -483,8 +564,8 @@ constexpr int kPairStageBytes = 2 * BM * BK * 2;            // 32 KB: A slice + 
 constexpr int kPairStages = kSmemPayload / kPairStageBytes;  // 6
 constexpr int kPairBN = 256;
 
-template <bool BF16, bool STATIC_LOCKS = false>
-__global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_pair_kernel(const __grid_constant__ GemmParams p) {
+template <bool BF16, bool STATIC_LOCKS = false, bool CONSUMER = false>
+__global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1) gemm_all_scatter_pair_kernel(const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* payload = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   CtrlBlock* ctrl = reinterpret_cast<CtrlBlock*>(payload + kSmemPayload);
@@ -533,7 +614,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_pair_kernel(
   };
   auto feed_release = [&](int slot) { ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&ctrl->sched_empty[slot]), 0)); };
 
-  if (is_comm) {
+  if (warp >= kGemmThreads / 32) {
+    if (CONSUMER && !is_comm) consumer_warp<BF16>(p, ctrl, warp - kGemmThreads / 32, lane);
+  } else if (is_comm) {
     comm_cta<STATIC_LOCKS, kPairBN / IRIS_TILE, 2>(p, ctrl, payload, warp, lane);
   } else if (warp == 0) {
     // ---------------- TMA producer (both CTAs); the leader's also claims and publishes the tiles ----------------
@@ -789,9 +872,9 @@ static int launch_gemm(const GemmParams& p, int grid, bool cooperative, cudaStre
   return IRIS_OK;
 }
 
-template <bool BF16, bool STATIC_LOCKS = false>
+template <bool BF16, bool STATIC_LOCKS = false, bool CONSUMER = false>
 static int launch_gemm_pair(const GemmParams& p, int grid, cudaStream_t st, int* max_pairs_out) {
-  auto kern = gemm_all_scatter_pair_kernel<BF16, STATIC_LOCKS>;
+  auto kern = gemm_all_scatter_pair_kernel<BF16, STATIC_LOCKS, CONSUMER>;
   static bool configured = false;
   if (!configured) {
     IRIS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal));
@@ -799,7 +882,7 @@ static int launch_gemm_pair(const GemmParams& p, int grid, cudaStream_t st, int*
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(max_pairs_out ? 2 : grid));
-  cfg.blockDim = dim3(kGemmThreads);
+  cfg.blockDim = dim3(CONSUMER ? kGemmThreadsFused : kGemmThreads);
   cfg.dynamicSmemBytes = kSmemTotal;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -882,6 +965,14 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   auto overlaps = [](uint64_t o1, uint64_t n1, uint64_t o2, uint64_t n2) { return n1 && n2 && o1 < o2 + n2 && o2 < o1 + n1; };
   if (overlaps(a->c_off, c_bytes, a->flag_off, (uint64_t)nt * 4) || (wg && (overlaps(a->c_off, c_bytes, a->lock_off, (uint64_t)nt * 4) || overlaps(a->flag_off, (uint64_t)nt * 4, a->lock_off, (uint64_t)nt * 4))))
     return fail(IRIS_ERR_ARG, "gemm_all_scatter: C, flag and lock regions overlap");
+  const bool fused_consumer = a->consumer_bias != nullptr;
+  if (fused_consumer) {
+    if ((uint64_t)a->consumer_bias % 16 != 0 || a->consumer_out_off % 16 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: consumer bias / OUT offset must be 16-byte aligned");
+    if (a->consumer_out_off > bpr || c_bytes > bpr - a->consumer_out_off) return fail(IRIS_ERR_RANGE, "gemm_all_scatter: OUT leaves the slot");
+    if (overlaps(a->consumer_out_off, c_bytes, a->c_off, c_bytes) || overlaps(a->consumer_out_off, c_bytes, a->flag_off, (uint64_t)nt * 4) ||
+        (wg && overlaps(a->consumer_out_off, c_bytes, a->lock_off, (uint64_t)nt * 4)))
+      return fail(IRIS_ERR_ARG, "gemm_all_scatter: OUT overlaps C, the flags or the locks");
+  }
   if (a->M == 0 || a->N == 0) return IRIS_OK;  // empty output: nothing to compute, nothing to publish
   if (!a->A && a->K > 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: A is NULL");
   if (!a->B_shards) return fail(IRIS_ERR_ARG, "gemm_all_scatter: B_shards is NULL");
@@ -985,7 +1076,10 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     p.tile_counter = h->status + 16;   // a spare word of the status block; every launch starts it at zero
     if (p.dynamic) IRIS_CUDA_TRY(cudaMemsetAsync(p.tile_counter, 0, sizeof(int32_t), st));
   }
-  if (pair)           rc = bf ? launch_gemm_pair<true>(p, grid, st, nullptr) : launch_gemm_pair<false>(p, grid, st, nullptr);
+  const bool cons_in_kernel = pair && fused_consumer && a->mode != IRIS_MODE_BULK_SYNCHRONOUS;  // BSP publishes in its 2nd kernel
+  if (cons_in_kernel) { p.bias = static_cast<const uint8_t*>(a->consumer_bias); p.out_off = a->consumer_out_off; }
+  if (cons_in_kernel) rc = bf ? launch_gemm_pair<true, false, true>(p, grid, st, nullptr) : launch_gemm_pair<false, false, true>(p, grid, st, nullptr);
+  else if (pair)      rc = bf ? launch_gemm_pair<true>(p, grid, st, nullptr) : launch_gemm_pair<false>(p, grid, st, nullptr);
   else if (bn == 256) rc = bf ? launch_gemm<256, true>(p, grid, wg, st) : launch_gemm<256, false>(p, grid, wg, st);
   else                rc = bf ? launch_gemm<128, true>(p, grid, wg, st) : launch_gemm<128, false>(p, grid, wg, st);
   if (rc != IRIS_OK) return rc;
@@ -995,6 +1089,10 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     all_scatter_kernel<<<g2, 256, 0, st>>>(p.tab, a->c_off, a->flag_off, a->M, a->N, nl, p.ptiles_m, p.ptiles_per_rank, a->epoch);
     IRIS_CUDA_TRY(cudaGetLastError());
   }
+  // Where the consumer does not ride inside the GEMM launch (single-CTA tiles, bulk-synchronous) it follows on
+  // the same stream: same flags, same result.
+  if (fused_consumer && !cons_in_kernel)
+    return iris_consume_bias(h, a->c_off, a->consumer_out_off, a->flag_off, a->consumer_bias, a->M, a->N, W, a->dtype, a->epoch, 0, a->spin_timeout_ns, stream);
   return IRIS_OK;
 }
 
@@ -1004,7 +1102,8 @@ static void short_form_layout(int M, int N, int world, uint64_t* flag_off, uint6
   *lock_off = *flag_off + align_up((uint64_t)(nt > 0 ? nt : 0) * 4, 256);
 }
 
-static int short_form(const void* A, const void* const* B_shards, iris_heap* heap, int M, int N, int K, int world, int mode, int dtype, void* stream) {
+static int short_form(const void* A, const void* const* B_shards, iris_heap* heap, int M, int N, int K, int world, int mode, int dtype, void* stream,
+                      const void* bias = nullptr, uint64_t out_off = 0) {
   if (!heap_ok(heap)) return fail(IRIS_ERR_STATE, "gemm_all_scatter: bad heap handle");
   if (num_tiles(M, N, world) < 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: bad M/N/world");
   iris_gemm_args a;
@@ -1014,6 +1113,8 @@ static int short_form(const void* A, const void* const* B_shards, iris_heap* hea
   a.c_off = 0;
   short_form_layout(M, N, world, &a.flag_off, &a.lock_off);
   a.epoch = heap->epoch + 1;
+  a.consumer_bias = bias;
+  a.consumer_out_off = out_off;
   const int rc = iris_gemm_all_scatter_ex(&a, stream);
   if (rc == IRIS_OK) heap->epoch = a.epoch;
   return rc;
@@ -1064,15 +1165,12 @@ int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_h
   }
   void* dbias = static_cast<char*>(heap->stage_b) + b_bytes;
   if (bias_host && N > 0) IRIS_CUDA_TRY(cudaMemcpyAsync(dbias, bias_host, (size_t)N * 2, cudaMemcpyHostToDevice, st));
-  int rc = short_form(heap->stage_a, dB, heap, M, N, K, world, mode, dtype, st);
+  // with a bias the consumer is part of the same call (inside the GEMM launch where the kernel supports it)
+  int rc = short_form(heap->stage_a, dB, heap, M, N, K, world, mode, dtype, st, (bias_host && c_bytes) ? dbias : nullptr, out_off);
   if (rc != IRIS_OK) return rc;
   uint64_t flag_off, lock_off;
   short_form_layout(M, N, world, &flag_off, &lock_off);
   char* slot = heap->base + (size_t)out_slot * heap->bytes_per_rank;
-  if (bias_host) {
-    rc = iris_consume_bias(heap, 0, out_off, flag_off, dbias, M, N, world, dtype, heap->epoch, 0, 0, st);
-    if (rc != IRIS_OK) return rc;
-  }
   if (c_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(C_host, slot, c_bytes, cudaMemcpyDeviceToHost, st));
   if (bias_host && c_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(OUT_host, slot + out_off, c_bytes, cudaMemcpyDeviceToHost, st));
   if (flags_host && nt > 0)

@@ -3,6 +3,9 @@
 // "translate the pointer, then do the memory operation" (Section 3.3).
 #pragma once
 
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
 #include <cstdint>
 
 #include "iris_internal.h"
@@ -87,6 +90,22 @@ __device__ __forceinline__ uint4 ld_global_v4(const void* p) {
 }
 __device__ __forceinline__ void st_global_v4(void* p, const uint4& v) {
   asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// ---- consumer arithmetic: two packed 16-bit elements, summed in fp32, rounded once (RNE) ----------
+template <bool BF16>
+__device__ __forceinline__ uint32_t add2(uint32_t c, uint32_t b) {
+  if (BF16) {
+    const float2 x = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&c));
+    const float2 y = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&b));
+    __nv_bfloat162 r = __floats2bfloat162_rn(x.x + y.x, x.y + y.y);
+    return *reinterpret_cast<uint32_t*>(&r);
+  } else {
+    const float2 x = __half22float2(*reinterpret_cast<const __half2*>(&c));
+    const float2 y = __half22float2(*reinterpret_cast<const __half2*>(&b));
+    __half2 r = __floats2half2_rn(x.x + y.x, x.y + y.y);
+    return *reinterpret_cast<uint32_t*>(&r);
+  }
 }
 
 // ---- device-detected errors ------------------------------------------------------------------

@@ -113,3 +113,57 @@ def test_communication_ctas_give_up_when_a_lock_is_never_released():
                                       iris.IRIS_BF16, c_off, flag_off, lock_off, 1)
         iris.iris_status_check(g.h)
         assert bool(torch.all(flags == 1))
+
+
+FUSED_SHAPES = [
+    # W, M, N_local, K, kwargs
+    (2, 1000, 512, 200, dict()),                     # CTA-pair kernel: consumer warps inside the GEMM launch
+    (8, 512, 256, 320, dict(comm_ctas=4)),
+    (4, 640, 512, 128, dict(static_schedule=1, max_ctas=12, comm_ctas=4)),
+    (4, 130, 136, 72, dict()),                       # ragged: single-CTA kernel, consumer follows as a kernel
+    (2, 384, 256, 192, dict(cta_pair=-1)),
+]
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("W,M,nl,K,kw", FUSED_SHAPES)
+def test_consumer_as_part_of_the_gemm_call(mode, W, M, nl, K, kw):
+    """gemm_all_scatter with consumer_bias set: C, flags, locks and OUT must equal the oracle's heap image byte for
+    byte (integer-valued inputs make the GEMM exact).  The heap starts as NaN patterns, so a consumer warp that read
+    a tile before its flag was published would leave NaNs in OUT."""
+    N, dtype = W * nl, "bf16"
+    A = inputs.matrix(71, inputs.STREAM_A, M, K, "ternary:0.5", dtype)
+    Bs = [inputs.matrix(71, inputs.STREAM_B0 + r, nl, K, "smallint:2", dtype) for r in range(W)]
+    bias = inputs.vector(71, inputs.STREAM_BIAS, N, "smallint:3", dtype)
+    c_off, flag_off, lock_off, out_off, bpr = gemm_layout(M, N, W, with_out=True)
+    nt = oracle.num_tiles(M, N, W)
+    with GpuHeap(W, bpr, fill=0xFF) as g:
+        img = g.image(fill=0xFF)
+        iris.iris_flags_fill(g.h, flag_off, nt, 0)
+        iris.iris_flags_fill(g.h, lock_off, nt, 0)
+        for s in range(W):
+            img.view(s, lock_off, nt * 4, np.int32)[:] = 0
+        dA, dB, dbias = dev16(A), [dev16(b) for b in Bs], dev16(bias)
+        for epoch in (1, 2, 3):
+            iris.iris_gemm_all_scatter_ex(g.h, dA, dB, M, N, K, W, mode, iris.IRIS_BF16, c_off, flag_off, lock_off, epoch,
+                                          consumer_bias=dbias, consumer_out_off=out_off, **kw)
+        iris.iris_status_check(g.h)
+        img.gemm_all_scatter(A, Bs, dtype, c_off, flag_off, 3, lock_off if mode == iris.IRIS_MODE_WORKGROUP_SPECIALIZED else None)
+        img.consume_bias(dtype, c_off, out_off, M, N, bias)
+        host = g.to_host()
+        assert np.array_equal(host, img.mem), first_diff(host, img.mem)
+
+
+def test_consumer_arguments_are_checked():
+    W, M, nl, K = 2, 256, 256, 64
+    N = W * nl
+    c_off, flag_off, lock_off, out_off, bpr = gemm_layout(M, N, W, with_out=True)
+    with GpuHeap(W, bpr) as g:
+        d = torch.zeros(1 << 16, dtype=torch.int16, device="cuda")
+        for out, code in [(c_off, iris.IRIS_ERR_ARG), (flag_off, iris.IRIS_ERR_ARG), (bpr - 256, iris.IRIS_ERR_RANGE), (out_off + 8, iris.IRIS_ERR_ARG)]:
+            with pytest.raises(iris.IrisError) as e:
+                iris.iris_gemm_all_scatter_ex(g.h, d, [d, d], M, N, K, W, 1, iris.IRIS_BF16, c_off, flag_off, lock_off, 1,
+                                              consumer_bias=d, consumer_out_off=out)
+            assert e.value.code == code, (out, e.value)
+        torch.cuda.synchronize()
+        assert bool(torch.all(g.mem == SENTINEL))
