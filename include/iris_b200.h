@@ -55,6 +55,8 @@ enum {
 /* Memory order and scope of atomics (Table 3 note; Section 3.3 "Atomic Operations and Memory Model"). */
 enum { IRIS_SEM_RELAXED = 0, IRIS_SEM_ACQUIRE = 1, IRIS_SEM_RELEASE = 2, IRIS_SEM_ACQ_REL = 3 };
 enum { IRIS_SCOPE_BLOCK = 0, IRIS_SCOPE_GPU = 1, IRIS_SCOPE_SYS = 2 };
+/* Read-modify-write atomics of Table 3 (atomic_cas has its own call). min / max compare as signed int32. */
+enum { IRIS_OP_ADD = 0, IRIS_OP_XCHG = 1, IRIS_OP_AND = 2, IRIS_OP_OR = 3, IRIS_OP_XOR = 4, IRIS_OP_MIN = 5, IRIS_OP_MAX = 6 };
 
 #define IRIS_MAX_WORLD 8
 #define IRIS_TILE 128 /* publication tile edge: one ready flag per 128 x 128 block of C */
@@ -128,6 +130,20 @@ int iris_put_tile(iris_heap* heap, const void* src, void* dst, size_t rows, size
 int iris_get_tile(iris_heap* heap, const void* src, void* dst, size_t rows, size_t row_bytes, size_t src_pitch,
                   size_t dst_pitch, int from_rank, int to_rank, void* stream);
 
+/* copy (Table 3: between any two ranks): src and dst are addresses valid in cur_rank's slot; the region is read
+ * at translate(src, cur_rank, from_rank) and written at translate(dst, cur_rank, to_rank).  Otherwise as put. */
+int iris_copy_tile(iris_heap* heap, const void* src, void* dst, size_t rows, size_t row_bytes, size_t src_pitch,
+                   size_t dst_pitch, int cur_rank, int from_rank, int to_rank, void* stream);
+
+/* load / store (Table 3, value-based): like get / put, but the local side is a device buffer of the caller's
+ * that need not lie in the heap (it stands in for the registers of the paper's tl.load / tl.store).
+ * load: read translate(src, from_rank, to_rank) -> out.   store: values -> translate(dst, from_rank, to_rank).
+ * Only the heap-side region is range-checked. */
+int iris_load_tile(iris_heap* heap, const void* src, void* out, size_t rows, size_t row_bytes, size_t src_pitch,
+                   size_t out_pitch, int from_rank, int to_rank, void* stream);
+int iris_store_tile(iris_heap* heap, const void* values, void* dst, size_t rows, size_t row_bytes, size_t values_pitch,
+                    size_t dst_pitch, int from_rank, int to_rank, void* stream);
+
 /* atomic_add / atomic_cas on int32 words of to_rank's memory.  `ptr` is valid in from_rank's slot
  * and is translated first.  Vector form: `count` words, `stride_bytes` apart (multiple of 4), one
  * GPU thread per word; old_out (device pointer to count int32, or NULL) receives the previous
@@ -137,6 +153,11 @@ int iris_atomic_add(iris_heap* heap, void* ptr, size_t count, size_t stride_byte
                     int32_t value, int sem, int scope, int32_t* old_out, void* stream);
 int iris_atomic_cas(iris_heap* heap, void* ptr, size_t count, size_t stride_bytes, int from_rank, int to_rank,
                     int32_t compare, int32_t value, int sem, int scope, int32_t* old_out, void* stream);
+
+/* The remaining atomics (atomic_xchg / and / or / xor / min / max; IRIS_OP_ADD is accepted too), vector form
+ * as iris_atomic_add: old_out receives the previous values. */
+int iris_atomic_rmw(iris_heap* heap, int op, void* ptr, size_t count, size_t stride_bytes, int from_rank, int to_rank,
+                    int32_t value, int sem, int scope, int32_t* old_out, void* stream);
 
 /* Contended forms used by the protocol tests and the atomics microbenchmark: `threads` GPU
  * threads all operate on the SAME word.  add: each adds `value`; cas: thread i tries

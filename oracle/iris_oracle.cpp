@@ -289,4 +289,44 @@ int orc_all_store(uint8_t* image, int world, uint64_t bpr, uint64_t payload_off,
   return 0;
 }
 
+// Remaining read-modify-write atomics of Table 3 on int32 words of rank `to_rank`'s memory, applied
+// sequentially: op 0 add, 1 xchg, 2 and, 3 or, 4 xor, 5 min (signed), 6 max (signed).
+int orc_atomic_rmw(uint8_t* image, int world, uint64_t bpr, int op, uint64_t off, int64_t count, int64_t stride,
+                   int to_rank, int32_t val, int32_t* old_out) {
+  if (bad_rank(to_rank, world) || op < 0 || op > 6) return -1;
+  if (count > 0 && off + (uint64_t)(count - 1) * stride + 4 > bpr) return -2;
+  for (int64_t i = 0; i < count; ++i) {
+    int32_t* p = (int32_t*)(slot(image, bpr, to_rank) + off + i * stride);
+    const int32_t old = *p;
+    int32_t neu = old;
+    switch (op) {
+      case 0: neu = (int32_t)((uint32_t)old + (uint32_t)val); break;
+      case 1: neu = val; break;
+      case 2: neu = old & val; break;
+      case 3: neu = old | val; break;
+      case 4: neu = old ^ val; break;
+      case 5: neu = old < val ? old : val; break;
+      case 6: neu = old > val ? old : val; break;
+    }
+    *p = neu;
+    if (old_out) old_out[i] = old;
+  }
+  return 0;
+}
+
+// copy (Table 3: between any two ranks): the caller `cur_rank` names both regions in its own address
+// space; bytes move from rank `from_rank`'s memory at src_off to rank `to_rank`'s memory at dst_off.
+int orc_copy(uint8_t* image, int world, uint64_t bpr, uint64_t src_off, uint64_t dst_off, int64_t rows, int64_t row_bytes,
+             int64_t src_pitch, int64_t dst_pitch, int from_rank, int to_rank) {
+  if (bad_rank(from_rank, world) || bad_rank(to_rank, world)) return -1;
+  if (rows == 0 || row_bytes == 0) return 0;
+  if (src_off + (uint64_t)(rows - 1) * src_pitch + row_bytes > bpr || dst_off + (uint64_t)(rows - 1) * dst_pitch + row_bytes > bpr) return -2;
+  std::vector<uint8_t> tmp((size_t)row_bytes);
+  for (int64_t i = 0; i < rows; ++i) {
+    std::memcpy(tmp.data(), slot(image, bpr, from_rank) + src_off + i * src_pitch, (size_t)row_bytes);
+    std::memcpy(slot(image, bpr, to_rank) + dst_off + i * dst_pitch, tmp.data(), (size_t)row_bytes);
+  }
+  return 0;
+}
+
 }  // extern "C"

@@ -60,6 +60,8 @@ def lib() -> C.CDLL:
                 f.argtypes = [u8p, C.c_int, u64, u64, u64, i64, i64, i64, i64, C.c_int, C.c_int]
             L.orc_atomic_add.argtypes = [u8p, C.c_int, u64, u64, i64, i64, C.c_int, i32, C.POINTER(i32)]
             L.orc_atomic_cas.argtypes = [u8p, C.c_int, u64, u64, i64, i64, C.c_int, i32, i32, C.POINTER(i32)]
+            L.orc_atomic_rmw.argtypes = [u8p, C.c_int, u64, C.c_int, u64, i64, i64, C.c_int, i32, C.POINTER(i32)]
+            L.orc_copy.argtypes = [u8p, C.c_int, u64, u64, u64, i64, i64, i64, i64, C.c_int, C.c_int]
             L.orc_consume_bias.argtypes = [u8p, C.c_int, u64, C.c_int, u64, u64, i64, i64, u16p]
             L.orc_all_store.argtypes = [u8p, C.c_int, u64, u64, u64, u64, u64, u64, i32]
             _lib = L
@@ -178,6 +180,19 @@ class HeapImage:
         _check(lib().orc_atomic_cas(_u8p(self.mem), self.world, self.bpr, off, count, stride, to_rank, cmp, val,
                                     old.ctypes.data_as(C.POINTER(C.c_int32))), "atomic_cas")
         return old
+
+    ATOMIC_OPS = {"add": 0, "xchg": 1, "and": 2, "or": 3, "xor": 4, "min": 5, "max": 6}
+
+    def atomic_rmw(self, op: str, off, count, stride, to_rank, val) -> np.ndarray:
+        old = np.empty(count, dtype=np.int32)
+        _check(lib().orc_atomic_rmw(_u8p(self.mem), self.world, self.bpr, self.ATOMIC_OPS[op], off, count, stride, to_rank, val,
+                                    old.ctypes.data_as(C.POINTER(C.c_int32))), "atomic_rmw")
+        return old
+
+    def copy(self, src_off, dst_off, rows, row_bytes, src_pitch, dst_pitch, from_rank, to_rank):
+        """copy between any two ranks (Table 3); load/store to a buffer outside the heap are the caller's slices of this."""
+        _check(lib().orc_copy(_u8p(self.mem), self.world, self.bpr, src_off, dst_off, rows, row_bytes, src_pitch, dst_pitch,
+                              from_rank, to_rank), "copy")
 
     # --- GEMM + all-scatter -------------------------------------------------------------
     def all_scatter(self, c_off: int, c_full: np.ndarray):

@@ -17,6 +17,8 @@ IRIS_MODE_BULK_SYNCHRONOUS, IRIS_MODE_FUSED_SEQUENTIAL, IRIS_MODE_WORKGROUP_SPEC
 MODES = {"bulk_synchronous": 0, "fused_sequential": 1, "workgroup_specialized": 2}
 IRIS_SEM_RELAXED, IRIS_SEM_ACQUIRE, IRIS_SEM_RELEASE, IRIS_SEM_ACQ_REL = 0, 1, 2, 3
 IRIS_SCOPE_BLOCK, IRIS_SCOPE_GPU, IRIS_SCOPE_SYS = 0, 1, 2
+IRIS_OP_ADD, IRIS_OP_XCHG, IRIS_OP_AND, IRIS_OP_OR, IRIS_OP_XOR, IRIS_OP_MIN, IRIS_OP_MAX = range(7)
+ATOMIC_OPS = {"add": 0, "xchg": 1, "and": 2, "or": 3, "xor": 4, "min": 5, "max": 6}
 IRIS_MAX_WORLD = 8
 IRIS_TILE = 128
 
@@ -30,7 +32,7 @@ EXPORTS = [
     "iris_atomic_add_contended", "iris_atomic_cas_contended", "iris_flags_fill", "iris_all_store_bench",
     "iris_gemm_all_scatter_ex", "gemm_all_scatter", "iris_gemm_heap_bytes", "iris_heap_epoch", "iris_num_tiles",
     "iris_consume_bias", "iris_gemm_all_scatter_host", "iris_gemm_out_offset",
-    "iris_gemm_all_scatter_noalloc",
+    "iris_gemm_all_scatter_noalloc", "iris_copy_tile", "iris_load_tile", "iris_store_tile", "iris_atomic_rmw",
 ]
 
 
@@ -81,6 +83,10 @@ def lib() -> C.CDLL:
     L.iris_status_check.argtypes = [vp, vp, C.POINTER(i32)]
     for f in (L.iris_put_tile, L.iris_get_tile):
         f.argtypes = [vp, vp, vp, sz, sz, sz, sz, ci, ci, vp]
+    L.iris_copy_tile.argtypes = [vp, vp, vp, sz, sz, sz, sz, ci, ci, ci, vp]
+    for f in (L.iris_load_tile, L.iris_store_tile):
+        f.argtypes = [vp, vp, vp, sz, sz, sz, sz, ci, ci, vp]
+    L.iris_atomic_rmw.argtypes = [vp, ci, vp, sz, sz, ci, ci, i32, ci, ci, vp, vp]
     L.iris_atomic_add.argtypes = [vp, vp, sz, sz, ci, ci, i32, ci, ci, vp, vp]
     L.iris_atomic_cas.argtypes = [vp, vp, sz, sz, ci, ci, i32, i32, ci, ci, vp, vp]
     L.iris_atomic_add_contended.argtypes = [vp, vp, sz, ci, ci, i32, ci, ci, vp, vp]
@@ -201,6 +207,23 @@ def iris_put_tile(heap, src, dst, rows, row_bytes, src_pitch, dst_pitch, from_ra
 
 def iris_get_tile(heap, src, dst, rows, row_bytes, src_pitch, dst_pitch, from_rank, to_rank, stream=None):
     _ck(lib().iris_get_tile(heap, src, dst, rows, row_bytes, src_pitch, dst_pitch, from_rank, to_rank, _stream(stream)))
+
+
+def iris_copy_tile(heap, src, dst, rows, row_bytes, src_pitch, dst_pitch, cur_rank, from_rank, to_rank, stream=None):
+    _ck(lib().iris_copy_tile(heap, src, dst, rows, row_bytes, src_pitch, dst_pitch, cur_rank, from_rank, to_rank, _stream(stream)))
+
+
+def iris_load_tile(heap, src, out, rows, row_bytes, src_pitch, out_pitch, from_rank, to_rank, stream=None):
+    _ck(lib().iris_load_tile(heap, src, _ptr(out), rows, row_bytes, src_pitch, out_pitch, from_rank, to_rank, _stream(stream)))
+
+
+def iris_store_tile(heap, values, dst, rows, row_bytes, values_pitch, dst_pitch, from_rank, to_rank, stream=None):
+    _ck(lib().iris_store_tile(heap, _ptr(values), dst, rows, row_bytes, values_pitch, dst_pitch, from_rank, to_rank, _stream(stream)))
+
+
+def iris_atomic_rmw(heap, op, ptr, count, stride_bytes, from_rank, to_rank, value, sem=IRIS_SEM_RELAXED, scope=IRIS_SCOPE_GPU,
+                    old_out=None, stream=None):
+    _ck(lib().iris_atomic_rmw(heap, op, ptr, count, stride_bytes, from_rank, to_rank, value, sem, scope, _ptr(old_out), _stream(stream)))
 
 
 def iris_atomic_add(heap, ptr, count, stride_bytes, from_rank, to_rank, value, sem=IRIS_SEM_RELAXED,

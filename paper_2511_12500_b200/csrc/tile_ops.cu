@@ -6,13 +6,19 @@
 namespace iris {
 
 // ---- 2-D copy between two (already range-checked) regions; translation happens here ----------
-// PUT: read src (from_rank's space), write translate(dst, from -> to).
-// GET: read translate(src, from -> to), write dst (from_rank's space).
+// Each side is either used as given (rank pair {-1, -1}: a local heap address or a buffer outside the heap)
+// or translated from the caller's address space to the rank whose memory is touched (Section 3.3).
+//   put   src as given,            dst translate(from -> to)
+//   get   src translate(from -> to), dst as given
+//   copy  src translate(cur -> from), dst translate(cur -> to)
+//   load / store: like get / put with the local side outside the heap (the value-based API of Table 3,
+//   with a device buffer standing in for the registers)
+struct Xlate { int from, to; };
 template <bool VEC16>
 __global__ void __launch_bounds__(256) copy2d_kernel(const __grid_constant__ HeapTable tab, uint64_t src, uint64_t dst, size_t rows, size_t row_bytes,
-                                                     size_t src_pitch, size_t dst_pitch, int from_rank, int to_rank, int is_get) {
-  const uint64_t s = is_get ? translate(src, from_rank, to_rank, tab) : src;
-  const uint64_t d = is_get ? dst : translate(dst, from_rank, to_rank, tab);
+                                                     size_t src_pitch, size_t dst_pitch, Xlate xs, Xlate xd) {
+  const uint64_t s = xs.from >= 0 ? translate(src, xs.from, xs.to, tab) : src;
+  const uint64_t d = xd.from >= 0 ? translate(dst, xd.from, xd.to, tab) : dst;
   const size_t unit = VEC16 ? 16 : 1;
   const size_t per_row = row_bytes / unit;
   const size_t total = rows * per_row;
@@ -33,6 +39,48 @@ __global__ void __launch_bounds__(256) atomic_vec_kernel(const __grid_constant__
   const uint64_t p = translate(ptr, from_rank, to_rank, tab);
   for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x) {
     const int32_t old = atomic_rmw<IS_CAS>(reinterpret_cast<int32_t*>(p + i * stride), cmp, val, sem, scope);
+    if (old_out) old_out[i] = old;
+  }
+}
+
+// The other read-modify-write atomics of Table 3 (xchg, and, or, xor, min, max), same sem x scope choice.
+#define IRIS_RMW_CASE(SEMV, SCOPEV, SEMS, SCOPES)                                                                      \
+  if (sem == SEMV && scope == SCOPEV) {                                                                                \
+    switch (op) {                                                                                                      \
+      case IRIS_OP_XCHG: asm volatile("atom." SEMS "." SCOPES ".global.exch.b32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(val) : "memory"); break; \
+      case IRIS_OP_AND:  asm volatile("atom." SEMS "." SCOPES ".global.and.b32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(val) : "memory"); break;  \
+      case IRIS_OP_OR:   asm volatile("atom." SEMS "." SCOPES ".global.or.b32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(val) : "memory"); break;   \
+      case IRIS_OP_XOR:  asm volatile("atom." SEMS "." SCOPES ".global.xor.b32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(val) : "memory"); break;  \
+      case IRIS_OP_MIN:  asm volatile("atom." SEMS "." SCOPES ".global.min.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(val) : "memory"); break;  \
+      case IRIS_OP_MAX:  asm volatile("atom." SEMS "." SCOPES ".global.max.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(val) : "memory"); break;  \
+      default:           asm volatile("atom." SEMS "." SCOPES ".global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(val) : "memory"); break;  \
+    }                                                                                                                  \
+    return old;                                                                                                        \
+  }
+
+__device__ __forceinline__ int32_t atomic_op(int32_t* p, int op, int32_t val, int sem, int scope) {
+  int32_t old = 0;
+  IRIS_RMW_CASE(IRIS_SEM_RELAXED, IRIS_SCOPE_BLOCK, "relaxed", "cta")
+  IRIS_RMW_CASE(IRIS_SEM_RELAXED, IRIS_SCOPE_GPU, "relaxed", "gpu")
+  IRIS_RMW_CASE(IRIS_SEM_RELAXED, IRIS_SCOPE_SYS, "relaxed", "sys")
+  IRIS_RMW_CASE(IRIS_SEM_ACQUIRE, IRIS_SCOPE_BLOCK, "acquire", "cta")
+  IRIS_RMW_CASE(IRIS_SEM_ACQUIRE, IRIS_SCOPE_GPU, "acquire", "gpu")
+  IRIS_RMW_CASE(IRIS_SEM_ACQUIRE, IRIS_SCOPE_SYS, "acquire", "sys")
+  IRIS_RMW_CASE(IRIS_SEM_RELEASE, IRIS_SCOPE_BLOCK, "release", "cta")
+  IRIS_RMW_CASE(IRIS_SEM_RELEASE, IRIS_SCOPE_GPU, "release", "gpu")
+  IRIS_RMW_CASE(IRIS_SEM_RELEASE, IRIS_SCOPE_SYS, "release", "sys")
+  IRIS_RMW_CASE(IRIS_SEM_ACQ_REL, IRIS_SCOPE_BLOCK, "acq_rel", "cta")
+  IRIS_RMW_CASE(IRIS_SEM_ACQ_REL, IRIS_SCOPE_GPU, "acq_rel", "gpu")
+  IRIS_RMW_CASE(IRIS_SEM_ACQ_REL, IRIS_SCOPE_SYS, "acq_rel", "sys")
+  return old;
+}
+#undef IRIS_RMW_CASE
+
+__global__ void __launch_bounds__(256) atomic_op_kernel(const __grid_constant__ HeapTable tab, uint64_t ptr, size_t count, size_t stride, int from_rank,
+                                                        int to_rank, int op, int32_t val, int sem, int scope, int32_t* old_out) {
+  const uint64_t p = translate(ptr, from_rank, to_rank, tab);
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x) {
+    const int32_t old = atomic_op(reinterpret_cast<int32_t*>(p + i * stride), op, val, sem, scope);
     if (old_out) old_out[i] = old;
   }
 }
@@ -128,28 +176,38 @@ static int grid_for(const iris_heap* h, size_t work_threads, int per_sm) {
   return blocks < 1 ? 1 : (int)blocks;
 }
 
-static int put_get(iris_heap* h, const void* src, void* dst, size_t rows, size_t row_bytes, size_t src_pitch, size_t dst_pitch,
-                   int from_rank, int to_rank, void* stream, int is_get) {
-  const char* name = is_get ? "iris_get_tile" : "iris_put_tile";
+// kind: 0 put, 1 get, 2 copy, 3 load (dst outside the heap), 4 store (src outside the heap)
+static int move2d(iris_heap* h, const void* src, void* dst, size_t rows, size_t row_bytes, size_t src_pitch, size_t dst_pitch,
+                  int cur_rank, int from_rank, int to_rank, void* stream, int kind, const char* name) {
   if (!heap_ok(h)) return fail(IRIS_ERR_STATE, "%s: bad heap handle", name);
-  if (from_rank < 0 || from_rank >= h->world || to_rank < 0 || to_rank >= h->world) return fail(IRIS_ERR_ARG, "%s: rank out of range", name);
+  if (from_rank < 0 || from_rank >= h->world || to_rank < 0 || to_rank >= h->world || cur_rank < 0 || cur_rank >= h->world)
+    return fail(IRIS_ERR_ARG, "%s: rank out of range", name);
   if (rows == 0 || row_bytes == 0) return IRIS_OK;
   if (!src || !dst) return fail(IRIS_ERR_ARG, "%s: NULL pointer", name);
   if (src_pitch < row_bytes || dst_pitch < row_bytes) return fail(IRIS_ERR_ARG, "%s: pitch smaller than row_bytes", name);
-  // Both addresses are given in from_rank's space; translation preserves offsets, so checking them
-  // against from_rank's slot also bounds the translated region.
-  int rc = check_region(h, src, from_rank, rows, row_bytes, src_pitch, name);
+  // Heap-side addresses are given in the caller's (cur_rank's) space; translation preserves offsets, so checking
+  // them against the caller's slot also bounds the translated region.  Buffers outside the heap are the caller's.
+  int rc = IRIS_OK;
+  if (kind != 4) rc = check_region(h, src, cur_rank, rows, row_bytes, src_pitch, name);
   if (rc != IRIS_OK) return rc;
-  rc = check_region(h, dst, from_rank, rows, row_bytes, dst_pitch, name);
+  if (kind != 3) rc = check_region(h, dst, cur_rank, rows, row_bytes, dst_pitch, name);
   if (rc != IRIS_OK) return rc;
+  Xlate xs{-1, -1}, xd{-1, -1};
+  switch (kind) {
+    case 0: xd = {from_rank, to_rank}; break;                              // put
+    case 1: xs = {from_rank, to_rank}; break;                              // get
+    case 2: xs = {cur_rank, from_rank}; xd = {cur_rank, to_rank}; break;   // copy
+    case 3: xs = {from_rank, to_rank}; break;                              // load
+    default: xd = {from_rank, to_rank}; break;                             // store
+  }
   const bool vec = ((uint64_t)src % 16 == 0) && ((uint64_t)dst % 16 == 0) && row_bytes % 16 == 0 && src_pitch % 16 == 0 && dst_pitch % 16 == 0;
   const size_t work = rows * (vec ? row_bytes / 16 : row_bytes);
   const int grid = grid_for(h, work, 8);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (vec)
-    copy2d_kernel<true><<<grid, 256, 0, st>>>(h->table(), (uint64_t)src, (uint64_t)dst, rows, row_bytes, src_pitch, dst_pitch, from_rank, to_rank, is_get);
+    copy2d_kernel<true><<<grid, 256, 0, st>>>(h->table(), (uint64_t)src, (uint64_t)dst, rows, row_bytes, src_pitch, dst_pitch, xs, xd);
   else
-    copy2d_kernel<false><<<grid, 256, 0, st>>>(h->table(), (uint64_t)src, (uint64_t)dst, rows, row_bytes, src_pitch, dst_pitch, from_rank, to_rank, is_get);
+    copy2d_kernel<false><<<grid, 256, 0, st>>>(h->table(), (uint64_t)src, (uint64_t)dst, rows, row_bytes, src_pitch, dst_pitch, xs, xd);
   IRIS_CUDA_TRY(cudaGetLastError());
   return IRIS_OK;
 }
@@ -171,12 +229,37 @@ extern "C" {
 
 int iris_put_tile(iris_heap* h, const void* src, void* dst, size_t rows, size_t row_bytes, size_t src_pitch, size_t dst_pitch,
                   int from_rank, int to_rank, void* stream) {
-  return put_get(h, src, dst, rows, row_bytes, src_pitch, dst_pitch, from_rank, to_rank, stream, 0);
+  return move2d(h, src, dst, rows, row_bytes, src_pitch, dst_pitch, from_rank, from_rank, to_rank, stream, 0, "iris_put_tile");
 }
 
 int iris_get_tile(iris_heap* h, const void* src, void* dst, size_t rows, size_t row_bytes, size_t src_pitch, size_t dst_pitch,
                   int from_rank, int to_rank, void* stream) {
-  return put_get(h, src, dst, rows, row_bytes, src_pitch, dst_pitch, from_rank, to_rank, stream, 1);
+  return move2d(h, src, dst, rows, row_bytes, src_pitch, dst_pitch, from_rank, from_rank, to_rank, stream, 1, "iris_get_tile");
+}
+
+int iris_copy_tile(iris_heap* h, const void* src, void* dst, size_t rows, size_t row_bytes, size_t src_pitch, size_t dst_pitch, int cur_rank,
+                   int from_rank, int to_rank, void* stream) {
+  return move2d(h, src, dst, rows, row_bytes, src_pitch, dst_pitch, cur_rank, from_rank, to_rank, stream, 2, "iris_copy_tile");
+}
+
+int iris_load_tile(iris_heap* h, const void* src, void* out, size_t rows, size_t row_bytes, size_t src_pitch, size_t out_pitch, int from_rank,
+                   int to_rank, void* stream) {
+  return move2d(h, src, out, rows, row_bytes, src_pitch, out_pitch, from_rank, from_rank, to_rank, stream, 3, "iris_load_tile");
+}
+
+int iris_store_tile(iris_heap* h, const void* values, void* dst, size_t rows, size_t row_bytes, size_t values_pitch, size_t dst_pitch, int from_rank,
+                    int to_rank, void* stream) {
+  return move2d(h, values, dst, rows, row_bytes, values_pitch, dst_pitch, from_rank, from_rank, to_rank, stream, 4, "iris_store_tile");
+}
+
+int iris_atomic_rmw(iris_heap* h, int op, void* ptr, size_t count, size_t stride, int from_rank, int to_rank, int32_t value, int sem, int scope,
+                    int32_t* old_out, void* stream) {
+  if (op < IRIS_OP_ADD || op > IRIS_OP_MAX) return fail(IRIS_ERR_ARG, "iris_atomic_rmw: unknown op %d", op);
+  int rc = atomic_common(h, ptr, count, stride, from_rank, to_rank, sem, scope, "iris_atomic_rmw");
+  if (rc != IRIS_OK) return rc > 0 ? IRIS_OK : rc;
+  atomic_op_kernel<<<grid_for(h, count, 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(h->table(), (uint64_t)ptr, count, stride, from_rank, to_rank, op, value, sem, scope, old_out);
+  IRIS_CUDA_TRY(cudaGetLastError());
+  return IRIS_OK;
 }
 
 int iris_atomic_add(iris_heap* h, void* ptr, size_t count, size_t stride, int from_rank, int to_rank, int32_t value, int sem, int scope,

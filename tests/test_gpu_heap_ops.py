@@ -175,3 +175,47 @@ def test_all_store_argument_errors():
                 iris.iris_all_store_bench(g.h, *args)
             assert e.value.code == code
         assert bool(torch.all(g.mem == SENTINEL))
+
+
+@pytest.mark.parametrize("op", ["add", "xchg", "and", "or", "xor", "min", "max"])
+def test_remaining_atomics_match_oracle(op):
+    with GpuHeap(3, 1 << 14) as g:
+        img = _random_heap(g, 11)
+        n, stride, off = 500, 12, 512
+        old = torch.empty(n, dtype=torch.int32, device="cuda")
+        for val, sem, scope in [(0x5A5A1234, iris.IRIS_SEM_RELAXED, iris.IRIS_SCOPE_GPU), (-77, iris.IRIS_SEM_ACQ_REL, iris.IRIS_SCOPE_SYS),
+                                (3, iris.IRIS_SEM_RELEASE, iris.IRIS_SCOPE_BLOCK)]:
+            iris.iris_atomic_rmw(g.h, iris.ATOMIC_OPS[op], g.addr(2, off), n, stride, 2, 0, val, sem, scope, old)
+            assert np.array_equal(old.cpu().numpy(), img.atomic_rmw(op, off, n, stride, 0, val)), (op, val)
+        assert np.array_equal(g.to_host(), img.mem)
+        with pytest.raises(iris.IrisError) as e:
+            iris.iris_atomic_rmw(g.h, 9, g.addr(0, 0), 1, 4, 0, 1, 1)
+        assert e.value.code == iris.IRIS_ERR_ARG
+
+
+def test_copy_load_store_byte_exact():
+    W, bpr = 4, 1 << 16
+    with GpuHeap(W, bpr) as g:
+        img = _random_heap(g, 12)
+        # copy: rank 0 moves a region from rank 1's memory to rank 3's
+        iris.iris_copy_tile(g.h, g.addr(0, 1024), g.addr(0, 20480), 17, 80, 96, 112, 0, 1, 3)
+        img.copy(1024, 20480, 17, 80, 96, 112, 1, 3)
+        assert np.array_equal(g.to_host(), img.mem)
+        # load: rank 2 reads rank 1's memory into a buffer outside the heap
+        out = torch.zeros(9 * 48, dtype=torch.uint8, device="cuda")
+        iris.iris_load_tile(g.h, g.addr(2, 4096 + 3), out, 9, 37, 64, 48, 2, 1)       # unaligned: byte path
+        host = img.mem.reshape(W, bpr)
+        exp = np.zeros((9, 48), dtype=np.uint8)
+        for i in range(9):
+            exp[i, :37] = host[1, 4099 + i * 64: 4099 + i * 64 + 37]
+        assert np.array_equal(out.cpu().numpy().reshape(9, 48), exp)
+        # store: rank 2 writes values from outside the heap into rank 0's memory
+        vals = torch.from_numpy(inputs.payload_bytes(13, 1, 32 * 256)).cuda()
+        iris.iris_store_tile(g.h, vals, g.addr(2, 32768), 32, 256, 256, 512, 2, 0)
+        v = vals.cpu().numpy().reshape(32, 256)
+        for i in range(32):
+            img.view(0, 32768 + i * 512, 256)[:] = v[i]
+        assert np.array_equal(g.to_host(), img.mem)
+        with pytest.raises(iris.IrisError) as e:
+            iris.iris_load_tile(g.h, g.addr(2, bpr - 16), out, 2, 32, 32, 48, 2, 1)
+        assert e.value.code == iris.IRIS_ERR_RANGE

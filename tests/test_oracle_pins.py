@@ -279,6 +279,34 @@ def test_atomics_sequential_semantics():
     assert list(olds) == [0, 0, 0, 0] and list(img.view(0, 32, 32, np.int32)[::2]) == [-2] * 4
 
 
+def test_remaining_atomics_against_numpy_semantics():
+    rng = np.random.default_rng(9)
+    init = rng.integers(-2**31, 2**31 - 1, 64, dtype=np.int64).astype(np.int32)
+    val = int(np.int32(rng.integers(-2**31, 2**31 - 1)))
+    ref = {"add": (init.astype(np.int64) + val).astype(np.int32), "xchg": np.full_like(init, val), "and": init & np.int32(val),
+           "or": init | np.int32(val), "xor": init ^ np.int32(val), "min": np.minimum(init, np.int32(val)), "max": np.maximum(init, np.int32(val))}
+    for op, expect in ref.items():
+        img = oracle.HeapImage(2, 1024)
+        img.view(1, 128, 256, np.int32)[:] = init
+        old = img.atomic_rmw(op, 128, 64, 4, 1, val)
+        assert np.array_equal(old, init), op
+        assert np.array_equal(img.view(1, 128, 256, np.int32), expect), op
+        assert not img.slot(0).any()
+
+
+def test_copy_between_two_other_ranks():
+    W, bpr = 4, 2048
+    rng = np.random.default_rng(6)
+    img = oracle.HeapImage(W, bpr)
+    img.mem[:] = rng.integers(0, 256, img.mem.size, dtype=np.uint8)
+    before = img.mem.copy().reshape(W, bpr)
+    img.copy(64, 1024, 3, 20, 32, 48, from_rank=1, to_rank=3)
+    exp = before.copy()
+    for i in range(3):
+        exp[3, 1024 + i * 48: 1024 + i * 48 + 20] = before[1, 64 + i * 32: 64 + i * 32 + 20]
+    assert np.array_equal(img.mem.reshape(W, bpr), exp)
+
+
 # ----------------------------------------------------------------------------- consumer
 def test_consumer_matches_library_float32_add():
     M, N = 9, 40
