@@ -396,7 +396,9 @@ def run_ours(args):
 
         # ---------------- all-store microbenchmark (replicated-store GB/s vs HBM peak) ----------------
         if args.sweep != "none":
-            result["all_store"] = all_store_sweep(iris, pk, args.sweep)
+            result["all_store"] = all_store_sweep(iris, pk, args.sweep, pull=0)
+            result["all_load"] = all_store_sweep(iris, pk, args.sweep, pull=1)
+            result["p2p"] = p2p_microbench(iris, pk)
 
         # ---------------- CPU oracle on a bounded sample of the same workload ----------------
         if not args.no_cpu_baseline:
@@ -413,8 +415,9 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def all_store_sweep(iris, pk, kind):
-    """W=8 all-store: message sizes 1 KiB .. (64 MiB | 1 GiB) in powers of 4; GB/s counts W*S read + W*W*S written."""
+def all_store_sweep(iris, pk, kind, pull=0):
+    """W=8 all-store (push) or all-load (pull): message sizes 1 KiB .. (64 MiB | 1 GiB) in powers of 4.
+    GB/s counts W*S read + W*W*S written (push) or W*W*S read + W*W*S written (pull)."""
     import torch
     W = 8
     top = 15 if kind == "full" else 13
@@ -436,23 +439,70 @@ def all_store_sweep(iris, pk, kind):
         iris.iris_flags_fill(h, flag_off, W * T, 0)
         stream = torch.cuda.current_stream()
         iters = 20 if S <= (1 << 24) else 5
-        iris.iris_all_store_bench(h, payload_off, recv_off, flag_off, S, tile, 1)
-        iris.iris_all_store_bench(h, payload_off, recv_off, flag_off, S, tile, 2)
+        iris.iris_all_store_bench(h, payload_off, recv_off, flag_off, S, tile, 1, 0, pull)
+        iris.iris_all_store_bench(h, payload_off, recv_off, flag_off, S, tile, 2, 0, pull)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         e0.record(stream)
         for i in range(iters):
-            iris.iris_all_store_bench(h, payload_off, recv_off, flag_off, S, tile, 3 + i)
+            iris.iris_all_store_bench(h, payload_off, recv_off, flag_off, S, tile, 3 + i, 0, pull)
         e1.record(stream)
         torch.cuda.synchronize()
         iris.iris_status_check(h)
         ms = e0.elapsed_time(e1) / iters
-        moved = float(W * S + W * W * S)
+        moved = float((W * W * S if pull else W * S) + W * W * S)
         out.append({"S": S, "ms": ms, "gbs": moved / ms / 1e6, "frac_of_hbm_peak": moved / ms / 1e6 / pk["hbm_gbs"],
                     "l2": "warm (working set below L2)" if W * W * S < (100 << 20) else "exceeds L2"})
         iris.iris_heap_destroy(h)
         del mem
         torch.cuda.empty_cache()
+    return out
+
+
+def p2p_microbench(iris, pk):
+    """Point-to-point put / get / copy / load / store between two emulated ranks (256 MiB) and atomic rates."""
+    import torch
+    nbytes = 256 << 20
+    bpr = 2 * nbytes + (64 << 20)
+    mem = torch.empty(3 * bpr, dtype=torch.uint8, device="cuda")
+    ext = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    h = iris.iris_heap_create(3, bpr, external_base=mem.data_ptr())
+    b0 = iris.iris_heap_base(h, 0)
+    stream = torch.cuda.current_stream()
+    rows, rb = nbytes // 65536, 65536
+
+    def timed(fn, iters=5):
+        fn(); fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(iters):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+
+    out = {}
+    ops = {"put": lambda: iris.iris_put_tile(h, b0, b0 + nbytes, rows, rb, rb, rb, 0, 1),
+           "get": lambda: iris.iris_get_tile(h, b0, b0 + nbytes, rows, rb, rb, rb, 0, 1),
+           "copy": lambda: iris.iris_copy_tile(h, b0, b0 + nbytes, rows, rb, rb, rb, 0, 1, 2),
+           "load": lambda: iris.iris_load_tile(h, b0, ext, rows, rb, rb, rb, 0, 1),
+           "store": lambda: iris.iris_store_tile(h, ext, b0, rows, rb, rb, rb, 0, 1)}
+    for name, fn in ops.items():
+        ms = timed(fn)
+        out[name] = {"bytes": nbytes, "ms": ms, "gbs": 2.0 * nbytes / ms / 1e6, "frac_of_hbm_peak": 2.0 * nbytes / ms / 1e6 / pk["hbm_gbs"]}
+    n = 1 << 24
+    flag_base = b0 + 2 * nbytes
+    iris.iris_flags_fill(h, 2 * nbytes, n, 0)
+    for name, fn in {"atomic_add": lambda: iris.iris_atomic_add(h, flag_base, n, 4, 0, 1, 1),
+                     "atomic_cas": lambda: iris.iris_atomic_cas(h, flag_base, n, 4, 0, 1, 0, 1, iris.IRIS_SEM_RELEASE),
+                     "atomic_xchg": lambda: iris.iris_atomic_rmw(h, iris.IRIS_OP_XCHG, flag_base, n, 4, 0, 1, 7),
+                     "atomic_add_one_word": lambda: iris.iris_atomic_add_contended(h, flag_base, n, 0, 1, 1)}.items():
+        ms = timed(fn, 3)
+        out[name] = {"ops": n, "ms": ms, "gops": n / ms / 1e6}
+    iris.iris_heap_destroy(h)
+    del mem, ext
+    torch.cuda.empty_cache()
     return out
 
 
