@@ -522,7 +522,7 @@ def main():
     ap.add_argument("--fused-consumer", type=int, default=0)
     ap.add_argument("--mode-iters", type=int, default=3)
     ap.add_argument("--e2e-steps", type=int, default=2)
-    ap.add_argument("--cpu-strips", type=int, default=16)
+    ap.add_argument("--cpu-strips", type=int, default=32)
     ap.add_argument("--sweep", default="short", choices=["none", "short", "full"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -20,7 +20,7 @@ def align(x, a=256):
     return (x + a - 1) // a * a
 
 
-def _run_fullsize(W, M, N, K, dist, dtype, mode, seed, n_sample, comm_ctas=0, with_consumer=True):
+def _run_fullsize(W, M, N, K, dist, dtype, mode, seed, n_sample, comm_ctas=0, with_consumer=True, fused=True):
     nl = N // W
     nt = iris.iris_num_tiles(M, N, W)
     flag_off = align(M * N * 2)
@@ -38,9 +38,13 @@ def _run_fullsize(W, M, N, K, dist, dtype, mode, seed, n_sample, comm_ctas=0, wi
         iris.iris_flags_fill(h, flag_off, nt, 0)
         iris.iris_flags_fill(h, lock_off, nt, 0)
         for epoch in (1, 2):           # the second pass runs over the first one's data, as the timed loop does
-            # the consumer rides inside the GEMM launch where the kernel supports it (what bench.py times), else follows it
+            # fused: the consumer rides inside the GEMM launch where the kernel supports it; otherwise it is the second
+            # kernel of the step, exactly as bench.py's default step launches it
             iris.iris_gemm_all_scatter_ex(h, dA, dB, M, N, K, W, iris.MODES[mode], iris.DTYPES[dtype], 0, flag_off, lock_off, epoch,
-                                          comm_ctas=comm_ctas, consumer_bias=dbias if with_consumer else None, consumer_out_off=out_off)
+                                          comm_ctas=comm_ctas, consumer_bias=dbias if (with_consumer and fused) else None,
+                                          consumer_out_off=out_off)
+            if with_consumer and not fused:
+                iris.iris_consume_bias(h, 0, out_off, flag_off, dbias, M, N, W, iris.DTYPES[dtype], epoch)
             iris.iris_status_check(h)
         slots = mem.view(W, bpr)
         c0 = slots[0, : M * N * 2]
@@ -68,9 +72,11 @@ def _run_fullsize(W, M, N, K, dist, dtype, mode, seed, n_sample, comm_ctas=0, wi
         iris.iris_heap_destroy(h)
 
 
-def test_bench_workload_workgroup_specialized_sampled_tiles():
-    """W=8, M=8192, N=K=16384, bf16 uniform[-1,1): the workload and schedule bench.py reports."""
-    _run_fullsize(8, 8192, 16384, 16384, "uniform", "bf16", "workgroup_specialized", inputs.SEED0 + 4, n_sample=10)
+@pytest.mark.parametrize("fused", [False, True], ids=["consumer_kernel", "consumer_warps"])
+def test_bench_workload_workgroup_specialized_sampled_tiles(fused):
+    """W=8, M=8192, N=K=16384, bf16 uniform[-1,1): the workload and schedule bench.py reports (its default step
+    launches the consumer as a second kernel; `fused_consumer_step` runs it as warps of the GEMM launch)."""
+    _run_fullsize(8, 8192, 16384, 16384, "uniform", "bf16", "workgroup_specialized", inputs.SEED0 + 4, n_sample=10, fused=fused)
 
 
 @pytest.mark.parametrize("mode", ["bulk_synchronous", "fused_sequential"])
