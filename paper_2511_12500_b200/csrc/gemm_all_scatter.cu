@@ -1047,6 +1047,13 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
         pair = false;
       }
     }
+    if (pair) {   // a cap on the grid that leaves no room for whole pairs: fall back to single-CTA tiles unless pairs were demanded
+      const int cap = a->max_ctas ? std::min(a->max_ctas, h->sm_count) : h->sm_count;
+      if ((cap & ~1) < (wg ? 4 : 2)) {
+        if (a->cta_pair > 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: max_ctas too small for CTA pairs");
+        pair = false;
+      }
+    }
     if (pair) bn = kPairBN;
     p.tab = h->table();
     p.c_off = a->c_off;
