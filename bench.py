@@ -43,7 +43,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 METRIC = "gemm_all_scatter_tflops"
 UNIT = "TFLOP/s"
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one workgroup_specialized launch on the default
-# workload, from the 1-pass ncu capture summarised in profiles/bench_default_launch_list.md: 6.22 GB + 2.10 GB.
+# workload, from a 1-pass ncu capture at full size: 6.22 GB read + 2.10 GB written.
 NCU_TRAFFIC_BYTES = {"cfg5_w8_m8192_n16384_k16384": 8.32e9}
 
 

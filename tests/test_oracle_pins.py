@@ -148,7 +148,7 @@ def test_gemm_matches_numpy_float64_matmul(dtype):
     ref = Ad @ Bcat.T
     bound = (np.abs(Ad) @ np.abs(Bcat).T) * 1e-12 + 1e-300
     assert np.all(np.abs(ref - c64) <= bound)
-    # the rounded result is the correctly rounded unrounded one (library cast as the judge for fp16)
+    # the rounded result is the correctly rounded unrounded one (numpy's direct double->half cast decides for fp16)
     if dtype == "fp16":
         assert np.array_equal(c16, c64.astype(np.float16).view(np.uint16))
 
