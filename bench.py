@@ -34,6 +34,10 @@ WORKLOADS = {
     # name: (W, M, N, K, dist, dtype)
     "cfg5_w8_m8192_n16384_k16384": (8, 8192, 16384, 16384, "uniform", "bf16"),
     "cfg5_w8_m1024_n16384_k16384": (8, 1024, 16384, 16384, "uniform", "bf16"),
+    "cfg5_w4_m8192_n16384_k16384": (4, 8192, 16384, 16384, "uniform", "bf16"),
+    "cfg5_w4_m1024_n16384_k16384": (4, 1024, 16384, 16384, "uniform", "bf16"),
+    "cfg5_w2_m8192_n16384_k16384": (2, 8192, 16384, 16384, "uniform", "bf16"),
+    "cfg5_w2_m1024_n16384_k16384": (2, 1024, 16384, 16384, "uniform", "bf16"),
     "cfg3_w8_m4096_n8192_k8192": (8, 4096, 8192, 8192, "normal002", "bf16"),
     "cfg4_w8_m128_n28672_k8192": (8, 128, 28672, 8192, "normal002", "bf16"),
     "cfg1_w2_256": (2, 256, 256, 256, "uniform", "fp16"),
