@@ -1,10 +1,15 @@
 // GEMM + all-scatter over the emulated symmetric heap, three schedules (Section 4, Listings 2-5).
 //
-// One persistent, warp-specialised kernel computes C tiles with tcgen05 MMAs:
+// Two persistent, warp-specialised tcgen05 kernels share this file:
+//   gemm_all_scatter_pair_kernel  a cluster of two CTAs per 256 x 256 tile (cta_group::2), tile ids claimed in
+//                                 raster order; the default whenever N/world is a multiple of 256 and M > 128
+//   gemm_all_scatter_kernel       one CTA per 128 x 256 or 128 x 128 tile, static tile stride; handles every
+//                                 ragged shape (TMA zero fill on loads, masks on stores)
+// Warp roles in a producer CTA:
 //   warp 0      TMA producer  (cp.async.bulk.tensor -> 128B-swizzled shared-memory stages, mbarrier ring)
 //   warp 1      MMA issuer    (one thread; tcgen05.mma into a double-buffered TMEM accumulator)
 //   warps 2..5  epilogue      (tcgen05.ld -> fp32 -> fp16/bf16 -> 16-byte global stores -> flags)
-// The tile loop is the paper's `for tile_id in range(pid, total_tiles, NUM_SMS)` (Listings 3-5).
+//   warps 6..9  consumer      (pair kernel, optional: acquire flags, OUT = C + bias)
 // What happens to a finished tile depends on the schedule:
 //   bulk_synchronous       store to the owner rank's slot; a second kernel scatters and publishes
 //   fused_sequential       store to all W slots from registers, then publish W ready flags
@@ -35,7 +40,7 @@ constexpr int kEpiThreads = 128;
 constexpr int kConsWarps = 4;     // optional consumer warps appended to every producer CTA of the pair kernel
 constexpr int kGemmThreadsFused = kGemmThreads + 32 * kConsWarps;
 constexpr int kConsUnroll = 16;   // 16-byte loads in flight per consumer lane
-constexpr int kPairBNc = 256;      // pair tile width (also used by the fused consumer's item decode)
+constexpr int kPairBNc = 256;     // pair tile width (also used by the fused consumer's item decode)
 constexpr int kSchedDepth = 4;    // pair kernel: tile ids in flight between the claiming thread and the other roles
 constexpr int kCommWarps = 6;     // communication CTA: every warp is a communicator with a 32 KB tile buffer
 constexpr int kTileBytes = IRIS_TILE * IRIS_TILE * 2;
@@ -59,11 +64,11 @@ struct alignas(64) GemmParams {
   uint64_t timeout_ns;
   int32_t* status;
   int M, N, K, n_local;
-  int tiles_m;          // ceil(M / 128)
+  int tiles_m;          // compute tile rows: ceil(M / 128), or ceil(M / 256) for CTA pairs
   int ctiles_per_rank;  // compute tiles per rank along N: ceil(N_local / BN)
   int ptiles_per_rank;  // publication tiles per rank along N: ceil(N_local / 128)
   int total_ctiles;     // tiles_m * W * ctiles_per_rank
-  int total_ptiles;     // tiles_m * W * ptiles_per_rank
+  int total_ptiles;     // ptiles_m * W * ptiles_per_rank
   int kblocks;          // ceil(K / 64)
   int ptiles_m;         // publication tile rows: ceil(M / 128)
   int dynamic;          // pair kernel: 1 = tiles are claimed from *tile_counter in raster order, 0 = static stride
