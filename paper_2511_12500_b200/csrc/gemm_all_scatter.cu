@@ -747,12 +747,14 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
             for (int s = 0; s < W; ++s) {
               const uint64_t dst = p.tab.base[s] + row_off + (uint64_t)c0 * 2;
 #pragma unroll
-              for (int i = 0; i < 4; ++i) st_global_v4(reinterpret_cast<void*>(dst + 16 * i), q[i]);
+              for (int i = 0; i < 4; ++i)
+                if (c0 + 8 * i < p.n_local) st_global_v4(reinterpret_cast<void*>(dst + 16 * i), q[i]);
             }
           } else {
             const uint64_t dst = p.tab.base[tc.rank] + row_off + (uint64_t)c0 * 2;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) st_global_v4(reinterpret_cast<void*>(dst + 16 * i), q[i]);
+            for (int i = 0; i < 4; ++i)
+              if (c0 + 8 * i < p.n_local) st_global_v4(reinterpret_cast<void*>(dst + 16 * i), q[i]);
           }
         }
       }
@@ -768,12 +770,18 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
           if (p.mode == IRIS_MODE_FUSED_SEQUENTIAL) {
             if (et < subs * W) {
               const int sub = et / W, s = et % W;
-              const int t = tm * pt_n + tc.rank * p.ptiles_per_rank + tc.jn * subs + sub;
-              st_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[s] + p.flag_off) + t, p.epoch);
+              const int pj = tc.jn * subs + sub;
+              if (pj < p.ptiles_per_rank) {   // a ragged shard's last tile may have only one publication tile
+                const int t = tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
+                st_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[s] + p.flag_off) + t, p.epoch);
+              }
             }
           } else if (et < subs) {
-            const int t = tm * pt_n + tc.rank * p.ptiles_per_rank + tc.jn * subs + et;
-            (void)cas_release_gpu(lock_addr<STATIC_LOCKS>(p, tc.rank, t), 0, 1);
+            const int pj = tc.jn * subs + et;
+            if (pj < p.ptiles_per_rank) {
+              const int t = tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
+              (void)cas_release_gpu(lock_addr<STATIC_LOCKS>(p, tc.rank, t), 0, 1);
+            }
           }
         }
       }
@@ -1038,11 +1046,14 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
       if ((int64_t)((a->M + BM - 1) / BM) * W * ((nl + 255) / 256) < h->sm_count) bn = 128;
     }
     if (nl <= 128) bn = 128;
-    // CTA pairs (256 x 256 tiles) when the shard is a whole number of 256-column tiles and there are at
-    // least two tile rows; otherwise the single-CTA kernel, which also handles every ragged case.
-    const bool pair_ok = nl % 256 == 0 && a->M > BM && a->block_n != 128 && h->sm_count >= 4;
-    if (a->cta_pair > 0 && !pair_ok) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: cta_pair needs (N/world) %% 256 == 0, M > 128 and block_n != 128");
-    pair = a->cta_pair >= 0 && pair_ok;
+    // CTA pairs (256 x 256 tiles) need at least two tile rows.  A shard that is not a whole number of 256-column
+    // tiles is fine (TMA zero-fills the missing B rows, stores and flags are masked) but wastes MMA work on the
+    // padding: by default pairs are used when that waste is at most 15 %, otherwise the single-CTA kernel with
+    // its narrower tiles.
+    const bool pair_ok = a->M > BM && nl > BM && a->block_n != 128 && h->sm_count >= 4;
+    if (a->cta_pair > 0 && !pair_ok) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: cta_pair needs M > 128, N/world > 128 and block_n != 128");
+    const bool pair_pays = (int64_t)((nl + 255) / 256) * 256 * 100 <= (int64_t)nl * 115;
+    pair = pair_ok && (a->cta_pair > 0 || (a->cta_pair == 0 && pair_pays));
     int max_pairs = 0;
     if (pair) {
       const int rc = a->dtype == IRIS_BF16 ? launch_gemm_pair<true>(p, 0, nullptr, &max_pairs) : launch_gemm_pair<false>(p, 0, nullptr, &max_pairs);

@@ -92,6 +92,8 @@ EXACT_SHAPES = [
     (2, 300, 640, 64),         # N_local > 512 and not a multiple of 256
     (2, 1000, 512, 200),       # CTA-pair tiles (256 x 256), ragged M: the last pair's second CTA has no rows
     (8, 257, 256, 64),         # CTA-pair tiles, one row in the second tile row
+    (2, 600, 448, 136),        # CTA-pair tiles with a ragged shard (448 = 256 + 192): masked stores, 4 flags of 4 + 2 of 4
+    (3, 384, 904, 64),         # 904 = 3 * 256 + 136: the last pair tile has two publication tiles, the second 8 columns wide
 ]
 
 

@@ -84,6 +84,8 @@ def test_random_shapes_exact_heap_image():
             kw["static_schedule"] = 1
         if rng.random() < 0.2:
             kw["cta_pair"] = -1
+        elif rng.random() < 0.4 and M > 128 and nl > 128:
+            kw["cta_pair"] = 1      # pairs even where the shard is ragged
         dtype = "bf16" if case % 2 else "fp16"
         N = W * nl
         A = inputs.matrix(900 + case, inputs.STREAM_A, M, K, "ternary:0.5", dtype)
