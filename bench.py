@@ -41,6 +41,12 @@ WORKLOADS = {
     "cfg3_w8_m4096_n8192_k8192": (8, 4096, 8192, 8192, "normal002", "bf16"),
     "cfg4_w8_m128_n28672_k8192": (8, 128, 28672, 8192, "normal002", "bf16"),
     "cfg1_w2_256": (2, 256, 256, 256, "uniform", "fp16"),
+    # the two shapes the paper names in Section 5.2 (M x N x K = 8192 x 4608 x 36864 and 8192 x 3584 x 14336, 8 ranks);
+    # the text does not say whether N is per rank or global, so both readings are available
+    "paper_8192x4608x36864_w8_n_per_rank": (8, 8192, 8 * 4608, 36864, "normal002", "bf16"),
+    "paper_8192x3584x14336_w8_n_per_rank": (8, 8192, 8 * 3584, 14336, "normal002", "bf16"),
+    "paper_8192x4608x36864_w8_n_global": (8, 8192, 4608, 36864, "normal002", "bf16"),
+    "paper_8192x3584x14336_w8_n_global": (8, 8192, 3584, 14336, "normal002", "bf16"),
 }
 DEFAULT_WORKLOAD = "cfg5_w8_m8192_n16384_k16384"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
