@@ -219,7 +219,7 @@ typedef struct iris_gemm_args {
   int block_n;                 /* compute-tile width: 0 = auto, 128 or 256                       */
   uint64_t spin_timeout_ns;    /* deadline of every device-side wait (0 = 2 s)                   */
   int cta_pair;                /* 0 = use 256 x 256 CTA-pair tiles (tcgen05 cta_group::2) when M > 128
-                                  and N/world fills its 256-column tiles to at least 87 %;
+                                  and N/world > 128 (a ragged last tile is padded);
                                   1 = use them whenever M > 128 and N/world > 128
                                   (IRIS_ERR_UNSUPPORTED otherwise); -1 = single-CTA tiles only   */
   int static_schedule;         /* CTA-pair kernel: 0 = pairs claim tile ids in raster order from

@@ -1047,12 +1047,13 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     }
     if (nl <= 128) bn = 128;
     // CTA pairs (256 x 256 tiles) need at least two tile rows.  A shard that is not a whole number of 256-column
-    // tiles is fine (TMA zero-fills the missing B rows, stores and flags are masked) but wastes MMA work on the
-    // padding: by default pairs are used when that waste is at most 15 %, otherwise the single-CTA kernel with
-    // its narrower tiles.
+    // tiles is fine (TMA zero-fills the missing B rows, stores and flags are masked) but spends MMA work on the
+    // padding.  Measured on a 576-column shard (33 % padding) pairs still take 2.44 ms where 128-wide single-CTA
+    // tiles (11 % padding) take 3.26 ms: per padded flop the pair kernel is about 1.6x as fast, so pairs are the
+    // default unless their padding exceeds the narrow tiles' by more than 1.5x.
     const bool pair_ok = a->M > BM && nl > BM && a->block_n != 128 && h->sm_count >= 4;
     if (a->cta_pair > 0 && !pair_ok) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: cta_pair needs M > 128, N/world > 128 and block_n != 128");
-    const bool pair_pays = (int64_t)((nl + 255) / 256) * 256 * 100 <= (int64_t)nl * 115;
+    const bool pair_pays = (int64_t)((nl + 255) / 256) * 256 * 2 <= (int64_t)((nl + 127) / 128) * 128 * 3;
     pair = pair_ok && (a->cta_pair > 0 || (a->cta_pair == 0 && pair_pays));
     int max_pairs = 0;
     if (pair) {
