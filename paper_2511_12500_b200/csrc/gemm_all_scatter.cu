@@ -531,6 +531,8 @@ __device__ void consumer_warp(const GemmParams& p, CtrlBlock* ctrl, int cwarp, i
     const uint64_t src = p.tab.base[s] + p.c_off + tile_off;
     const uint64_t dst = p.tab.base[s] + p.out_off + tile_off;
     const int ch = lane & 15;  // 16-byte chunk within the 256-byte tile row
+    const int cols = min(IRIS_TILE, p.n_local - pj * IRIS_TILE);
+    if (ch * 8 >= cols) continue;  // ragged shard: the last publication tile is narrower (whole chunks: N_local % 8 == 0)
     const uint4 b = *reinterpret_cast<const uint4*>(p.bias + (col0 + (uint64_t)ch * 8) * 2);
     // 2 rows per pass, kConsUnroll passes (= 8 KB per warp) in flight: at ~2 us of loaded-memory latency that is
     // ~4 GB/s per warp, several times the 1.3 GB/s each warp must sustain to keep up with the GEMM.
