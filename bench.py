@@ -229,9 +229,10 @@ def run_ours(args):
     flops = 2.0 * M * N * K
     store_bytes = float(W) * M * N * 2
 
-    def gemm(epoch, m=mode, fused=False, **kw):
+    def gemm(epoch, m=mode, fused=False, wg_tail=None, **kw):
         iris.iris_gemm_all_scatter_ex(h, dA, dB, M, N, K, W, m, dt, 0, flag_off, lock_off, epoch, comm_ctas=args.comm_ctas,
-                                      raster_group=args.raster_group, block_n=args.block_n, cta_pair=args.cta_pair, static_schedule=args.static_schedule,
+                                      raster_group=args.raster_group, block_n=args.block_n, cta_pair=args.cta_pair, static_schedule=args.static_schedule, stream_k=args.stream_k,
+                                      wg_tail=args.wg_tail if wg_tail is None else wg_tail,
                                       consumer_bias=dbias if fused else None, consumer_out_off=out_off, **kw)
 
     def consume(epoch):
@@ -298,6 +299,7 @@ def run_ours(args):
         # ---------------- roofline of the dominant kernel ----------------
         t_tensor = flops / (pk["bf16_tflops"] * 1e12) * 1e3
         t_store = store_bytes / (pk["hbm_gbs"] * 1e9) * 1e3
+        t_bytes = ((M * K + N * K) * 2.0 + store_bytes) / (pk["hbm_gbs"] * 1e9) * 1e3   # operand reads + replicated stores
         achieved = flops / (gemm_ms * 1e-3) / 1e12
         result["roofline"] = {"kernel": f"gemm_all_scatter_pair_kernel<bf16> ({args.mode}); single-CTA kernel when --cta-pair -1 or the shape needs it", "bound": "tensor", "achieved": achieved,
                               "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / pk["bf16_tflops"],
@@ -306,6 +308,7 @@ def run_ours(args):
                               "algorithmic_bytes": (M * K + N * K) * 2.0 + store_bytes,
                               "kernel_ms": gemm_ms, "combined_roofline_ms": max(t_tensor, t_store),
                               "frac_of_combined_roofline": max(t_tensor, t_store) / gemm_ms,
+                              "full_traffic_roofline_ms": max(t_tensor, t_bytes), "frac_of_full_traffic_roofline": max(t_tensor, t_bytes) / gemm_ms,
                               "replicated_store_gbs": store_bytes / (gemm_ms * 1e-3) / 1e9}
         cons_bytes = 2.0 * store_bytes + N * 2
         if fused:   # time the stand-alone consumer kernel too, for its own HBM figure
@@ -324,18 +327,31 @@ def run_ours(args):
 
         # ---------------- the three schedules on the same workload (context for the headline) ----------------
         modes = {}
-        for name, m in (iris.MODES.items() if args.mode_iters > 0 else ()):
-            ts = []
-            for _ in range(1 + args.mode_iters):
+        # Round-robin over the variants, one launch each per round, so that clock drift under the power cap (launch times
+        # grow by 10-30 % over the first few hundred ms of continuous load) hits all of them alike.
+        variants = list(iris.MODES.items()) + [("workgroup_specialized_every_tile_via_comm_ctas", iris.IRIS_MODE_WORKGROUP_SPECIALIZED)]
+        tA = dA.view(torch.bfloat16 if dtype == "bf16" else torch.float16).view(M, K)
+        tB = torch.cat([b.view(tA.dtype).view(nl, K) for b in dB], dim=0)
+        variants.append(("library_gemm_no_scatter", None))   # context: cuBLAS through torch.matmul, same operands, same moment
+        series = {name: [] for name, _ in variants}
+        for it in range(1 + args.mode_iters if args.mode_iters > 0 else 0):
+            for name, m in variants:
                 epoch += 1
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
-                gemm(epoch, m)
+                if m is None:
+                    tC = tA @ tB.t()
+                else:
+                    gemm(epoch, m, wg_tail=-1 if name.endswith("comm_ctas") else None)
                 e1.record(stream)
                 torch.cuda.synchronize()
-                ts.append(e0.elapsed_time(e1))
-            ms = float(np.median(ts[1:]))
-            modes[name] = {"ms": ms, "tflops": flops / ms / 1e9, "store_gbs": store_bytes / ms / 1e6,
+                if it > 0:
+                    series[name].append(e0.elapsed_time(e1))
+        for name, ts in series.items():
+            if not ts:
+                continue
+            ms = float(np.median(ts))
+            modes[name] = {"ms": ms, "ms_min": float(min(ts)), "tflops": flops / ms / 1e9, "store_gbs": store_bytes / ms / 1e6,
                            "frac_of_combined_roofline": max(t_tensor, t_store) / ms}
         iris.iris_status_check(h)
         result["modes"] = modes
@@ -362,8 +378,6 @@ def run_ours(args):
         # Not part of the path and not a target: it shows what the same data, clocks and power cap give a plain
         # GEMM without any scatter, next to the burst / sustained peaks measured on other data.
         try:
-            tA = dA.view(torch.bfloat16 if dtype == "bf16" else torch.float16).view(M, K)
-            tB = torch.cat([b.view(tA.dtype).view(nl, K) for b in dB], dim=0)
             for _ in range(3):
                 tC = tA @ tB.t()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -530,6 +544,8 @@ def main():
     ap.add_argument("--cta-pair", type=int, default=0)
     ap.add_argument("--static-schedule", type=int, default=0)
     ap.add_argument("--fused-consumer", type=int, default=0)
+    ap.add_argument("--stream-k", type=int, default=0)
+    ap.add_argument("--wg-tail", type=int, default=0, help="workgroup_specialized: 0 = producers scatter the last wave themselves, -1 = never, n = last n tiles")
     ap.add_argument("--mode-iters", type=int, default=3)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-strips", type=int, default=32)

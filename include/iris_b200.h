@@ -226,6 +226,19 @@ typedef struct iris_gemm_args {
                                   an atomic counter as they become free; 1 = the listings' static
                                   loop tile = pid, pid + NUM, ... (the single-CTA kernel always
                                   uses the static loop)                                          */
+  int stream_k;                /* single-CTA kernel: 1 = split the k-steps of all tiles into equal
+                                  ranges, one per CTA; tiles that straddle ranges are computed in
+                                  parts and reduced in k order through a workspace the heap
+                                  allocates on first use; 0 and -1 = whole tiles only (measured
+                                  faster on every benchmark shape, hence the default)            */
+  int wg_tail;                 /* workgroup-specialised: which compute tiles the producers scatter
+                                  themselves (to all W slots from registers, as fused_sequential
+                                  does) instead of handing them to the communication CTAs.
+                                  0 = the last wave (the last P tiles of the raster order, P =
+                                  producer CTAs or pairs: no GEMM work is left to overlap their
+                                  scatter with, and all store ports beat a few); n > 0 = the last
+                                  n tiles; -1 = none (Listing 5 for every tile).  The final heap
+                                  image is the same in every case                                */
   const void* consumer_bias;   /* not NULL: also run the flag-gated consumer OUT = C + bias (see
                                   iris_consume_bias) as part of this call: inside the same launch,
                                   as extra warps that acquire each tile's flag while the GEMM is

@@ -23,6 +23,7 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
+#include <climits>
 #include <cmath>
 #include <cstring>
 #include <mutex>
@@ -76,6 +77,11 @@ struct alignas(64) GemmParams {
   const uint8_t* bias;  // fused consumer: bias[N] of the element type (NULL = no consumer warps)
   uint64_t out_off;     // fused consumer: OUT region in every slot
   int gemm_ctas, comm_ctas;
+  int streamk;          // single-CTA kernel: 1 = equal k-step ranges per CTA (tiles may be computed in parts)
+  float* ws;            // stream-K: two fp32 tile slots per CTA for partial sums
+  int32_t* arrive;      // stream-K: per compute tile, how many parts have been parked
+  int seq_from;         // compute tiles with raster id >= seq_from are scattered by their producer (Listing 4's loop); 0 in
+                        // fused_sequential mode, the first tile of the last wave in workgroup_specialized mode
   int raster_group;
   int mode;
   int32_t epoch;
@@ -92,6 +98,7 @@ struct CtrlBlock {  // lives in shared memory after the payload area
   volatile int32_t sched_tile[kSchedDepth];
   uint32_t tmem_base;
   volatile int abort;
+  volatile int last_part;   // stream-K: this CTA parked the last part of the tile and reduces it
 };
 
 struct TileCoord { int tm, rank, jn; };
@@ -195,7 +202,7 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
   const int W = p.tab.world;
   const int ncw = p.comm_ctas * kCommWarps;
   const int cw = ((int)blockIdx.x - p.gemm_ctas) * kCommWarps + warp;
-  const int items = p.total_ctiles * SUBS * SUBS_M;
+  const int items = min(p.total_ctiles, p.seq_from) * SUBS * SUBS_M;   // the tail wave's tiles are scattered by their producers
   const int n_my = cw < items ? (items - cw + ncw - 1) / ncw : 0;  // items cw, cw + ncw, ...
   const int pt_n = W * p.ptiles_per_rank;
   const uint32_t buf = ptx::smem_u32(payload + warp * kTileBytes);
@@ -304,8 +311,54 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
 }
 
 // ------------------------------------------------------------------------------------------------
-// The GEMM + scatter kernel.
+// The single-CTA GEMM + scatter kernel.
+//
+// Work is handed out as segments (tile, kb0, kb1) of the k-loop:
+//   static stride   CTA c takes whole tiles c, c + NUM, ... (the listings' loop): every segment is a full tile
+//   stream-K        the T x KB k-steps of all tiles are cut into NUM equal, contiguous ranges, one per CTA, so
+//                   every SM streams the same number of operand bytes whatever T mod NUM is (the skinny,
+//                   memory-bound shapes: one tile row, a tile count that is not a multiple of the SM count).
+//                   A tile that straddles two or more ranges is computed in parts: each part's fp32 accumulator
+//                   goes to a workspace slot, the part that arrives last (one atomic per part) adds the parts in
+//                   k order -- a fixed order, so the result does not depend on who was last -- converts,
+//                   scatters and publishes.
 // ------------------------------------------------------------------------------------------------
+struct Segment { int tile, kb0, kb1; bool first; };
+
+struct SegmentIter {
+  long long u, u_end;   // stream-K: next k-step unit and end of this CTA's range
+  int tile, stride;     // static: next tile and stride
+  bool streamk, started;
+  __device__ __forceinline__ SegmentIter(const GemmParams& p, int cta) : started(false) {
+    streamk = p.streamk != 0;
+    const long long units = (long long)p.total_ctiles * p.kblocks;
+    u = streamk ? units * cta / p.gemm_ctas : 0;
+    u_end = streamk ? units * (cta + 1) / p.gemm_ctas : 0;
+    tile = cta;
+    stride = p.gemm_ctas;
+  }
+  __device__ __forceinline__ bool next(const GemmParams& p, Segment& s) {
+    if (streamk) {
+      if (u >= u_end) return false;
+      s.tile = (int)(u / p.kblocks);
+      s.kb0 = (int)(u % p.kblocks);
+      s.kb1 = (int)min((long long)p.kblocks, s.kb0 + (u_end - u));
+      s.first = !started;
+      u += s.kb1 - s.kb0;
+    } else {
+      if (tile >= p.total_ctiles) return false;
+      s.tile = tile; s.kb0 = 0; s.kb1 = p.kblocks; s.first = !started;
+      tile += stride;
+    }
+    started = true;
+    return true;
+  }
+};
+
+// stream-K bookkeeping: which CTA's range holds k-step unit x, and where that CTA's range starts
+__device__ __forceinline__ int streamk_cta_of(long long x, long long units, int ctas) { return (int)(((x + 1) * ctas + units - 1) / units - 1); }
+__device__ __forceinline__ long long streamk_begin(int cta, long long units, int ctas) { return units * cta / ctas; }
+
 template <int BN, bool BF16, bool STATIC_LOCKS = false>
 __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const __grid_constant__ GemmParams p) {
   using Cfg = TileCfg<BN>;
@@ -346,10 +399,12 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < p.total_ctiles && ok; tile += p.gemm_ctas) {
-        const TileCoord tc = decode_ctile(tile, p);
-        for (int kb = 0; kb < p.kblocks; ++kb) {
-          if (!mbar_wait(ptx::smem_u32(&ctrl->empty[stage]), phase ^ 1, p, ctrl, tile)) { ok = false; break; }
+      SegmentIter it(p, (int)blockIdx.x);
+      Segment sg;
+      while (ok && it.next(p, sg)) {
+        const TileCoord tc = decode_ctile(sg.tile, p);
+        for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
+          if (!mbar_wait(ptx::smem_u32(&ctrl->empty[stage]), phase ^ 1, p, ctrl, sg.tile)) { ok = false; break; }
           const uint32_t bar = ptx::smem_u32(&ctrl->full[stage]);
           uint8_t* sa = payload + stage * Cfg::kStageBytes;
           ptx::mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
@@ -367,24 +422,26 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < p.total_ctiles && ok; tile += p.gemm_ctas) {
-        if (!mbar_wait(ptx::smem_u32(&ctrl->tmem_empty[acc]), acc_phase ^ 1, p, ctrl, tile)) break;
+      SegmentIter it(p, (int)blockIdx.x);
+      Segment sg;
+      while (ok && it.next(p, sg)) {
+        if (!mbar_wait(ptx::smem_u32(&ctrl->tmem_empty[acc]), acc_phase ^ 1, p, ctrl, sg.tile)) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < p.kblocks; ++kb) {
-          if (!mbar_wait(ptx::smem_u32(&ctrl->full[stage]), phase, p, ctrl, tile)) { ok = false; break; }
+        for (int kb = sg.kb0; kb < sg.kb1; ++kb) {
+          if (!mbar_wait(ptx::smem_u32(&ctrl->full[stage]), phase, p, ctrl, sg.tile)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t sa = ptx::smem_u32(payload + stage * Cfg::kStageBytes);
           const uint64_t adesc = ptx::smem_desc_k_sw128(sa);
           const uint64_t bdesc = ptx::smem_desc_k_sw128(sa + BM * BK * 2);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k)  // +32 bytes per K step: +2 in the (>>4) address field
-            ptx::mma_f16_ss(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+            ptx::mma_f16_ss(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb > sg.kb0) || k != 0);
           ptx::mma_commit(ptx::smem_u32(&ctrl->empty[stage]));  // stage reusable once these MMAs have read it
           if (++stage == Cfg::kStages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
-        ptx::mma_commit(ptx::smem_u32(&ctrl->tmem_full[acc]));  // accumulator complete
+        ptx::mma_commit(ptx::smem_u32(&ctrl->tmem_full[acc]));  // accumulator (of this segment) complete
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       }
     }
@@ -395,19 +452,25 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
     int acc = 0;
     uint32_t acc_phase = 0;
     const uint32_t tmem_base = ctrl->tmem_base;
-    for (int tile = blockIdx.x; tile < p.total_ctiles; tile += p.gemm_ctas) {
+    const long long units = (long long)p.total_ctiles * p.kblocks;
+    SegmentIter it(p, (int)blockIdx.x);
+    Segment sg;
+    while (it.next(p, sg)) {
+      const int tile = sg.tile;
       const TileCoord tc = decode_ctile(tile, p);
       const bool ok = mbar_wait(ptx::smem_u32(&ctrl->tmem_full[acc]), acc_phase, p, ctrl, tile);
       if (ptx::bar_red_or(1, kEpiThreads, !ok)) break;  // uniform decision for all four warps
       ptx::tc_fence_after();
-      const int row = tc.tm * BM + quad * 32 + lane;
+      const bool whole = sg.kb0 == 0 && sg.kb1 == p.kblocks;   // this CTA computed the tile's entire k range
+      const bool seq = tile >= p.seq_from;                      // scatter from registers (Listing 4) or hand over (Listing 5)
+      const int row_in_tile = quad * 32 + lane;
+      const int row = tc.tm * BM + row_in_tile;
       const int col_in_shard = tc.jn * BN;
       const uint64_t row_off = p.c_off + ((uint64_t)row * p.N + (uint64_t)tc.rank * p.n_local) * 2;
-#pragma unroll 1
-      for (int ch = 0; ch < BN / 32; ++ch) {
-        uint32_t v[32];
-        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + ch * 32), v);
-        ptx::tmem_wait_ld();
+      const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN);
+
+      // converts 32 fp32 columns of this thread's row and stores them where the schedule wants them
+      auto emit = [&](const uint32_t (&v)[32], int ch) {
         uint4 q[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -422,7 +485,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
         }
         if (row < p.M) {
           const int c0 = col_in_shard + ch * 32;
-          if (p.mode == IRIS_MODE_FUSED_SEQUENTIAL) {
+          if (seq) {
             // Listing 4: for remote_rank in range(world_size): iris.store(C + offset, c, cur_rank, remote_rank)
             for (int s = 0; s < W; ++s) {
               const uint64_t dst = p.tab.base[s] + row_off + (uint64_t)c0 * 2;  // translate(C + offset, rank -> s)
@@ -438,18 +501,76 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
               if (c0 + 8 * i < p.n_local) st_global_v4(reinterpret_cast<void*>(dst + 16 * i), q[i]);
           }
         }
+      };
+      auto release_accumulator = [&]() {
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[acc]));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      };
+
+      bool publish = true;
+      if (whole) {
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          uint32_t v[32];
+          ptx::tmem_ld_32x32(t_addr + (uint32_t)(ch * 32), v);
+          ptx::tmem_wait_ld();
+          emit(v, ch);
+        }
+        release_accumulator();   // accumulator drained: hand it back to the MMA warp
+      } else {
+        // ---- stream-K: a part of the tile.  Park the fp32 partial sums, then see whether we are the last part. ----
+        float* mine = p.ws + (size_t)(2 * (int)blockIdx.x + (sg.first ? 0 : 1)) * (BM * BN) + (size_t)row_in_tile * BN;
+#pragma unroll 1
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          uint32_t v[32];
+          ptx::tmem_ld_32x32(t_addr + (uint32_t)(ch * 32), v);
+          ptx::tmem_wait_ld();
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            st_global_v4(mine + ch * 32 + 4 * i, make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
+        }
+        release_accumulator();
+        const int c_lo = streamk_cta_of((long long)tile * p.kblocks, units, p.gemm_ctas);
+        const int c_hi = streamk_cta_of((long long)tile * p.kblocks + p.kblocks - 1, units, p.gemm_ctas);
+        __threadfence();   // the partial sums are visible device-wide before our arrival is counted
+        asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
+        if (et == 0) ctrl->last_part = atomic_rmw<false>(p.arrive + tile, 0, 1, IRIS_SEM_ACQ_REL, IRIS_SCOPE_GPU) == c_hi - c_lo;
+        asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
+        publish = ctrl->last_part != 0;
+        if (publish) {
+          __threadfence();
+#pragma unroll 1
+          for (int ch = 0; ch < BN / 32; ++ch) {
+            float sum[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) sum[i] = 0.0f;
+            for (int c = c_lo; c <= c_hi; ++c) {   // parts in k order: CTA c_lo holds the lowest k range
+              const bool its_first = streamk_begin(c, units, p.gemm_ctas) >= (long long)tile * p.kblocks;
+              const float* part = p.ws + (size_t)(2 * c + (its_first ? 0 : 1)) * (BM * BN) + (size_t)row_in_tile * BN + ch * 32;
+#pragma unroll
+              for (int i = 0; i < 8; ++i) {
+                const uint4 w = ld_global_v4(part + 4 * i);
+                sum[4 * i + 0] += __uint_as_float(w.x);
+                sum[4 * i + 1] += __uint_as_float(w.y);
+                sum[4 * i + 2] += __uint_as_float(w.z);
+                sum[4 * i + 3] += __uint_as_float(w.w);
+              }
+            }
+            uint32_t v[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(sum[i]);
+            emit(v, ch);
+          }
+        }
       }
-      // accumulator drained: hand it back to the MMA warp
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[acc]));
-      if (++acc == 2) { acc = 0; acc_phase ^= 1; }
-      if (p.mode != IRIS_MODE_BULK_SYNCHRONOUS) {
+      if (publish && p.mode != IRIS_MODE_BULK_SYNCHRONOUS) {
         // every epilogue thread's stores happen-before the barrier; the release below is cumulative
         asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
         const int subs = BN / IRIS_TILE;
         const int pt_n = W * p.ptiles_per_rank;
-        if (p.mode == IRIS_MODE_FUSED_SEQUENTIAL) {
+        if (seq) {
           if (et < subs * W) {
             const int sub = et / W, s = et % W;
             const int pj = tc.jn * subs + sub;
@@ -726,6 +847,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
       const int row = tm * BM + quad * 32 + lane;
       const int col_in_shard = tc.jn * kPairBN;
       const uint64_t row_off = p.c_off + ((uint64_t)row * p.N + (uint64_t)tc.rank * p.n_local) * 2;
+      const bool seq = tile >= p.seq_from;   // scatter from registers (Listing 4) or hand over to the communicators (Listing 5)
 #pragma unroll 1
       for (int ch = 0; ch < kPairBN / 32; ++ch) {
         uint32_t v[32];
@@ -745,7 +867,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         }
         if (row < p.M) {
           const int c0 = col_in_shard + ch * 32;
-          if (p.mode == IRIS_MODE_FUSED_SEQUENTIAL) {
+          if (seq) {
             for (int s = 0; s < W; ++s) {
               const uint64_t dst = p.tab.base[s] + row_off + (uint64_t)c0 * 2;
 #pragma unroll
@@ -769,7 +891,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         constexpr int subs = kPairBN / IRIS_TILE;
         const int pt_n = W * p.ptiles_per_rank;
         if (tm < p.ptiles_m) {
-          if (p.mode == IRIS_MODE_FUSED_SEQUENTIAL) {
+          if (seq) {
             if (et < subs * W) {
               const int sub = et / W, s = et % W;
               const int pj = tc.jn * subs + sub;
@@ -879,6 +1001,14 @@ static int launch_gemm(const GemmParams& p, int grid, bool cooperative, cudaStre
   cfg.blockDim = dim3(kGemmThreads);
   cfg.dynamicSmemBytes = kSmemTotal;
   cfg.stream = st;
+  if (cooperative) {   // CTAs that wait on one another: refuse, with a clear message, a grid that cannot be resident all at once
+    int per_sm = 0, dev = 0, sms = 0;
+    IRIS_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kGemmThreads, kSmemTotal));
+    IRIS_CUDA_TRY(cudaGetDevice(&dev));
+    IRIS_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    if (grid > per_sm * sms)
+      return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: %d CTAs cannot be co-resident (%d per SM x %d SMs)", grid, per_sm, sms);
+  }
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeCooperative;  // CTAs that wait on one another must be co-resident
   attr[0].val.cooperative = cooperative ? 1 : 0;
@@ -936,10 +1066,10 @@ struct PlanKey {
   const void* A; const void* B[IRIS_MAX_WORLD];
   int M, N, K, world, mode, dtype;
   uint64_t c_off, flag_off, lock_off;
-  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule;
+  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail;
   uint64_t spin_timeout_ns;
 };
-struct Plan { GemmParams p; int bn, grid; bool pair; };
+struct Plan { GemmParams p; int bn, grid; bool pair, streamk; };
 static std::mutex g_plan_mutex;
 static Plan g_plan;
 static PlanKey g_plan_key;
@@ -953,7 +1083,7 @@ static void make_key(PlanKey* k, const iris_gemm_args* a, const iris_heap* h) {
   k->M = a->M; k->N = a->N; k->K = a->K; k->world = a->world; k->mode = a->mode; k->dtype = a->dtype;
   k->c_off = a->c_off; k->flag_off = a->flag_off; k->lock_off = a->lock_off;
   k->comm_ctas = a->comm_ctas; k->max_ctas = a->max_ctas; k->raster_group = a->raster_group; k->block_n = a->block_n;
-  k->cta_pair = a->cta_pair; k->static_schedule = a->static_schedule;
+  k->cta_pair = a->cta_pair; k->static_schedule = a->static_schedule; k->stream_k = a->stream_k; k->wg_tail = a->wg_tail;
   k->spin_timeout_ns = a->spin_timeout_ns;
 }
 
@@ -998,6 +1128,8 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   if (a->c_off % 256 != 0 || a->flag_off % 4 != 0 || a->lock_off % 4 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: misaligned heap offsets");
   if (a->comm_ctas < 0 || a->max_ctas < 0 || a->raster_group < 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: negative tuning parameter");
   if (a->cta_pair < -1 || a->cta_pair > 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: cta_pair must be -1, 0 or 1");
+  if (a->wg_tail < -1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: wg_tail must be -1, 0 or a tile count");
+  if (a->stream_k < -1 || a->stream_k > 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: stream_k must be -1, 0 or 1");
   const int64_t nt = num_tiles(a->M, a->N, W);
   const uint64_t bpr = h->bytes_per_rank;
   const uint64_t c_bytes = (uint64_t)a->M * a->N * 2;
@@ -1027,14 +1159,14 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   // call with the same arguments over and over, so the last plan is kept and re-used when nothing else changed.
   GemmParams p;
   int bn = 0, grid = 0;
-  bool pair = false;
+  bool pair = false, streamk = false;
   PlanKey key;
   make_key(&key, a, h);
   bool hit = false;
   {
     std::lock_guard<std::mutex> lock(g_plan_mutex);
     if (g_plan_valid && std::memcmp(&key, &g_plan_key, sizeof(key)) == 0) {
-      p = g_plan.p; bn = g_plan.bn; grid = g_plan.grid; pair = g_plan.pair;
+      p = g_plan.p; bn = g_plan.bn; grid = g_plan.grid; pair = g_plan.pair; streamk = g_plan.streamk;
       hit = true;
     }
   }
@@ -1043,9 +1175,10 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     bn = a->block_n;
     if (bn == 0) {
       bn = (nl % 256 == 0 || nl > 1024) ? 256 : 128;
-      // skinny problems (one tile row): 256-wide tiles would leave SMs without work while the kernel is bound by
-      // how many operand bytes all SMs together keep in flight; narrower tiles spread the B panels over every SM
-      if ((int64_t)((a->M + BM - 1) / BM) * W * ((nl + 255) / 256) < h->sm_count) bn = 128;
+      // skinny problems (one tile row) with stream-K switched off: 256-wide tiles would leave SMs without work while
+      // the kernel is bound by how many operand bytes all SMs together keep in flight; narrower tiles spread the
+      // B panels over every SM.  (With stream-K every SM gets the same share of k-steps whatever the tile width.)
+      if (a->stream_k <= 0 && (int64_t)((a->M + BM - 1) / BM) * W * ((nl + 255) / 256) < h->sm_count) bn = 128;
     }
     if (nl <= 128) bn = 128;
     // CTA pairs (256 x 256 tiles) need at least two tile rows.  A shard that is not a whole number of 256-column
@@ -1116,7 +1249,34 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
       p.comm_ctas = 0;
       p.gemm_ctas = std::min(grid, p.total_ctiles);
     }
+    // stream-K (single-CTA kernel): when the tile count leaves the last wave badly filled, cut the k-steps of all
+    // tiles into equal ranges instead, one per producer CTA.
+    streamk = false;
+    if (!pair && a->stream_k >= 0 && p.kblocks > 0) {
+      const int producers = wg ? std::max(1, std::min(grid, h->sm_count) - p.comm_ctas) : grid;
+      const int64_t waves = (p.total_ctiles + producers - 1) / producers;
+      const bool badly_filled = (int64_t)p.total_ctiles * 10 < waves * producers * 9;      // < 90 % of the slots used
+      const bool enough_k = (int64_t)p.total_ctiles * p.kblocks >= (int64_t)producers * 4 && p.kblocks >= 8;
+      (void)badly_filled;   // measured: on the skinny shapes this was meant for, operand streaming -- not the wave fill -- is the
+                            // limit and the parts' round trip through the workspace costs more than it saves: on request only
+      if (enough_k && a->stream_k > 0) {
+        streamk = true;
+        p.gemm_ctas = producers;
+      }
+    }
+    p.streamk = streamk ? 1 : 0;
     grid = p.gemm_ctas + p.comm_ctas;
+    // Which tiles the producers scatter themselves.  In workgroup_specialized mode the tiles of the last wave
+    // (raster ids >= total - producer units; every unit's final tile is one of them) have no GEMM work left to
+    // overlap with, so handing them to a few communication CTAs would leave their store ports as the only ones
+    // busy at the end of the kernel: the producers write those tiles to all W slots and publish them, as in
+    // fused_sequential mode.  wg_tail: -1 = never (Listing 5 for every tile), n > 0 = the last n compute tiles.
+    if (a->mode == IRIS_MODE_FUSED_SEQUENTIAL) p.seq_from = 0;
+    else if (!wg || a->wg_tail < 0) p.seq_from = INT_MAX;
+    else {
+      const int units = pair ? p.gemm_ctas / 2 : p.gemm_ctas;
+      p.seq_from = std::max(0, p.total_ctiles - (a->wg_tail > 0 ? a->wg_tail : units));
+    }
 
     // Tensor maps.  K == 0 has no operand to describe; the kernel then never issues a load.
     if (a->K > 0) {
@@ -1147,7 +1307,7 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     const int brc = build();
     if (brc != IRIS_OK) return brc;
     std::lock_guard<std::mutex> lock(g_plan_mutex);
-    g_plan.p = p; g_plan.bn = bn; g_plan.grid = grid; g_plan.pair = pair;
+    g_plan.p = p; g_plan.bn = bn; g_plan.grid = grid; g_plan.pair = pair; g_plan.streamk = streamk;
     g_plan_key = key;
     g_plan_valid = true;
   }
@@ -1156,6 +1316,20 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int rc;
   const bool bf = a->dtype == IRIS_BF16;
+  if (streamk) {
+    // two fp32 tile slots per producer CTA, then one arrival counter per compute tile (zeroed for every launch)
+    const size_t slots_bytes = (size_t)2 * p.gemm_ctas * BM * bn * sizeof(float);
+    const size_t need = slots_bytes + align_up((uint64_t)p.total_ctiles * 4, 256);
+    if (need > h->ws_bytes) {
+      if (h->ws) { IRIS_CUDA_TRY(cudaStreamSynchronize(st)); cudaFree(h->ws); }
+      h->ws = nullptr; h->ws_bytes = 0;
+      if (cudaMalloc(&h->ws, need) != cudaSuccess) { cudaGetLastError(); return fail(IRIS_ERR_NOMEM, "gemm_all_scatter: stream-K workspace (%zu bytes)", need); }
+      h->ws_bytes = need;
+    }
+    p.ws = static_cast<float*>(h->ws);
+    p.arrive = reinterpret_cast<int32_t*>(static_cast<char*>(h->ws) + slots_bytes);
+    IRIS_CUDA_TRY(cudaMemsetAsync(p.arrive, 0, (size_t)p.total_ctiles * 4, st));
+  }
   if (pair) {
     p.dynamic = a->static_schedule ? 0 : 1;
     p.tile_counter = h->status + 16;   // a spare word of the status block; every launch starts it at zero
@@ -1333,6 +1507,7 @@ int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, co
   p.epoch = epoch;
   p.comm_ctas = std::min(auto_comm_ctas(M, N, K, world, sms), std::min(sms - 1, p.total_ptiles));
   p.gemm_ctas = std::min(sms - p.comm_ctas, p.total_ctiles);
+  p.seq_from = std::max(0, p.total_ctiles - p.gemm_ctas);   // the last wave is scattered by its producers
   if (K > 0) {
     const cuuint64_t dimsA[2] = {(cuuint64_t)K, (cuuint64_t)M};
     const cuuint64_t strA[1] = {(cuuint64_t)K * 2};

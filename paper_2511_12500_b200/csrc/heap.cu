@@ -98,6 +98,7 @@ int iris_heap_destroy(iris_heap* h) {
   cudaFree(h->status);
   if (h->stage_a) cudaFree(h->stage_a);
   if (h->stage_b) cudaFree(h->stage_b);
+  if (h->ws) cudaFree(h->ws);
   h->magic = 0;
   delete h;
   cudaGetLastError();

@@ -54,6 +54,9 @@ struct iris_heap {
   void* stage_a;
   void* stage_b;
   size_t stage_a_bytes, stage_b_bytes;
+  // stream-K workspace (partial sums + arrival counters), allocated on first use
+  void* ws;
+  size_t ws_bytes;
   iris::HeapTable table() const {
     iris::HeapTable t{};
     for (int r = 0; r < world; ++r) t.base[r] = (uint64_t)(base + (size_t)r * bytes_per_rank);

@@ -101,7 +101,7 @@ def test_communication_ctas_give_up_when_a_lock_is_never_released():
         iris.iris_flags_fill(g.h, lock_off, nt, 2)
         iris.iris_flags_fill(g.h, flag_off, nt, 0)
         iris.iris_gemm_all_scatter_ex(g.h, dev16(A), [dev16(b) for b in Bs], M, N, K, W, iris.IRIS_MODE_WORKGROUP_SPECIALIZED,
-                                      iris.IRIS_BF16, c_off, flag_off, lock_off, 1, spin_timeout_ns=3_000_000)
+                                      iris.IRIS_BF16, c_off, flag_off, lock_off, 1, spin_timeout_ns=3_000_000, wg_tail=-1)
         with pytest.raises(iris.IrisError) as e:
             iris.iris_status_check(g.h)
         assert e.value.code == iris.IRIS_ERR_TIMEOUT and e.value.detail[1] == 1
@@ -125,9 +125,10 @@ FUSED_SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("mode,wg_tail", [(MODES[0], 0), (MODES[1], 0), (MODES[2], -1), (MODES[2], 0), (MODES[2], 2)],
+                         ids=["bulk_synchronous", "fused_sequential", "workgroup_specialized_no_tail", "workgroup_specialized", "workgroup_specialized_tail2"])
 @pytest.mark.parametrize("W,M,nl,K,kw", FUSED_SHAPES)
-def test_consumer_as_part_of_the_gemm_call(mode, W, M, nl, K, kw):
+def test_consumer_as_part_of_the_gemm_call(mode, wg_tail, W, M, nl, K, kw):
     """gemm_all_scatter with consumer_bias set: C, flags, locks and OUT must equal the oracle's heap image byte for
     byte (integer-valued inputs make the GEMM exact).  The heap starts as NaN patterns, so a consumer warp that read
     a tile before its flag was published would leave NaNs in OUT."""
@@ -146,7 +147,7 @@ def test_consumer_as_part_of_the_gemm_call(mode, W, M, nl, K, kw):
         dA, dB, dbias = dev16(A), [dev16(b) for b in Bs], dev16(bias)
         for epoch in (1, 2, 3):
             iris.iris_gemm_all_scatter_ex(g.h, dA, dB, M, N, K, W, mode, iris.IRIS_BF16, c_off, flag_off, lock_off, epoch,
-                                          consumer_bias=dbias, consumer_out_off=out_off, **kw)
+                                          consumer_bias=dbias, consumer_out_off=out_off, wg_tail=wg_tail, **kw)
         iris.iris_status_check(g.h)
         img.gemm_all_scatter(A, Bs, dtype, c_off, flag_off, 3, lock_off if mode == iris.IRIS_MODE_WORKGROUP_SPECIALIZED else None)
         img.consume_bias(dtype, c_off, out_off, M, N, bias)

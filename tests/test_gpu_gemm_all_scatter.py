@@ -28,6 +28,10 @@ def run_gemm(g, A, Bs, dtype, mode, epoch=1, with_locks_zeroed=True, **kw):
     nt = oracle.num_tiles(M, N, W) if M and N else 0
     if with_locks_zeroed and nt:
         iris.iris_flags_fill(g.h, lock_off, nt, 0)
+    # These shapes are a wave or two: by default the producers would scatter most tiles themselves.  Unless a test
+    # asks otherwise, every tile takes the lock handshake and the communication CTAs (Listing 5 as printed).
+    if mode == iris.IRIS_MODE_WORKGROUP_SPECIALIZED:
+        kw.setdefault("wg_tail", -1)
     iris.iris_gemm_all_scatter_ex(g.h, dA, dB, M, N, K, W, mode, iris.DTYPES[dtype], c_off, flag_off, lock_off, epoch, **kw)
     iris.iris_status_check(g.h)
     return c_off, flag_off, lock_off, out_off, nt
@@ -284,3 +288,77 @@ def test_short_form_and_host_entry_point():
         iris.iris_gemm_all_scatter_host(A, Bs, C_host, None, bias, OUT_host, g.h, M, N, K, W, iris.IRIS_MODE_FUSED_SEQUENTIAL,
                                         iris.IRIS_BF16, 0)
         assert np.array_equal(C_host, c_ref) and np.array_equal(OUT_host, oracle.consume_bias_rows(c_ref, bias, "bf16"))
+
+
+STREAMK_SHAPES = [
+    # W, M, N_local, K, kwargs  (single-CTA kernel; K long enough to be cut into ranges)
+    (8, 128, 512, 2048, dict()),                         # one tile row, 16 tiles for 148 SMs: chosen automatically
+    (8, 128, 512, 2048, dict(stream_k=1, block_n=128)),
+    (2, 300, 640, 1024, dict(stream_k=1, cta_pair=-1)),  # ragged M and N_local, tiles split at arbitrary k
+    (4, 100, 136, 4096, dict(stream_k=1)),               # a single ragged tile row
+    (8, 128, 3584, 512, dict(stream_k=1, max_ctas=37, comm_ctas=5)),
+    (3, 640, 256, 1536, dict(stream_k=1, cta_pair=-1, max_ctas=13)),   # ranges longer than a tile: whole tiles + two parts
+]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("dtype", ["bf16", "fp16"])
+@pytest.mark.parametrize("W,M,nl,K,kw", STREAMK_SHAPES)
+def test_stream_k_exact_integer_full_heap_image(mode, dtype, W, M, nl, K, kw):
+    """Tiles computed in k-range parts and reduced through the workspace: with integer-valued inputs the sums are
+    exact in any order, so the whole heap image must still equal the oracle's byte for byte; run twice so that the
+    arrival counters and the workspace are seen to be reusable."""
+    N = W * nl
+    A = inputs.matrix(47, inputs.STREAM_A, M, K, "ternary:0.25", dtype)
+    Bs = [inputs.matrix(47, inputs.STREAM_B0 + r, nl, K, "smallint:1", dtype) for r in range(W)]
+    bpr = gemm_layout(M, N, W, True)[4]
+    with GpuHeap(W, bpr) as g:
+        img = None
+        for epoch in (1, 2):
+            run_gemm(g, A, Bs, dtype, mode, epoch=epoch, with_locks_zeroed=(epoch == 1), **kw)
+            host = g.to_host()
+            img, _ = expected_image(g, A, Bs, dtype, mode, epoch=epoch, c_full=None if img is None else c_slot(img.mem, g, 0, gemm_layout(M, N, W, True)[0], M, N).copy())
+            assert np.array_equal(host, img.mem), (epoch, first_diff(host, img.mem))
+
+
+def test_stream_k_real_valued_is_deterministic_and_within_tolerance():
+    W, M, nl, K, dtype = 8, 128, 1024, 4096, "bf16"
+    N = W * nl
+    A, Bs = inputs.gemm_inputs(inputs.SEED0 + 3, W, M, N, K, "normal002", dtype)
+    c_ref = oracle.gemm_block(A, Bs, dtype)
+    bpr = gemm_layout(M, N, W, True)[4]
+    with GpuHeap(W, bpr) as g:
+        outs = []
+        for rep in range(3):
+            g.mem.fill_(SENTINEL)
+            c_off = run_gemm(g, A, Bs, dtype, iris.IRIS_MODE_WORKGROUP_SPECIALIZED, stream_k=1)[0]
+            host = g.to_host()
+            c0 = c_slot(host, g, 0, c_off, M, N).copy()
+            check_tolerance(c0, c_ref, dtype)
+            for s in range(1, W):
+                assert np.array_equal(c_slot(host, g, s, c_off, M, N), c0)
+            outs.append(c0)
+        assert np.array_equal(outs[0], outs[1]) and np.array_equal(outs[0], outs[2])   # the parts are added in a fixed order
+
+
+@pytest.mark.parametrize("wg_tail", [0, 1, 3, 1000])
+@pytest.mark.parametrize("W,M,nl,K,kw", [
+    (2, 1000, 512, 200, dict()),                            # CTA pairs, 4 x 4 pair tiles
+    (2, 1000, 512, 200, dict(static_schedule=1, max_ctas=8)),
+    (8, 1280, 384, 64, dict(max_ctas=24, comm_ctas=4)),     # single-CTA kernel, several waves
+    (3, 520, 392, 328, dict(cta_pair=-1, max_ctas=9)),
+    (4, 640, 512, 1024, dict(cta_pair=-1, stream_k=1, max_ctas=21)),
+    (2, 600, 448, 136, dict(max_ctas=6)),                   # CTA pairs with a ragged shard: 2 producer pairs, 1 communication pair
+])
+def test_workgroup_specialized_tail_tiles_scattered_by_producers(wg_tail, W, M, nl, K, kw):
+    """The last wave's tiles (or the last n) are written to all slots by their producers, the rest go through the lock
+    handshake: the heap image -- C everywhere, flags, locks back at 0 -- is the oracle's either way."""
+    N, dtype, mode = W * nl, "bf16", iris.IRIS_MODE_WORKGROUP_SPECIALIZED
+    A = inputs.matrix(53, inputs.STREAM_A, M, K, "ternary:0.5", dtype)
+    Bs = [inputs.matrix(53, inputs.STREAM_B0 + r, nl, K, "smallint:2", dtype) for r in range(W)]
+    bpr = gemm_layout(M, N, W, True)[4]
+    with GpuHeap(W, bpr) as g:
+        run_gemm(g, A, Bs, dtype, mode, wg_tail=wg_tail, **kw)
+        host = g.to_host()
+        img, _ = expected_image(g, A, Bs, dtype, mode)
+        assert np.array_equal(host, img.mem), first_diff(host, img.mem)

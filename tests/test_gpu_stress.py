@@ -25,6 +25,9 @@ MODES = [iris.IRIS_MODE_BULK_SYNCHRONOUS, iris.IRIS_MODE_FUSED_SEQUENTIAL, iris.
     (8, 2048, 256, 64, dict(comm_ctas=2)),                   # communicators are the bottleneck
     (4, 1024, 512, 128, dict(static_schedule=1, comm_ctas=40)),
     (8, 1280, 384, 64, dict()),                              # single-CTA kernel (N_local % 256 != 0)
+    (8, 2048, 256, 64, dict(wg_tail=-1)),                    # one wave: every tile through the lock handshake
+    (8, 2048, 512, 64, dict(max_ctas=40)),                   # several waves, the last one scattered by its producers
+    (8, 1280, 384, 64, dict(wg_tail=-1, comm_ctas=3)),
 ])
 def test_repeated_launches_on_a_poisoned_heap(mode, W, M, nl, K, kw):
     N, dtype = W * nl, "bf16"
@@ -86,6 +89,10 @@ def test_random_shapes_exact_heap_image():
             kw["cta_pair"] = -1
         elif rng.random() < 0.4 and M > 128 and nl > 128:
             kw["cta_pair"] = 1      # pairs even where the shard is ragged
+        if rng.random() < 0.5:
+            kw["wg_tail"] = int(rng.choice([-1, 1, 2, 5]))
+        if kw.get("cta_pair") == -1 and rng.random() < 0.6:
+            kw["stream_k"] = 1
         dtype = "bf16" if case % 2 else "fp16"
         N = W * nl
         A = inputs.matrix(900 + case, inputs.STREAM_A, M, K, "ternary:0.5", dtype)
