@@ -60,6 +60,7 @@ struct alignas(64) GemmParams {
   CUtensorMap tmA;                    // A [M, K], box 64 x 128, 128B swizzle
   CUtensorMap tmB[IRIS_MAX_WORLD];    // B_r [N_local, K], box 64 x BN, 128B swizzle
   CUtensorMap tmC[IRIS_MAX_WORLD];    // C of slot s viewed as [W][M][N_local], box 128 x 128 x 1, no swizzle
+  CUtensorMap tmCs[IRIS_MAX_WORLD];   // the same view, box 64 x 128 x 1, 128B swizzle: the pair kernel's epilogue stores
   HeapTable tab;
   uint64_t c_off, flag_off, lock_off;
   uint64_t timeout_ns;
@@ -689,15 +690,21 @@ __device__ void consumer_warp(const GemmParams& p, CtrlBlock* ctrl, int cwarp, i
 //   tmem_full[a]   both CTAs; multicast commit after a tile's last MMA
 //   tmem_empty[a]  leader only; 8 arrivals = 4 epilogue warps x 2 CTAs (the peer's arrive remotely)
 // ------------------------------------------------------------------------------------------------
-constexpr int kPairStageBytes = 2 * BM * BK * 2;            // 32 KB: A slice + B half
-constexpr int kPairStages = kSmemPayload / kPairStageBytes;  // 6
 constexpr int kPairBN = 256;
+constexpr int kPairStageBytes = 2 * BM * BK * 2;            // 32 KB: A slice + B half
+constexpr int kPairStages = 5;
+constexpr int kStoreBoxBytes = BM * 64 * 2;                 // 16 KB: 128 rows x 64 columns, one TMA store box
+constexpr int kPairStoreBytes = (kPairBN / 64) * kStoreBoxBytes;   // 64 KB: this CTA's 128 x 256 half of the converted tile
+constexpr int kPairSmemPayload = kPairStages * kPairStageBytes + kPairStoreBytes;   // 224 KB
+constexpr int kPairSmemTotal = kPairSmemPayload + kSmemCtrl + 1024;
+static_assert(kPairSmemPayload >= kCommWarps * kTileBytes, "communication warps' tile buffers share the payload area");
+static_assert(kPairSmemTotal <= 232448, "shared memory per CTA");
 
 template <bool BF16, bool STATIC_LOCKS = false, bool CONSUMER = false>
 __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1) gemm_all_scatter_pair_kernel(const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* payload = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  CtrlBlock* ctrl = reinterpret_cast<CtrlBlock*>(payload + kSmemPayload);
+  CtrlBlock* ctrl = reinterpret_cast<CtrlBlock*>(payload + kPairSmemPayload);
   const int warp = (int)threadIdx.x / 32, lane = (int)threadIdx.x % 32;
   const int cta_rank = (int)ptx::cluster_ctarank();
   const bool leader = cta_rank == 0;
@@ -720,6 +727,8 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
     }
     if (is_comm)
       for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmC[r]);
+    else
+      for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmCs[r]);
   }
   if (warp == 1 && !is_comm) {
     ptx::tmem_alloc_pair(ptx::smem_u32(&ctrl->tmem_base), 2 * kPairBN);
@@ -844,48 +853,57 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
       const TileCoord tc = decode_ctile(tile, p);
       ptx::tc_fence_after();
       const int tm = tc.tm * 2 + cta_rank;  // publication tile row of this CTA's half
-      const int row = tm * BM + quad * 32 + lane;
+      const int row_in_half = quad * 32 + lane;
       const int col_in_shard = tc.jn * kPairBN;
-      const uint64_t row_off = p.c_off + ((uint64_t)row * p.N + (uint64_t)tc.rank * p.n_local) * 2;
-      const bool seq = tile >= p.seq_from;   // scatter from registers (Listing 4) or hand over to the communicators (Listing 5)
+      const bool seq = tile >= p.seq_from;   // scatter to every slot (Listing 4) or store locally and hand over (Listings 3, 5)
+      // Convert and stage this CTA's 128 x 256 half in shared memory as four 64-column boxes in the 128B-swizzle
+      // layout of the store maps: a lane owns a row, so its 16-byte pieces go to (piece ^ row % 8) and a warp's
+      // 512 bytes per instruction spread over all banks.  (The previous tile's stores have been waited for
+      // before the barrier at the top of this loop, so the boxes are free.)
+      const uint32_t stg = ptx::smem_u32(payload + kPairStages * kPairStageBytes);
 #pragma unroll 1
       for (int ch = 0; ch < kPairBN / 32; ++ch) {
         uint32_t v[32];
         ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kPairBN + ch * 32), v);
         ptx::tmem_wait_ld();
-        uint4 q[4];
+        const uint32_t row_base = stg + (uint32_t)((ch >> 1) * kStoreBoxBytes + row_in_half * 128);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
+          uint4 q;
           if (p.kblocks == 0) {
-            q[i] = make_uint4(0, 0, 0, 0);
+            q = make_uint4(0, 0, 0, 0);   // K == 0: the sum is empty
           } else {
-            q[i].x = pack2<BF16>(v[8 * i + 0], v[8 * i + 1]);
-            q[i].y = pack2<BF16>(v[8 * i + 2], v[8 * i + 3]);
-            q[i].z = pack2<BF16>(v[8 * i + 4], v[8 * i + 5]);
-            q[i].w = pack2<BF16>(v[8 * i + 6], v[8 * i + 7]);
+            q.x = pack2<BF16>(v[8 * i + 0], v[8 * i + 1]);
+            q.y = pack2<BF16>(v[8 * i + 2], v[8 * i + 3]);
+            q.z = pack2<BF16>(v[8 * i + 4], v[8 * i + 5]);
+            q.w = pack2<BF16>(v[8 * i + 6], v[8 * i + 7]);
           }
-        }
-        if (row < p.M) {
-          const int c0 = col_in_shard + ch * 32;
-          if (seq) {
-            for (int s = 0; s < W; ++s) {
-              const uint64_t dst = p.tab.base[s] + row_off + (uint64_t)c0 * 2;
-#pragma unroll
-              for (int i = 0; i < 4; ++i)
-                if (c0 + 8 * i < p.n_local) st_global_v4(reinterpret_cast<void*>(dst + 16 * i), q[i]);
-            }
-          } else {
-            const uint64_t dst = p.tab.base[tc.rank] + row_off + (uint64_t)c0 * 2;
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-              if (c0 + 8 * i < p.n_local) st_global_v4(reinterpret_cast<void*>(dst + 16 * i), q[i]);
-          }
+          const int piece = (ch & 1) * 4 + i;
+          ptx::st_shared_v4(row_base + (uint32_t)(((piece ^ (row_in_half & 7)) << 4)), q);
         }
       }
+      // accumulator drained: hand it back to the MMA warp before the stores go out
       ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&ctrl->tmem_empty[acc]), 0));
       if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+      fence_proxy_async();   // this thread's shared-memory writes -> the TMA unit's reads
+      asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
+      if (et == 0) {
+        // One thread stores the boxes with TMA: whole 128-byte lines, clipped by the maps at row M and column
+        // N_local, to the owner's slot or (Listing 4: for remote_rank in range(world_size): iris.store(...)) to all.
+        if (tm < p.ptiles_m) {
+          for (int s = 0; s < W; ++s) {
+            if (!seq && s != tc.rank) continue;
+#pragma unroll
+            for (int b = 0; b < kPairBN / 64; ++b)
+              if (col_in_shard + 64 * b < p.n_local)
+                ptx::tma_store_3d(&p.tmCs[s], col_in_shard + 64 * b, tm * BM, tc.rank, stg + (uint32_t)(b * kStoreBoxBytes));
+          }
+          ptx::bulk_commit_group();
+        }
+        ptx::bulk_wait_group<0>();   // stores performed: the boxes are free and the tile may be published
+      }
       if (p.mode != IRIS_MODE_BULK_SYNCHRONOUS) {
         asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
         constexpr int subs = kPairBN / IRIS_TILE;
@@ -1023,13 +1041,13 @@ static int launch_gemm_pair(const GemmParams& p, int grid, cudaStream_t st, int*
   auto kern = gemm_all_scatter_pair_kernel<BF16, STATIC_LOCKS, CONSUMER>;
   static bool configured = false;
   if (!configured) {
-    IRIS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal));
+    IRIS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemTotal));
     configured = true;
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(max_pairs_out ? 2 : grid));
   cfg.blockDim = dim3(CONSUMER ? kGemmThreadsFused : kGemmThreads);
-  cfg.dynamicSmemBytes = kSmemTotal;
+  cfg.dynamicSmemBytes = kPairSmemTotal;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -1289,6 +1307,15 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
         const cuuint64_t dimsB[2] = {(cuuint64_t)a->K, (cuuint64_t)nl};
         const cuuint32_t boxB[2] = {BK, (cuuint32_t)(pair ? kPairBN / 2 : bn)};   // a pair's CTA loads its half of the tile
         rc = make_map(&p.tmB[r], a->dtype, 2, const_cast<void*>(a->B_shards[r]), dimsB, strA, boxB, CU_TENSOR_MAP_SWIZZLE_128B, "B");
+        if (rc != IRIS_OK) return rc;
+      }
+    }
+    if (pair) {
+      for (int s = 0; s < W; ++s) {
+        const cuuint64_t dimsC[3] = {(cuuint64_t)nl, (cuuint64_t)a->M, (cuuint64_t)W};
+        const cuuint64_t strC[2] = {(cuuint64_t)a->N * 2, (cuuint64_t)nl * 2};
+        const cuuint32_t boxC[3] = {64, BM, 1};
+        int rc = make_map(&p.tmCs[s], a->dtype, 3, h->base + (size_t)s * bpr + a->c_off, dimsC, strC, boxC, CU_TENSOR_MAP_SWIZZLE_128B, "C (epilogue stores)");
         if (rc != IRIS_OK) return rc;
       }
     }
