@@ -2,20 +2,23 @@
 //
 // Two persistent, warp-specialised tcgen05 kernels share this file:
 //   gemm_all_scatter_pair_kernel  a cluster of two CTAs per 256 x 256 tile (cta_group::2), tile ids claimed in
-//                                 raster order; the default whenever N/world is a multiple of 256 and M > 128
-//   gemm_all_scatter_kernel       one CTA per 128 x 256 or 128 x 128 tile, static tile stride; handles every
-//                                 ragged shape (TMA zero fill on loads, masks on stores)
+//                                 raster order; the default whenever M > 128 and N/world > 128 (ragged edges are
+//                                 zero-filled by the loads and clipped by the stores)
+//   gemm_all_scatter_kernel       one CTA per 128 x 256 or 128 x 128 tile, static tile stride or stream-K; the
+//                                 skinny and the tiny shapes (TMA zero fill on loads, masks on stores)
 // Warp roles in a producer CTA:
 //   warp 0      TMA producer  (cp.async.bulk.tensor -> 128B-swizzled shared-memory stages, mbarrier ring)
 //   warp 1      MMA issuer    (one thread; tcgen05.mma into a double-buffered TMEM accumulator)
-//   warps 2..5  epilogue      (tcgen05.ld -> fp32 -> fp16/bf16 -> 16-byte global stores -> flags)
+//   warps 2..5  epilogue      (tcgen05.ld -> fp32 -> fp16/bf16 -> pair kernel: swizzled shared-memory boxes, TMA
+//                              stores by one thread; single-CTA kernel: 16-byte global stores -> flags or lock)
 //   warps 6..9  consumer      (pair kernel, optional: acquire flags, OUT = C + bias)
 // What happens to a finished tile depends on the schedule:
 //   bulk_synchronous       store to the owner rank's slot; a second kernel scatters and publishes
 //   fused_sequential       store to all W slots from registers, then publish W ready flags
 //   workgroup_specialized  store to the owner slot, cas(lock, 0->1, release); reserved communication
 //                          CTAs poll the locks (acquire), copy the tile to the other W-1 slots with
-//                          TMA and publish the flags
+//                          TMA and publish the flags.  Tiles of the last wave (raster id >= seq_from) are
+//                          scattered and published by their producers instead: nothing is left to overlap with
 // Because the TMEM accumulator is double buffered, the epilogue of tile i (including the W-way
 // scatter) overlaps the main loop of tile i+1 inside one CTA.
 #include <cuda.h>
@@ -682,9 +685,11 @@ __device__ void consumer_warp(const GemmParams& p, CtrlBlock* ctrl, int cwarp, i
 // CTA r of the pair owns rows [128 r, 128 r + 128) of the tile: it TMA-loads its own 128 x 64 slice of A
 // and its own half (128 of the 256 columns) of the B tile -- no multicast, every CTA fetches only what
 // it keeps -- and the leader's MMA thread issues one 256 x 256 x 16 instruction for both: each SM's
-// tensor core reads its A slice locally and both B halves.  Per CTA and k-step 32 KB are staged instead
-// of 48 KB for the same flops per SM, which is what the single-CTA kernel's shared-memory port cannot
-// afford.  Accumulators: 2 x 256 columns of TMEM in each CTA (rows of its own half).
+// tensor core reads its A slice locally and both B halves.  Per CTA and k-step 32 KB are pulled in instead
+// of 48 KB for the same flops per SM: 64 B/clk, which the SM's port to the L2 sustains, instead of 96, which
+// it does not (the single-CTA kernel's tensor pipe is 67 % busy, this one's 92 %).
+// Accumulators: 2 x 256 columns of TMEM in each CTA (rows of its own half).  Shared memory: 5 stages of
+// 32 KB + four 16 KB store boxes (the CTA's converted 128 x 256 half, 128B-swizzled for the TMA stores).
 //   full[s]        leader only; the leader's producer expects 64 KB, all four loads (two per CTA) complete on it
 //   empty[s]       both CTAs; the leader's tcgen05.commit multicasts the arrival to the pair
 //   tmem_full[a]   both CTAs; multicast commit after a tile's last MMA
