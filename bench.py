@@ -347,12 +347,20 @@ def run_ours(args):
                 torch.cuda.synchronize()
                 if it > 0:
                     series[name].append(e0.elapsed_time(e1))
+        kept = {}
+        for name, m in (variants if args.mode_iters > 0 else ()):
+            if m == iris.IRIS_MODE_WORKGROUP_SPECIALIZED and not name.endswith("comm_ctas"):
+                epoch += 1
+                gemm(epoch, m)
+                kept[name] = iris.iris_gemm_takeover_stats(h)[0]
         for name, ts in series.items():
             if not ts:
                 continue
             ms = float(np.median(ts))
             modes[name] = {"ms": ms, "ms_min": float(min(ts)), "tflops": flops / ms / 1e9, "store_gbs": store_bytes / ms / 1e6,
                            "frac_of_combined_roofline": max(t_tensor, t_store) / ms}
+            if name in kept:
+                modes[name]["half_tiles_kept_by_producers_before_the_last_wave"] = kept[name]
         iris.iris_status_check(h)
         result["modes"] = modes
 

@@ -232,13 +232,16 @@ typedef struct iris_gemm_args {
                                   allocates on first use; 0 and -1 = whole tiles only (measured
                                   faster on every benchmark shape, hence the default)            */
   int wg_tail;                 /* workgroup-specialised: which compute tiles the producers scatter
-                                  themselves (to all W slots from registers, as fused_sequential
-                                  does) instead of handing them to the communication CTAs.
+                                  themselves (to all W slots, as fused_sequential does) instead of
+                                  handing them to the communication CTAs.
                                   0 = the last wave (the last P tiles of the raster order, P =
                                   producer CTAs or pairs: no GEMM work is left to overlap their
-                                  scatter with, and all store ports beat a few); n > 0 = the last
-                                  n tiles; -1 = none (Listing 5 for every tile).  The final heap
-                                  image is the same in every case                                */
+                                  scatter with) and, in the CTA-pair kernel, every tile that the
+                                  communication CTAs could not finish before the kernel ends,
+                                  judged when the tile completes from their backlog and the waves
+                                  still to come (so too few communication CTAs cost little);
+                                  n > 0 = exactly the last n tiles; -1 = none (Listing 5 for every
+                                  tile).  The final heap image is the same in every case        */
   const void* consumer_bias;   /* not NULL: also run the flag-gated consumer OUT = C + bias (see
                                   iris_consume_bias) as part of this call: inside the same launch,
                                   as extra warps that acquire each tile's flag while the GEMM is
@@ -284,6 +287,12 @@ int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_h
                                int M, int N, int K, int world, int mode, int dtype, int out_slot);
 /* Offset of OUT in the short form's layout: right after the lock array (256-byte aligned). */
 uint64_t iris_gemm_out_offset(int M, int N, int world);
+
+/* How the last workgroup-specialised launch of the CTA-pair kernel on this heap split the scatter:
+ * out[0] = 128-row half tiles that their producers kept under the takeover rule (wg_tail = 0; the last
+ * wave, which is never handed over, is not counted), out[1] = publication tiles still queued for the
+ * communication CTAs (0 after a completed launch).  Synchronises the device; `out` is host memory. */
+int iris_gemm_takeover_stats(const iris_heap* heap, int32_t out[2]);
 
 /* ------------------------------------------------------------------------------------------ */
 /* An entry point that allocates nothing                                                       */

@@ -31,7 +31,7 @@ EXPORTS = [
     "iris_status_check", "iris_put_tile", "iris_get_tile", "iris_atomic_add", "iris_atomic_cas",
     "iris_atomic_add_contended", "iris_atomic_cas_contended", "iris_flags_fill", "iris_all_store_bench",
     "iris_gemm_all_scatter_ex", "gemm_all_scatter", "iris_gemm_heap_bytes", "iris_heap_epoch", "iris_num_tiles",
-    "iris_consume_bias", "iris_gemm_all_scatter_host", "iris_gemm_out_offset",
+    "iris_consume_bias", "iris_gemm_all_scatter_host", "iris_gemm_out_offset", "iris_gemm_takeover_stats",
     "iris_gemm_all_scatter_noalloc", "iris_copy_tile", "iris_load_tile", "iris_store_tile", "iris_atomic_rmw",
 ]
 
@@ -103,6 +103,7 @@ def lib() -> C.CDLL:
     L.iris_num_tiles.argtypes = [ci, ci, ci]
     L.iris_consume_bias.argtypes = [vp, u64, u64, u64, vp, ci, ci, ci, ci, i32, ci, u64, vp]
     L.iris_gemm_all_scatter_host.argtypes = [vp, C.POINTER(vp), vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci]
+    L.iris_gemm_takeover_stats.argtypes = [vp, C.POINTER(C.c_int32)]
     L.iris_gemm_out_offset.restype = u64
     L.iris_gemm_out_offset.argtypes = [ci, ci, ci]
     L.iris_gemm_all_scatter_noalloc.argtypes = [vp, C.POINTER(vp), C.POINTER(u64), sz, ci, ci, ci, ci, ci, u64, u64, i32, vp]
@@ -291,6 +292,13 @@ def gemm_all_scatter(A, B_shards, heap, M, N, K, world, mode):
 
 def iris_consume_bias(heap, c_off, out_off, flag_off, bias, M, N, world, dtype, epoch, ctas=0, timeout_ns=0, stream=None):
     _ck(lib().iris_consume_bias(heap, c_off, out_off, flag_off, _ptr(bias), M, N, world, dtype, epoch, ctas, timeout_ns, _stream(stream)))
+
+
+def iris_gemm_takeover_stats(heap):
+    """(half tiles kept by their producers, publication tiles still queued) of the last workgroup-specialised pair launch."""
+    out = (C.c_int32 * 2)()
+    _ck(lib().iris_gemm_takeover_stats(heap, out))
+    return int(out[0]), int(out[1])
 
 
 def iris_gemm_out_offset(M: int, N: int, world: int) -> int:

@@ -86,6 +86,11 @@ struct alignas(64) GemmParams {
   int32_t* arrive;      // stream-K: per compute tile, how many parts have been parked
   int seq_from;         // compute tiles with raster id >= seq_from are scattered by their producer (Listing 4's loop); 0 in
                         // fused_sequential mode, the first tile of the last wave in workgroup_specialized mode
+  int takeover;         // pair kernel, workgroup_specialized: 1 = a producer also keeps (scatters itself) a tile below seq_from
+                        // when the communication CTAs could not drain their backlog plus this tile before the kernel ends
+  int32_t* backlog;     // publication tiles handed over and not yet published ([0]), tiles kept by that rule ([1])
+  uint32_t t_pt_ns;     // estimate: time a communication warp needs for one publication tile, its CTA's port shared by all warps
+  uint32_t t_tile_ns;   // estimate: main-loop time of one compute tile
   int raster_group;
   int mode;
   int32_t epoch;
@@ -103,6 +108,7 @@ struct CtrlBlock {  // lives in shared memory after the payload area
   uint32_t tmem_base;
   volatile int abort;
   volatile int last_part;   // stream-K: this CTA parked the last part of the tile and reduces it
+  volatile int keep_tile;   // pair kernel: this CTA scatters the current tile itself
 };
 
 struct TileCoord { int tm, rank, jn; };
@@ -237,7 +243,11 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
   assign();
   while (ok && __any_sync(kFull, widx >= 0)) {
     bool ready = false;
-    if (widx >= 0) ready = t < 0 || ld_acquire_gpu(lock_addr<STATIC_LOCKS>(p, rank, t)) == 1;
+    int state = 0;   // 1: the producer handed the tile over; 2: the producer scattered and published it itself
+    if (widx >= 0) {
+      if (t >= 0) state = ld_acquire_gpu(lock_addr<STATIC_LOCKS>(p, rank, t));
+      ready = t < 0 || state == 1 || state == 2;
+    }
     const uint32_t mask = __ballot_sync(kFull, ready);
 #ifdef IRIS_COMM_TRACE
     unsigned long long* tr = &g_comm_trace[(size_t)cw * 8];
@@ -260,7 +270,7 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
     }
     // Listing 5: tl.atomic_cas(locks + tile_id, 1, 0, sem="acquire", scope="gpu"); all ready lanes at once.
     IRIS_TR(tc0);
-    if (ready && t >= 0) (void)cas_acquire_gpu(lock_addr<STATIC_LOCKS>(p, rank, t), 1, 0);
+    if (ready && t >= 0) (void)cas_acquire_gpu(lock_addr<STATIC_LOCKS>(p, rank, t), state, 0);
     __syncwarp();
 #ifdef IRIS_COMM_TRACE
     if (lane == 0) tr[6] += globaltimer_ns() - tc0;
@@ -271,7 +281,8 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
       todo &= todo - 1;
       const int rt = __shfl_sync(kFull, t, src);
       const int rrank = __shfl_sync(kFull, rank, src);
-      if (rt < 0) continue;
+      const int rstate = __shfl_sync(kFull, state, src);
+      if (rt < 0 || rstate == 2) continue;   // no such sub-tile, or nothing left to do but the lock reset above
       const int tm = rt / pt_n, pj = (rt % pt_n) % p.ptiles_per_rank;
       bool fail = false;
       IRIS_TR(t0);
@@ -298,6 +309,7 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
       if (__any_sync(kFull, fail)) { ok = false; break; }
       IRIS_TR(t4);
       if (lane < W) st_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[lane] + p.flag_off) + rt, p.epoch);
+      if (p.takeover && lane == 0) atomicAdd(p.backlog, -1);
       __syncwarp();
 #ifdef IRIS_COMM_TRACE
       if (lane == 0) { tr[4] += globaltimer_ns() - t4; last_poll = globaltimer_ns(); }
@@ -860,7 +872,9 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
       const int tm = tc.tm * 2 + cta_rank;  // publication tile row of this CTA's half
       const int row_in_half = quad * 32 + lane;
       const int col_in_shard = tc.jn * kPairBN;
-      const bool seq = tile >= p.seq_from;   // scatter to every slot (Listing 4) or store locally and hand over (Listings 3, 5)
+      // Scatter to every slot (Listing 4) or store locally and hand over (Listings 3, 5).  Below seq_from the
+      // workgroup-specialised schedule hands over unless the takeover rule (decided by thread 0 further down) keeps the tile.
+      bool seq = tile >= p.seq_from;
       // Convert and stage this CTA's 128 x 256 half in shared memory as four 64-column boxes in the 128B-swizzle
       // layout of the store maps: a lane owns a row, so its 16-byte pieces go to (piece ^ row % 8) and a warp's
       // 512 bytes per instruction spread over all banks.  (The previous tile's stores have been waited for
@@ -895,6 +909,18 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
       fence_proxy_async();   // this thread's shared-memory writes -> the TMA unit's reads
       asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
       if (et == 0) {
+        if (p.takeover && !seq && tm < p.ptiles_m) {
+          // Hand over only what the communication warps can still finish: their backlog plus this CTA's publication
+          // tiles, at t_pt_ns each spread over all of them, against the main-loop time of the waves still to come.
+          // Near the end of the kernel (and whenever they fall behind) the producers' own store ports take the rest.
+          const int mine = min(kPairBN / IRIS_TILE, p.ptiles_per_rank - tc.jn * (kPairBN / IRIS_TILE));
+          const int waves_left = (p.total_ctiles - 1 - tile) / (p.gemm_ctas >> 1);
+          const int queued = ld_relaxed_gpu(p.backlog);
+          seq = (uint64_t)(queued + mine) * p.t_pt_ns > (uint64_t)waves_left * p.t_tile_ns * (uint64_t)(p.comm_ctas * kCommWarps);
+          if (seq) atomicAdd(p.backlog + 1, 1);
+          else atomicAdd(p.backlog, mine);
+        }
+        ctrl->keep_tile = seq ? 1 : 0;
         // One thread stores the boxes with TMA: whole 128-byte lines, clipped by the maps at row M and column
         // N_local, to the owner's slot or (Listing 4: for remote_rank in range(world_size): iris.store(...)) to all.
         if (tm < p.ptiles_m) {
@@ -911,6 +937,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
       }
       if (p.mode != IRIS_MODE_BULK_SYNCHRONOUS) {
         asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
+        seq = ctrl->keep_tile != 0;   // (the next write to keep_tile comes after the barrier at the top of the loop)
         constexpr int subs = kPairBN / IRIS_TILE;
         const int pt_n = W * p.ptiles_per_rank;
         if (tm < p.ptiles_m) {
@@ -921,6 +948,13 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
               if (pj < p.ptiles_per_rank) {   // a ragged shard's last tile may have only one publication tile
                 const int t = tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
                 st_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[s] + p.flag_off) + t, p.epoch);
+              }
+            } else if (p.takeover && tile < p.seq_from && et >= 64 && et < 64 + subs) {
+              // a tile the communication warps are watching: tell its warp that only the lock is left to reset
+              const int pj = tc.jn * subs + (et - 64);
+              if (pj < p.ptiles_per_rank) {
+                const int t = tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
+                (void)cas_release_gpu(lock_addr<STATIC_LOCKS>(p, tc.rank, t), 0, 2);
               }
             }
           } else if (et < subs) {
@@ -1083,13 +1117,36 @@ static int auto_comm_ctas(int M, int N, int K, int W, int sms) {
   return std::max(4, std::min(c, sms / 3));
 }
 
+// CTA-pair kernel with the takeover rule: producers keep what the communication CTAs cannot finish, so the count only
+// has to balance two things -- every communication pair is a producer pair less (and can add a wave), every byte the
+// communicators do not take is stored through the producers' own ports instead.  Model per candidate count c:
+// waves = ceil(tiles / pairs), t = waves * t_tile + (remote bytes - what c SMs move in that time) / (producer SMs' ports);
+// the smallest t among the counts that leave at least three quarters of the scatter to the communication CTAs
+// (the schedule stays what its name says; measured differences between the candidates are a few per cent).  Constants: 45 GB/s sustained per communication SM (57 at best), 57 GB/s per
+// producer port, 270 ns per k-step of a pair tile.
+static int auto_comm_ctas_pair(int total_ctiles, int kblocks, double remote_bytes, int grid) {
+  int best_c = 2;
+  double best_t = 1e30;
+  for (int c = 2; c <= grid - 2 && c <= 64; c += 2) {
+    const int pairs = std::min((grid - c) / 2, std::max(1, total_ctiles));
+    const double waves = std::ceil((double)total_ctiles / pairs);
+    const double t_gemm = waves * (kblocks * 0.27e-6 + 2e-6);
+    const double cap = c * 45e9 * t_gemm;
+    if (cap < remote_bytes * 0.75 && c < std::min(grid - 2, 64) - 1) continue;
+    const double kept = std::max(0.0, remote_bytes - cap);
+    const double t = t_gemm + kept / (2.0 * pairs * 57e9);
+    if (t < best_t * 0.999) { best_t = t; best_c = c; }
+  }
+  return best_c;
+}
+
 // ---- launch-plan cache -------------------------------------------------------------------------------
 struct PlanKey {
   const void* heap; const void* base; const void* status; uint64_t bytes_per_rank;
   const void* A; const void* B[IRIS_MAX_WORLD];
   int M, N, K, world, mode, dtype;
   uint64_t c_off, flag_off, lock_off;
-  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail;
+  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail, fused_consumer;
   uint64_t spin_timeout_ns;
 };
 struct Plan { GemmParams p; int bn, grid; bool pair, streamk; };
@@ -1107,6 +1164,7 @@ static void make_key(PlanKey* k, const iris_gemm_args* a, const iris_heap* h) {
   k->c_off = a->c_off; k->flag_off = a->flag_off; k->lock_off = a->lock_off;
   k->comm_ctas = a->comm_ctas; k->max_ctas = a->max_ctas; k->raster_group = a->raster_group; k->block_n = a->block_n;
   k->cta_pair = a->cta_pair; k->static_schedule = a->static_schedule; k->stream_k = a->stream_k; k->wg_tail = a->wg_tail;
+  k->fused_consumer = a->consumer_bias != nullptr;   // the split between producers and communicators depends on it
   k->spin_timeout_ns = a->spin_timeout_ns;
 }
 
@@ -1254,7 +1312,11 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
       grid = std::min(grid & ~1, 2 * max_pairs);
       if (grid < (wg ? 4 : 2)) return fail(IRIS_ERR_ARG, "gemm_all_scatter: max_ctas too small for CTA pairs");
       if (wg) {
-        int comm = a->comm_ctas ? a->comm_ctas : auto_comm_ctas(a->M, a->N, a->K, W, grid);
+        int comm = a->comm_ctas;
+        // (with consumer warps in the producer CTAs their ports are busy with OUT = C + bias: the communication CTAs
+        // then get the whole scatter, as they do without the takeover rule)
+        if (!comm) comm = a->wg_tail == 0 && !fused_consumer ? auto_comm_ctas_pair(p.total_ctiles, p.kblocks, (double)(W - 1) * a->M * a->N * 2.0, grid)
+                                                              : auto_comm_ctas(a->M, a->N, a->K, W, grid);
         comm = std::max(2, std::min((comm + 1) & ~1, grid - 2));   // whole pairs on both sides
         p.comm_ctas = comm;
         p.gemm_ctas = 2 * std::min((grid - comm) / 2, p.total_ctiles);
@@ -1294,11 +1356,20 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     // overlap with, so handing them to a few communication CTAs would leave their store ports as the only ones
     // busy at the end of the kernel: the producers write those tiles to all W slots and publish them, as in
     // fused_sequential mode.  wg_tail: -1 = never (Listing 5 for every tile), n > 0 = the last n compute tiles.
+    p.takeover = 0;
     if (a->mode == IRIS_MODE_FUSED_SEQUENTIAL) p.seq_from = 0;
     else if (!wg || a->wg_tail < 0) p.seq_from = INT_MAX;
     else {
       const int units = pair ? p.gemm_ctas / 2 : p.gemm_ctas;
       p.seq_from = std::max(0, p.total_ctiles - (a->wg_tail > 0 ? a->wg_tail : units));
+      // wg_tail = 0 on the pair kernel: producers also keep tiles the communication CTAs could not finish in time.
+      // Estimates: one SM's port stores at most 57 GB/s, shared by the CTA's communicator warps; a k-step of a pair
+      // tile takes 512 tensor cycles.
+      if (pair && a->wg_tail == 0) {
+        p.takeover = 1;
+        p.t_pt_ns = (uint32_t)((uint64_t)kCommWarps * kTileBytes * (W - 1) / 45);   // 45 GB/s: what a communication SM sustains
+        p.t_tile_ns = (uint32_t)std::min<int64_t>((int64_t)p.kblocks * 260, 1 << 30);   // at full clocks: errs towards keeping
+      }
     }
 
     // Tensor maps.  K == 0 has no operand to describe; the kernel then never issues a load.
@@ -1364,8 +1435,9 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   }
   if (pair) {
     p.dynamic = a->static_schedule ? 0 : 1;
-    p.tile_counter = h->status + 16;   // a spare word of the status block; every launch starts it at zero
-    if (p.dynamic) IRIS_CUDA_TRY(cudaMemsetAsync(p.tile_counter, 0, sizeof(int32_t), st));
+    p.tile_counter = h->status + 16;   // spare words of the status block; every launch starts them at zero
+    p.backlog = h->status + 17;        // [17] publication tiles waiting for the communication CTAs, [18] tiles kept by producers
+    if (p.dynamic || p.takeover) IRIS_CUDA_TRY(cudaMemsetAsync(p.tile_counter, 0, 3 * sizeof(int32_t), st));
   }
   const bool cons_in_kernel = pair && fused_consumer && a->mode != IRIS_MODE_BULK_SYNCHRONOUS;  // BSP publishes in its 2nd kernel
   if (cons_in_kernel) { p.bias = static_cast<const uint8_t*>(a->consumer_bias); p.out_off = a->consumer_out_off; }
@@ -1413,6 +1485,16 @@ static int short_form(const void* A, const void* const* B_shards, iris_heap* hea
 
 int gemm_all_scatter(const void* A, const void* const* B_shards, iris_heap* heap, int M, int N, int K, int world, int mode) {
   return short_form(A, B_shards, heap, M, N, K, world, mode, IRIS_BF16, nullptr);
+}
+
+int iris_gemm_takeover_stats(const iris_heap* heap, int32_t out[2]) {
+  if (!heap_ok(heap) || !out) return fail(IRIS_ERR_ARG, "iris_gemm_takeover_stats: bad argument");
+  int32_t w[2];
+  IRIS_CUDA_TRY(cudaSetDevice(heap->device));
+  IRIS_CUDA_TRY(cudaMemcpy(w, heap->status + 17, sizeof(w), cudaMemcpyDeviceToHost));
+  out[0] = w[1];
+  out[1] = w[0];
+  return IRIS_OK;
 }
 
 uint64_t iris_gemm_out_offset(int M, int N, int world) {

@@ -98,7 +98,7 @@ def test_communication_ctas_give_up_when_a_lock_is_never_released():
     c_off, flag_off, lock_off, out_off, bpr = gemm_layout(M, N, W, with_out=True)
     with GpuHeap(W, bpr) as g:
         nt = oracle.num_tiles(M, N, W)
-        iris.iris_flags_fill(g.h, lock_off, nt, 2)
+        iris.iris_flags_fill(g.h, lock_off, nt, 3)    # neither free (0) nor a state the communicators act on (1, 2)
         iris.iris_flags_fill(g.h, flag_off, nt, 0)
         iris.iris_gemm_all_scatter_ex(g.h, dev16(A), [dev16(b) for b in Bs], M, N, K, W, iris.IRIS_MODE_WORKGROUP_SPECIALIZED,
                                       iris.IRIS_BF16, c_off, flag_off, lock_off, 1, spin_timeout_ns=3_000_000, wg_tail=-1)

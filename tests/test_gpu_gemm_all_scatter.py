@@ -362,3 +362,26 @@ def test_workgroup_specialized_tail_tiles_scattered_by_producers(wg_tail, W, M, 
         host = g.to_host()
         img, _ = expected_image(g, A, Bs, dtype, mode)
         assert np.array_equal(host, img.mem), first_diff(host, img.mem)
+
+
+def test_producers_take_over_what_the_communication_ctas_cannot_finish():
+    """Two communication CTAs for a scatter that needs many more: with the default rule the producers keep most tiles
+    (and say so), with Listing 5 throughout they keep none; the heap image is the oracle's in both cases."""
+    W, M, nl, K, dtype, mode = 8, 2048, 512, 512, "bf16", iris.IRIS_MODE_WORKGROUP_SPECIALIZED
+    N = W * nl
+    A = inputs.matrix(59, inputs.STREAM_A, M, K, "ternary:0.25", dtype)
+    Bs = [inputs.matrix(59, inputs.STREAM_B0 + r, nl, K, "smallint:1", dtype) for r in range(W)]
+    bpr = gemm_layout(M, N, W, True)[4]
+    c_full = None
+    for wg_tail, comm in ((0, 2), (0, 0), (-1, 2), (0, 40)):
+        with GpuHeap(W, bpr) as g:
+            run_gemm(g, A, Bs, dtype, mode, wg_tail=wg_tail, comm_ctas=comm)
+            kept, queued = iris.iris_gemm_takeover_stats(g.h)
+            host = g.to_host()
+            img, c_full = expected_image(g, A, Bs, dtype, mode, c_full=c_full)
+            assert np.array_equal(host, img.mem), (wg_tail, comm, first_diff(host, img.mem))
+            assert queued == 0
+            if wg_tail < 0:
+                assert kept == 0
+            elif comm == 2:
+                assert kept > 0          # 8 x 16 pair tiles, 73 producer pairs: one full wave before the last, far too much for 12 warps
