@@ -18,6 +18,7 @@ cross-GPU exchange step); the value is the sum over ranks, timed as the max over
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
 import os
 import subprocess
@@ -70,13 +71,14 @@ def align(x, a=256):
 
 
 class ClockSampler:
-    """nvidia-smi clocks / throttle reasons sampled every 20 ms while the timed region runs."""
+    """nvidia-smi clocks / throttle reasons sampled every 20 ms.  The sampler is started before the warm-up (nvidia-smi
+    needs 100-200 ms to deliver its first line); only the lines stamped inside the timed region [mark(), stop()] count."""
 
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
-        self.index, self.proc, self.path = index, None, None
+        self.index, self.proc, self.path, self.t0 = index, None, None, None
 
     def start(self):
         try:
@@ -87,11 +89,15 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def mark(self):
+        self.t0 = datetime.datetime.now()
+
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
-        time.sleep(0.15)
+        t1 = datetime.datetime.now()
+        time.sleep(0.1)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -101,13 +107,17 @@ class ClockSampler:
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in open(self.path):
             f = [x.strip() for x in line.split(",")]
-            if len(f) < 7:
+            if len(f) < 8:
                 continue
             try:
-                sm.append(float(f[0])); mx.append(float(f[1])); pw.append(float(f[2]))
+                stamp = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f")
+                if self.t0 is not None and not (self.t0 <= stamp <= t1):
+                    continue
+                vals = (float(f[1]), float(f[2]), float(f[3]))
             except ValueError:
                 continue
-            for n, v in zip(names, f[3:7]):
+            sm.append(vals[0]); mx.append(vals[1]); pw.append(vals[2])
+            for n, v in zip(names, f[4:8]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         os.unlink(self.path)
@@ -220,6 +230,8 @@ def run_ours(args):
 
     A, Bs = inputs.gemm_inputs(seed, W, M, N, K, dist_name, dtype)
     bias = inputs.vector(seed, inputs.STREAM_BIAS, N, "uniform", dtype)
+    sampler = ClockSampler(local_rank)
+    sampler.start()           # long before the timed region: see the class
     dA = torch.from_numpy(A.view(np.int16)).cuda()
     dB = [torch.from_numpy(b.view(np.int16)).cuda() for b in Bs]
     dbias = torch.from_numpy(bias.view(np.int16)).cuda()
@@ -270,9 +282,8 @@ def run_ours(args):
 
     # ---------------- timed region: exactly K steps ----------------
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    sampler = ClockSampler(local_rank)
     barrier()
-    sampler.start()
+    sampler.mark()
     for i in range(args.steps):
         epoch += 1
         step(epoch, ev[i])
