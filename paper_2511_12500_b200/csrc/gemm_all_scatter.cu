@@ -1256,10 +1256,10 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     bn = a->block_n;
     if (bn == 0) {
       bn = (nl % 256 == 0 || nl > 1024) ? 256 : 128;
-      // skinny problems (one tile row) with stream-K switched off: 256-wide tiles would leave SMs without work while
-      // the kernel is bound by how many operand bytes all SMs together keep in flight; narrower tiles spread the
-      // B panels over every SM.  (With stream-K every SM gets the same share of k-steps whatever the tile width.)
-      if (a->stream_k <= 0 && (int64_t)((a->M + BM - 1) / BM) * W * ((nl + 255) / 256) < h->sm_count) bn = 128;
+      // Few tiles (the skinny shapes): when the 128-wide tiles all fit in one wave they put more SMs to work on the
+      // B panels; when they need a second, partly filled wave (config 4: 224 tiles on 148 SMs) one wave of 256-wide
+      // tiles is faster (measured 0.127 vs 0.142 ms) although a quarter of the SMs then idle.
+      if ((int64_t)((a->M + BM - 1) / BM) * W * ((nl + 127) / 128) <= h->sm_count) bn = 128;
     }
     if (nl <= 128) bn = 128;
     // CTA pairs (256 x 256 tiles) need at least two tile rows.  A shard that is not a whole number of 256-column
