@@ -280,8 +280,13 @@ int iris_consume_bias(iris_heap* heap, uint64_t c_off, uint64_t out_off, uint64_
  * iris_gemm_out_offset(M, N, world); copies slot `out_slot`'s C ([M, N], to C_host), its OUT (to
  * OUT_host; bias_host and OUT_host are both NULL or both non-NULL) and the flags of all slots
  * (world * iris_num_tiles int32, slot-major, to flags_host; may be NULL) back, and returns after
- * everything has completed.  Runs on the legacy default stream.  Host buffers should be pinned for
- * full copy speed.  With a bias the heap needs bytes_per_rank >= iris_gemm_out_offset + M*N*2. */
+ * everything has completed.  The work is pipelined over blocks of rows (M >= 1024: up to 8 blocks of
+ * whole 256-row tiles) on three streams the heap handle owns: while block i computes, block i+1's rows
+ * of A arrive and block i-1's rows of C and OUT leave, so both directions of the host link are busy
+ * at once; every block is the same operation on its rows, and the result is the one an unblocked call
+ * gives.  Synchronises the device on entry (the call owns the heap until it returns).  Host buffers
+ * should be pinned for full copy speed.  With a bias the heap needs bytes_per_rank >=
+ * iris_gemm_out_offset + M*N*2. */
 int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_host, void* C_host,
                                int32_t* flags_host, const void* bias_host, void* OUT_host, iris_heap* heap,
                                int M, int N, int K, int world, int mode, int dtype, int out_slot);

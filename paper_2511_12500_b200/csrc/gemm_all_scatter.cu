@@ -1174,6 +1174,26 @@ int64_t num_tiles(int M, int N, int world) {
   return (int64_t)((M + IRIS_TILE - 1) / IRIS_TILE) * world * ((nl + IRIS_TILE - 1) / IRIS_TILE);
 }
 
+// Streams and events of iris_gemm_all_scatter_host's copy / compute / copy-back pipeline.
+constexpr int kHostPipeChunks = 8;
+struct HostPipe {
+  cudaStream_t s[3];
+  cudaEvent_t b_ready, a_ready[kHostPipeChunks + 1], c_ready[kHostPipeChunks + 1];
+};
+
+void free_host_pipe(iris_heap* h) {
+  HostPipe* hp = static_cast<HostPipe*>(h->host_pipe);
+  if (!hp) return;
+  for (cudaStream_t st : hp->s) if (st) cudaStreamDestroy(st);
+  if (hp->b_ready) cudaEventDestroy(hp->b_ready);
+  for (int i = 0; i <= kHostPipeChunks; ++i) {
+    if (hp->a_ready[i]) cudaEventDestroy(hp->a_ready[i]);
+    if (hp->c_ready[i]) cudaEventDestroy(hp->c_ready[i]);
+  }
+  delete hp;
+  h->host_pipe = nullptr;
+}
+
 }  // namespace iris
 
 using namespace iris;
@@ -1517,6 +1537,8 @@ int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_h
   if (bias_host && out_off + c_bytes > heap->bytes_per_rank) return fail(IRIS_ERR_RANGE, "gemm_all_scatter_host: heap slot too small for OUT");
   const size_t a_bytes = (size_t)M * K * 2, b_bytes = (size_t)N * K * 2, shard_bytes = world ? b_bytes / world : 0;
   const size_t stage_b_need = b_bytes + (bias_host ? align_up((uint64_t)N * 2, 256) : 0);
+  IRIS_CUDA_TRY(cudaSetDevice(heap->device));
+  IRIS_CUDA_TRY(cudaDeviceSynchronize());   // the call owns the heap from here on; it returns only when everything is done
   if (a_bytes > heap->stage_a_bytes) {
     if (heap->stage_a) cudaFree(heap->stage_a);
     heap->stage_a = nullptr; heap->stage_a_bytes = 0;
@@ -1529,27 +1551,78 @@ int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_h
     if (cudaMalloc(&heap->stage_b, stage_b_need) != cudaSuccess) { cudaGetLastError(); return fail(IRIS_ERR_NOMEM, "gemm_all_scatter_host: staging for B"); }
     heap->stage_b_bytes = stage_b_need;
   }
-  cudaStream_t st = nullptr;
+  HostPipe* hp = static_cast<HostPipe*>(heap->host_pipe);
+  if (!hp) {
+    hp = new HostPipe();
+    std::memset(hp, 0, sizeof(*hp));
+    heap->host_pipe = hp;
+    for (int i = 0; i < 3; ++i) IRIS_CUDA_TRY(cudaStreamCreateWithFlags(&hp->s[i], cudaStreamNonBlocking));
+    IRIS_CUDA_TRY(cudaEventCreateWithFlags(&hp->b_ready, cudaEventDisableTiming));
+    for (int i = 0; i <= kHostPipeChunks; ++i) {
+      IRIS_CUDA_TRY(cudaEventCreateWithFlags(&hp->a_ready[i], cudaEventDisableTiming));
+      IRIS_CUDA_TRY(cudaEventCreateWithFlags(&hp->c_ready[i], cudaEventDisableTiming));
+    }
+  }
+  cudaStream_t s_in = hp->s[0], s_run = hp->s[1], s_out = hp->s[2];
+
+  // Three streams: host-to-device copies, kernels, device-to-host copies.  B (and the bias) go first; A goes in
+  // blocks of rows, and every block is its own gemm_all_scatter over rows [r0, r1) -- C, OUT, flags and locks of a
+  // row block are contiguous in the short form's layout, so a block is the same call with shifted offsets -- whose
+  // rows of C (and OUT) start back to the host as soon as its kernels are done.  PCIe carries both directions at
+  // once, and the GEMM hides behind the copies.
   const void* dB[IRIS_MAX_WORLD] = {nullptr};
-  if (a_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(heap->stage_a, A_host, a_bytes, cudaMemcpyHostToDevice, st));
   for (int r = 0; r < world; ++r) {
     dB[r] = static_cast<char*>(heap->stage_b) + (size_t)r * shard_bytes;
-    if (shard_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(dB[r]), B_shards_host[r], shard_bytes, cudaMemcpyHostToDevice, st));
+    if (shard_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(dB[r]), B_shards_host[r], shard_bytes, cudaMemcpyHostToDevice, s_in));
   }
   void* dbias = static_cast<char*>(heap->stage_b) + b_bytes;
-  if (bias_host && N > 0) IRIS_CUDA_TRY(cudaMemcpyAsync(dbias, bias_host, (size_t)N * 2, cudaMemcpyHostToDevice, st));
-  // with a bias the consumer is part of the same call (inside the GEMM launch where the kernel supports it)
-  int rc = short_form(heap->stage_a, dB, heap, M, N, K, world, mode, dtype, st, (bias_host && c_bytes) ? dbias : nullptr, out_off);
-  if (rc != IRIS_OK) return rc;
+  if (bias_host && N > 0) IRIS_CUDA_TRY(cudaMemcpyAsync(dbias, bias_host, (size_t)N * 2, cudaMemcpyHostToDevice, s_in));
+  IRIS_CUDA_TRY(cudaEventRecord(hp->b_ready, s_in));
+  IRIS_CUDA_TRY(cudaStreamWaitEvent(s_run, hp->b_ready, 0));
+
   uint64_t flag_off, lock_off;
   short_form_layout(M, N, world, &flag_off, &lock_off);
+  const int nl = world ? N / world : 0;
+  const int64_t tiles_per_row = (int64_t)world * ((nl + IRIS_TILE - 1) / IRIS_TILE);
+  int rows_per_block = M;   // whole problem unless it is tall enough to be worth cutting (blocks of whole pair tiles)
+  if (M >= 1024) rows_per_block = std::max(512, (int)align_up((uint64_t)(M + kHostPipeChunks - 1) / kHostPipeChunks, 256));
   char* slot = heap->base + (size_t)out_slot * heap->bytes_per_rank;
-  if (c_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(C_host, slot, c_bytes, cudaMemcpyDeviceToHost, st));
-  if (bias_host && c_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(OUT_host, slot + out_off, c_bytes, cudaMemcpyDeviceToHost, st));
+  const int32_t epoch = heap->epoch + 1;
+  int blk = 0;
+  for (int r0 = 0; r0 < M || (r0 == 0 && blk == 0); r0 += rows_per_block, ++blk) {
+    const int rows = std::min(rows_per_block, M - r0);
+    const size_t a_off = (size_t)r0 * K * 2, row_off = (size_t)r0 * N * 2;
+    if (rows > 0 && K > 0) IRIS_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(heap->stage_a) + a_off, static_cast<const char*>(A_host) + a_off, (size_t)rows * K * 2, cudaMemcpyHostToDevice, s_in));
+    IRIS_CUDA_TRY(cudaEventRecord(hp->a_ready[blk], s_in));
+    IRIS_CUDA_TRY(cudaStreamWaitEvent(s_run, hp->a_ready[blk], 0));
+    iris_gemm_args a;
+    std::memset(&a, 0, sizeof(a));
+    a.A = static_cast<char*>(heap->stage_a) + a_off;
+    a.B_shards = dB; a.heap = heap;
+    a.M = rows; a.N = N; a.K = K; a.world = world; a.mode = mode; a.dtype = dtype;
+    a.c_off = row_off;
+    a.flag_off = flag_off + (uint64_t)(r0 / IRIS_TILE) * tiles_per_row * 4;
+    a.lock_off = lock_off + (uint64_t)(r0 / IRIS_TILE) * tiles_per_row * 4;
+    a.epoch = epoch;
+    // with a bias the consumer is part of the same call (inside the GEMM launch where the kernel supports it)
+    a.consumer_bias = (bias_host && c_bytes) ? dbias : nullptr;
+    a.consumer_out_off = out_off + row_off;
+    const int rc = iris_gemm_all_scatter_ex(&a, s_run);
+    if (rc != IRIS_OK) { cudaDeviceSynchronize(); return rc; }
+    IRIS_CUDA_TRY(cudaEventRecord(hp->c_ready[blk], s_run));
+    IRIS_CUDA_TRY(cudaStreamWaitEvent(s_out, hp->c_ready[blk], 0));
+    if (rows > 0 && N > 0) {
+      IRIS_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(C_host) + row_off, slot + row_off, (size_t)rows * N * 2, cudaMemcpyDeviceToHost, s_out));
+      if (bias_host) IRIS_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(OUT_host) + row_off, slot + out_off + row_off, (size_t)rows * N * 2, cudaMemcpyDeviceToHost, s_out));
+    }
+  }
+  heap->epoch = epoch;
   if (flags_host && nt > 0)
     for (int s = 0; s < world; ++s)
-      IRIS_CUDA_TRY(cudaMemcpyAsync(flags_host + (size_t)s * nt, heap->base + (size_t)s * heap->bytes_per_rank + flag_off, (size_t)nt * 4, cudaMemcpyDeviceToHost, st));
-  return iris_status_check(heap, st, nullptr);
+      IRIS_CUDA_TRY(cudaMemcpyAsync(flags_host + (size_t)s * nt, heap->base + (size_t)s * heap->bytes_per_rank + flag_off, (size_t)nt * 4, cudaMemcpyDeviceToHost, s_out));
+  IRIS_CUDA_TRY(cudaStreamSynchronize(s_out));
+  IRIS_CUDA_TRY(cudaStreamSynchronize(s_in));
+  return iris_status_check(heap, s_run, nullptr);
 }
 
 // The one entry point that allocates nothing (see the header).  Workgroup-specialised schedule with the

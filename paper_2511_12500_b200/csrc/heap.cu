@@ -99,6 +99,7 @@ int iris_heap_destroy(iris_heap* h) {
   if (h->stage_a) cudaFree(h->stage_a);
   if (h->stage_b) cudaFree(h->stage_b);
   if (h->ws) cudaFree(h->ws);
+  iris::free_host_pipe(h);
   h->magic = 0;
   delete h;
   cudaGetLastError();

@@ -57,6 +57,8 @@ struct iris_heap {
   // stream-K workspace (partial sums + arrival counters), allocated on first use
   void* ws;
   size_t ws_bytes;
+  // streams and events of the host-buffer entry point's copy/compute pipeline, created on first use
+  void* host_pipe;
   iris::HeapTable table() const {
     iris::HeapTable t{};
     for (int r = 0; r < world; ++r) t.base[r] = (uint64_t)(base + (size_t)r * bytes_per_rank);
@@ -68,4 +70,5 @@ struct iris_heap {
 
 namespace iris {
 inline bool heap_ok(const iris_heap* h) { return h && h->magic == kHeapMagic; }
+void free_host_pipe(iris_heap* h);   // gemm_all_scatter.cu
 }  // namespace iris

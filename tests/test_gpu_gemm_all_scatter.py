@@ -385,3 +385,37 @@ def test_producers_take_over_what_the_communication_ctas_cannot_finish():
                 assert kept == 0
             elif comm == 2:
                 assert kept > 0          # 8 x 16 pair tiles, 73 producer pairs: one full wave before the last, far too much for 12 warps
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+def test_host_buffer_call_pipelined_over_row_blocks(mode):
+    """M = 1300 is cut into row blocks (512, 512, 276) that are copied, computed and copied back on three streams: the
+    host outputs and the whole heap image must be what the single call on device buffers gives (the oracle's)."""
+    W, M, nl, K, dtype = 4, 1300, 384, 136, "bf16"
+    N = W * nl
+    A = inputs.matrix(61, inputs.STREAM_A, M, K, "ternary:0.5", dtype)
+    Bs = [inputs.matrix(61, inputs.STREAM_B0 + r, nl, K, "smallint:2", dtype) for r in range(W)]
+    bias = inputs.vector(61, inputs.STREAM_BIAS, N, "smallint:3", dtype)
+    nt = oracle.num_tiles(M, N, W)
+    c_off, flag_off = 0, (M * N * 2 + 255) // 256 * 256                  # the short form's layout
+    lock_off = flag_off + (nt * 4 + 255) // 256 * 256
+    out_off = lock_off + (nt * 4 + 255) // 256 * 256
+    assert out_off == iris.iris_gemm_out_offset(M, N, W)
+    bpr = out_off + (M * N * 2 + 255) // 256 * 256 + 256
+    with GpuHeap(W, bpr) as g:
+        img = g.image()
+        for s in range(W):
+            img.view(s, lock_off, nt * 4, np.int32)[:] = 0
+        iris.iris_flags_fill(g.h, lock_off, nt, 0)
+        C_host, OUT_host = np.zeros((M, N), dtype=np.uint16), np.zeros((M, N), dtype=np.uint16)
+        flags = np.zeros((W, nt), dtype=np.int32)
+        for call in (1, 2):                      # the second call reuses the handle's streams, events and staging
+            iris.iris_gemm_all_scatter_host(A, Bs, C_host, flags, bias, OUT_host, g.h, M, N, K, W, mode, iris.IRIS_BF16, W - 1)
+            assert np.all(flags == call)
+        img.gemm_all_scatter(A, Bs, dtype, c_off, flag_off, 2, lock_off if mode == iris.IRIS_MODE_WORKGROUP_SPECIALIZED else None)
+        img.consume_bias(dtype, c_off, out_off, M, N, bias)
+        host = g.to_host()
+        assert np.array_equal(host, img.mem), first_diff(host, img.mem)
+        c_ref = c_slot(img.mem, g, 0, c_off, M, N)
+        assert np.array_equal(C_host, c_ref)
+        assert np.array_equal(OUT_host, oracle.consume_bias_rows(c_ref, bias, dtype))
