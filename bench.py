@@ -74,7 +74,7 @@ class ClockSampler:
     """nvidia-smi clocks / throttle reasons sampled every 20 ms.  The sampler is started before the warm-up (nvidia-smi
     needs 100-200 ms to deliver its first line); only the lines stamped inside the timed region [mark(), stop()] count."""
 
-    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,power.limit,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
          "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index: int):
@@ -103,27 +103,27 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, pw, reasons = [], [], [], set()
+        sm, mx, pw, reasons, lim = [], [], [], set(), None
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in open(self.path):
             f = [x.strip() for x in line.split(",")]
-            if len(f) < 8:
+            if len(f) < 9:
                 continue
             try:
                 stamp = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f")
                 if self.t0 is not None and not (self.t0 <= stamp <= t1):
                     continue
-                vals = (float(f[1]), float(f[2]), float(f[3]))
+                vals = (float(f[1]), float(f[2]), float(f[3]), float(f[4]))
             except ValueError:
                 continue
-            sm.append(vals[0]); mx.append(vals[1]); pw.append(vals[2])
-            for n, v in zip(names, f[4:8]):
+            sm.append(vals[0]); mx.append(vals[1]); pw.append(vals[2]); lim = vals[3]
+            for n, v in zip(names, f[5:9]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         os.unlink(self.path)
         if sm:
             out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), power_w_max=float(max(pw)), reasons=sorted(reasons),
-                       samples=len(sm))
+                       samples=len(sm), power_limit_w=lim)
         return out
 
 
