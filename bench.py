@@ -432,7 +432,7 @@ def run_ours(args):
             h2d = (M * K + N * K + N) * 2
             d2h = 2 * M * N * 2 + W * nt * 4
             result["e2e"] = {"value": flops / e2e_s / 1e12, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                             "ms_per_step": e2e_s * 1e3, "api": "iris_gemm_all_scatter_host (pinned host buffers; row blocks pipelined over copy-in, compute and copy-out streams)"}
+                             "ms_per_step": e2e_s * 1e3, "api": "iris_gemm_all_scatter_host (pinned host buffers; one block per rank shard, pipelined over copy-in, compute and copy-out streams)"}
             del hA, hB, hC, hOUT
         except Exception as exc:  # pragma: no cover
             result["e2e"] = {"value": None, "unit": UNIT, "error": str(exc)}

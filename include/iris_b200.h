@@ -242,6 +242,13 @@ typedef struct iris_gemm_args {
                                   still to come (so too few communication CTAs cost little);
                                   n > 0 = exactly the last n tiles; -1 = none (Listing 5 for every
                                   tile).  The final heap image is the same in every case        */
+  int rank_first, rank_count;  /* compute, scatter and publish only the shards of ranks
+                                  [rank_first, rank_first + rank_count): what one rank of a real
+                                  W-GPU job runs (its own N/world columns into every slot), and
+                                  what a pipeline over shards runs per stage.  0, 0 = every rank.
+                                  B_shards entries outside the range are not read; tiles, flags and
+                                  locks of other ranks are not touched; a consumer that is part of
+                                  the call covers the same ranks                                  */
   const void* consumer_bias;   /* not NULL: also run the flag-gated consumer OUT = C + bias (see
                                   iris_consume_bias) as part of this call: inside the same launch,
                                   as extra warps that acquire each tile's flag while the GEMM is
@@ -273,6 +280,11 @@ int64_t iris_num_tiles(int M, int N, int world);
  * row-major [M, N] region at out_off in every slot.  ctas: grid size (0 = 8 per SM). */
 int iris_consume_bias(iris_heap* heap, uint64_t c_off, uint64_t out_off, uint64_t flag_off, const void* bias, int M,
                       int N, int world, int dtype, int32_t epoch, int ctas, uint64_t timeout_ns, void* stream);
+/* The same for the publication tiles of ranks [rank_first, rank_first + rank_count) only (the column
+ * shards those ranks own, in every slot); rank_count = 0 does nothing. */
+int iris_consume_bias_ranks(iris_heap* heap, uint64_t c_off, uint64_t out_off, uint64_t flag_off, const void* bias,
+                            int M, int N, int world, int rank_first, int rank_count, int dtype, int32_t epoch,
+                            int ctas, uint64_t timeout_ns, void* stream);
 
 /* End-to-end form with HOST buffers: copies A and the W shards (and bias, if given) to device staging
  * owned by the heap (allocated on first use, reused afterwards), runs gemm_all_scatter in `mode` with

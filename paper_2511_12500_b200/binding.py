@@ -31,7 +31,7 @@ EXPORTS = [
     "iris_status_check", "iris_put_tile", "iris_get_tile", "iris_atomic_add", "iris_atomic_cas",
     "iris_atomic_add_contended", "iris_atomic_cas_contended", "iris_flags_fill", "iris_all_store_bench",
     "iris_gemm_all_scatter_ex", "gemm_all_scatter", "iris_gemm_heap_bytes", "iris_heap_epoch", "iris_num_tiles",
-    "iris_consume_bias", "iris_gemm_all_scatter_host", "iris_gemm_out_offset", "iris_gemm_takeover_stats",
+    "iris_consume_bias", "iris_consume_bias_ranks", "iris_gemm_all_scatter_host", "iris_gemm_out_offset", "iris_gemm_takeover_stats",
     "iris_gemm_all_scatter_noalloc", "iris_copy_tile", "iris_load_tile", "iris_store_tile", "iris_atomic_rmw",
 ]
 
@@ -48,7 +48,7 @@ class GemmArgs(C.Structure):
         ("M", C.c_int), ("N", C.c_int), ("K", C.c_int), ("world", C.c_int), ("mode", C.c_int), ("dtype", C.c_int),
         ("c_off", C.c_uint64), ("flag_off", C.c_uint64), ("lock_off", C.c_uint64),
         ("epoch", C.c_int32), ("comm_ctas", C.c_int), ("max_ctas", C.c_int), ("raster_group", C.c_int),
-        ("block_n", C.c_int), ("spin_timeout_ns", C.c_uint64), ("cta_pair", C.c_int), ("static_schedule", C.c_int), ("stream_k", C.c_int), ("wg_tail", C.c_int),
+        ("block_n", C.c_int), ("spin_timeout_ns", C.c_uint64), ("cta_pair", C.c_int), ("static_schedule", C.c_int), ("stream_k", C.c_int), ("wg_tail", C.c_int), ("rank_first", C.c_int), ("rank_count", C.c_int),
         ("consumer_bias", C.c_void_p), ("consumer_out_off", C.c_uint64),
     ]
 
@@ -102,6 +102,7 @@ def lib() -> C.CDLL:
     L.iris_num_tiles.restype = C.c_int64
     L.iris_num_tiles.argtypes = [ci, ci, ci]
     L.iris_consume_bias.argtypes = [vp, u64, u64, u64, vp, ci, ci, ci, ci, i32, ci, u64, vp]
+    L.iris_consume_bias_ranks.argtypes = [vp, u64, u64, u64, vp, ci, ci, ci, ci, ci, ci, i32, ci, u64, vp]
     L.iris_gemm_all_scatter_host.argtypes = [vp, C.POINTER(vp), vp, vp, vp, vp, vp, ci, ci, ci, ci, ci, ci, ci]
     L.iris_gemm_takeover_stats.argtypes = [vp, C.POINTER(C.c_int32)]
     L.iris_gemm_out_offset.restype = u64
@@ -277,10 +278,10 @@ def _shards(B_shards):
 
 
 def iris_gemm_all_scatter_ex(heap, A, B_shards, M, N, K, world, mode, dtype, c_off, flag_off, lock_off=0, epoch=1,
-                             comm_ctas=0, max_ctas=0, raster_group=0, block_n=0, spin_timeout_ns=0, cta_pair=0, static_schedule=0, stream_k=0, wg_tail=0, consumer_bias=None, consumer_out_off=0, stream=None):
+                             comm_ctas=0, max_ctas=0, raster_group=0, block_n=0, spin_timeout_ns=0, cta_pair=0, static_schedule=0, stream_k=0, wg_tail=0, rank_first=0, rank_count=0, consumer_bias=None, consumer_out_off=0, stream=None):
     arr = _shards(B_shards)
     a = GemmArgs(_ptr(A), C.cast(arr, C.POINTER(C.c_void_p)), heap, M, N, K, world, mode, dtype, c_off, flag_off, lock_off,
-                 epoch, comm_ctas, max_ctas, raster_group, block_n, spin_timeout_ns, cta_pair, static_schedule, stream_k, wg_tail, _ptr(consumer_bias), consumer_out_off)
+                 epoch, comm_ctas, max_ctas, raster_group, block_n, spin_timeout_ns, cta_pair, static_schedule, stream_k, wg_tail, rank_first, rank_count, _ptr(consumer_bias), consumer_out_off)
     _ck(lib().iris_gemm_all_scatter_ex(C.byref(a), _stream(stream)))
 
 
@@ -292,6 +293,11 @@ def gemm_all_scatter(A, B_shards, heap, M, N, K, world, mode):
 
 def iris_consume_bias(heap, c_off, out_off, flag_off, bias, M, N, world, dtype, epoch, ctas=0, timeout_ns=0, stream=None):
     _ck(lib().iris_consume_bias(heap, c_off, out_off, flag_off, _ptr(bias), M, N, world, dtype, epoch, ctas, timeout_ns, _stream(stream)))
+
+
+def iris_consume_bias_ranks(heap, c_off, out_off, flag_off, bias, M, N, world, rank_first, rank_count, dtype, epoch, ctas=0, timeout_ns=0, stream=None):
+    _ck(lib().iris_consume_bias_ranks(heap, c_off, out_off, flag_off, _ptr(bias), M, N, world, rank_first, rank_count, dtype, epoch, ctas, timeout_ns,
+                                      _stream(stream)))
 
 
 def iris_gemm_takeover_stats(heap):

@@ -12,12 +12,16 @@ constexpr int kConsThreads = 256;
 template <bool BF16>
 __global__ void __launch_bounds__(kConsThreads) consume_bias_kernel(const __grid_constant__ HeapTable tab, uint64_t c_off, uint64_t out_off, uint64_t flag_off,
                                                                     const uint8_t* bias, int M, int N, int n_local, int tiles_m,
-                                                                    int ptiles_per_rank, int32_t epoch, uint64_t timeout_ns, int32_t* status) {
+                                                                    int ptiles_per_rank, int rank_first, int rank_count, int32_t epoch,
+                                                                    uint64_t timeout_ns, int32_t* status) {
   const int W = tab.world;
-  const int pt_n = W * ptiles_per_rank;
-  const int items = tiles_m * pt_n * W;  // (tile, slot) pairs, tile-major so early tiles are consumed first everywhere
+  const int pt_n = W * ptiles_per_rank;            // publication tiles per tile row, all ranks (the flag index uses this)
+  const int pt_sel = rank_count * ptiles_per_rank; // ... of the ranks this call covers
+  const int items = tiles_m * pt_sel * W;  // (tile, slot) pairs, tile-major so early tiles are consumed first everywhere
   for (int it = blockIdx.x; it < items; it += gridDim.x) {
-    const int t = it / W, s = it % W;
+    const int ti = it / W, s = it % W;
+    const int tm = ti / pt_sel, rank = rank_first + (ti % pt_sel) / ptiles_per_rank, pj = (ti % pt_sel) % ptiles_per_rank;
+    const int t = tm * pt_n + rank * ptiles_per_rank + pj;
     // ---- acquire the tile in slot s ----
     int failed = 0;
     if (threadIdx.x == 0) {
@@ -37,7 +41,6 @@ __global__ void __launch_bounds__(kConsThreads) consume_bias_kernel(const __grid
     }
     // the barrier orders thread 0's acquire before every thread's reads of the tile
     if (__syncthreads_or(failed)) return;
-    const int tm = t / pt_n, rank = (t % pt_n) / ptiles_per_rank, pj = (t % pt_n) % ptiles_per_rank;
     const int rows = min(IRIS_TILE, M - tm * IRIS_TILE);
     const int cols = min(IRIS_TILE, n_local - pj * IRIS_TILE);
     const int cpr = cols / 8;
@@ -79,12 +82,18 @@ using namespace iris;
 
 extern "C" int iris_consume_bias(iris_heap* h, uint64_t c_off, uint64_t out_off, uint64_t flag_off, const void* bias, int M, int N, int world,
                                  int dtype, int32_t epoch, int ctas, uint64_t timeout_ns, void* stream) {
+  return iris_consume_bias_ranks(h, c_off, out_off, flag_off, bias, M, N, world, 0, world, dtype, epoch, ctas, timeout_ns, stream);
+}
+
+extern "C" int iris_consume_bias_ranks(iris_heap* h, uint64_t c_off, uint64_t out_off, uint64_t flag_off, const void* bias, int M, int N, int world,
+                                       int rank_first, int rank_count, int dtype, int32_t epoch, int ctas, uint64_t timeout_ns, void* stream) {
   if (!heap_ok(h)) return fail(IRIS_ERR_STATE, "iris_consume_bias: bad heap handle");
   if (world != h->world) return fail(IRIS_ERR_ARG, "iris_consume_bias: world differs from the heap's");
+  if (rank_first < 0 || rank_count < 0 || rank_first + rank_count > world) return fail(IRIS_ERR_ARG, "iris_consume_bias: rank range outside [0, world)");
   if (dtype != IRIS_F16 && dtype != IRIS_BF16) return fail(IRIS_ERR_ARG, "iris_consume_bias: unknown dtype");
   if (M < 0 || N < 0 || N % world != 0 || (N / world) % 8 != 0) return fail(IRIS_ERR_ARG, "iris_consume_bias: bad M/N (N/world must be a multiple of 8)");
   if (c_off % 16 != 0 || out_off % 16 != 0 || flag_off % 4 != 0) return fail(IRIS_ERR_ARG, "iris_consume_bias: misaligned offsets");
-  if (M == 0 || N == 0) return IRIS_OK;
+  if (M == 0 || N == 0 || rank_count == 0) return IRIS_OK;
   if (!bias || (uint64_t)bias % 16 != 0) return fail(IRIS_ERR_ARG, "iris_consume_bias: bias is NULL or not 16-byte aligned");
   const uint64_t bpr = h->bytes_per_rank, bytes = (uint64_t)M * N * 2;
   const int nl = N / world;
@@ -93,15 +102,15 @@ extern "C" int iris_consume_bias(iris_heap* h, uint64_t c_off, uint64_t out_off,
   if (c_off > bpr || bytes > bpr - c_off || out_off > bpr || bytes > bpr - out_off || flag_off > bpr || nt * 4 > bpr - flag_off)
     return fail(IRIS_ERR_RANGE, "iris_consume_bias: a region leaves the slot");
   if (c_off < out_off + bytes && out_off < c_off + bytes) return fail(IRIS_ERR_ARG, "iris_consume_bias: C and OUT overlap");
-  const uint64_t items = nt * world;
+  const uint64_t items = (uint64_t)tiles_m * rank_count * ptr_ * world;
   uint64_t grid = ctas > 0 ? (uint64_t)ctas : (uint64_t)h->sm_count * 8;
   if (grid > items) grid = items;
   const uint64_t to = timeout_ns ? timeout_ns : kDefaultTimeoutNs;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (dtype == IRIS_BF16)
-    consume_bias_kernel<true><<<(int)grid, kConsThreads, 0, st>>>(h->table(), c_off, out_off, flag_off, static_cast<const uint8_t*>(bias), M, N, nl, tiles_m, ptr_, epoch, to, h->status);
+    consume_bias_kernel<true><<<(int)grid, kConsThreads, 0, st>>>(h->table(), c_off, out_off, flag_off, static_cast<const uint8_t*>(bias), M, N, nl, tiles_m, ptr_, rank_first, rank_count, epoch, to, h->status);
   else
-    consume_bias_kernel<false><<<(int)grid, kConsThreads, 0, st>>>(h->table(), c_off, out_off, flag_off, static_cast<const uint8_t*>(bias), M, N, nl, tiles_m, ptr_, epoch, to, h->status);
+    consume_bias_kernel<false><<<(int)grid, kConsThreads, 0, st>>>(h->table(), c_off, out_off, flag_off, static_cast<const uint8_t*>(bias), M, N, nl, tiles_m, ptr_, rank_first, rank_count, epoch, to, h->status);
   IRIS_CUDA_TRY(cudaGetLastError());
   return IRIS_OK;
 }

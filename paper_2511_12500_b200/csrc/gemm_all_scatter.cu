@@ -81,6 +81,7 @@ struct alignas(64) GemmParams {
   const uint8_t* bias;  // fused consumer: bias[N] of the element type (NULL = no consumer warps)
   uint64_t out_off;     // fused consumer: OUT region in every slot
   int gemm_ctas, comm_ctas;
+  int rank_first, rank_count;   // the ranks whose shards this call computes and scatters (all: 0, W)
   int streamk;          // single-CTA kernel: 1 = equal k-step ranges per CTA (tiles may be computed in parts)
   float* ws;            // stream-K: two fp32 tile slots per CTA for partial sums
   int32_t* arrive;      // stream-K: per compute tile, how many parts have been parked
@@ -117,7 +118,7 @@ struct TileCoord { int tm, rank, jn; };
 // `raster_group` tile rows before moving to the next tile column, so CTAs that run at the same
 // time share A row panels and B column panels in L2.
 __device__ __forceinline__ TileCoord decode_ctile(int id, const GemmParams& p) {
-  const int tiles_n = p.tab.world * p.ctiles_per_rank;
+  const int tiles_n = p.rank_count * p.ctiles_per_rank;
   const int per_group = p.raster_group * tiles_n;
   const int g = id / per_group;
   const int first_m = g * p.raster_group;
@@ -126,7 +127,7 @@ __device__ __forceinline__ TileCoord decode_ctile(int id, const GemmParams& p) {
   const int tn = in / gsz;
   TileCoord c;
   c.tm = first_m + in % gsz;
-  c.rank = tn / p.ctiles_per_rank;
+  c.rank = p.rank_first + tn / p.ctiles_per_rank;
   c.jn = tn % p.ctiles_per_rank;
   return c;
 }
@@ -394,7 +395,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
     fence_proxy_async();
     if (p.kblocks > 0 && !is_comm) {
       ptx::prefetch_tensormap(&p.tmA);
-      for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmB[r]);
+      for (int r = p.rank_first; r < p.rank_first + p.rank_count; ++r) ptx::prefetch_tensormap(&p.tmB[r]);
     }
     if (is_comm)
       for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmC[r]);
@@ -740,7 +741,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
     fence_proxy_async();
     if (p.kblocks > 0 && !is_comm) {
       ptx::prefetch_tensormap(&p.tmA);
-      for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmB[r]);
+      for (int r = p.rank_first; r < p.rank_first + p.rank_count; ++r) ptx::prefetch_tensormap(&p.tmB[r]);
     }
     if (is_comm)
       for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmC[r]);
@@ -983,12 +984,13 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
 // tile to every other rank, then publish the W ready flags.
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) all_scatter_kernel(const __grid_constant__ HeapTable tab, uint64_t c_off, uint64_t flag_off, int M, int N, int n_local,
-                                                          int tiles_m, int ptiles_per_rank, int32_t epoch) {
+                                                          int tiles_m, int ptiles_per_rank, int rank_first, int rank_count, int32_t epoch) {
   const int W = tab.world;
-  const int pt_n = W * ptiles_per_rank;
-  const int total = tiles_m * pt_n;
-  for (int t = blockIdx.x; t < total; t += gridDim.x) {
-    const int tm = t / pt_n, rank = (t % pt_n) / ptiles_per_rank, pj = (t % pt_n) % ptiles_per_rank;
+  const int pt_n = W * ptiles_per_rank, pt_sel = rank_count * ptiles_per_rank;
+  const int total = tiles_m * pt_sel;
+  for (int it = blockIdx.x; it < total; it += gridDim.x) {
+    const int tm = it / pt_sel, rank = rank_first + (it % pt_sel) / ptiles_per_rank, pj = (it % pt_sel) % ptiles_per_rank;
+    const int t = tm * pt_n + rank * ptiles_per_rank + pj;
     const int rows = min(IRIS_TILE, M - tm * IRIS_TILE);
     const int cols = min(IRIS_TILE, n_local - pj * IRIS_TILE);
     const int cpr = cols / 8;  // 16-byte chunks per row
@@ -1146,7 +1148,7 @@ struct PlanKey {
   const void* A; const void* B[IRIS_MAX_WORLD];
   int M, N, K, world, mode, dtype;
   uint64_t c_off, flag_off, lock_off;
-  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail, fused_consumer;
+  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail, fused_consumer, rank_first, rank_count;
   uint64_t spin_timeout_ns;
 };
 struct Plan { GemmParams p; int bn, grid; bool pair, streamk; };
@@ -1159,11 +1161,13 @@ static void make_key(PlanKey* k, const iris_gemm_args* a, const iris_heap* h) {
   std::memset(k, 0, sizeof(*k));   // padding too: keys are compared with memcmp
   k->heap = h; k->base = h->base; k->status = h->status; k->bytes_per_rank = h->bytes_per_rank;
   k->A = a->A;
-  for (int r = 0; r < a->world && r < IRIS_MAX_WORLD; ++r) k->B[r] = a->B_shards ? a->B_shards[r] : nullptr;
+  const int r_end = a->rank_count ? a->rank_first + a->rank_count : a->world;
+  for (int r = a->rank_first; r < r_end && r < IRIS_MAX_WORLD; ++r) k->B[r] = a->B_shards ? a->B_shards[r] : nullptr;
   k->M = a->M; k->N = a->N; k->K = a->K; k->world = a->world; k->mode = a->mode; k->dtype = a->dtype;
   k->c_off = a->c_off; k->flag_off = a->flag_off; k->lock_off = a->lock_off;
   k->comm_ctas = a->comm_ctas; k->max_ctas = a->max_ctas; k->raster_group = a->raster_group; k->block_n = a->block_n;
   k->cta_pair = a->cta_pair; k->static_schedule = a->static_schedule; k->stream_k = a->stream_k; k->wg_tail = a->wg_tail;
+  k->rank_first = a->rank_first; k->rank_count = a->rank_count;
   k->fused_consumer = a->consumer_bias != nullptr;   // the split between producers and communicators depends on it
   k->spin_timeout_ns = a->spin_timeout_ns;
 }
@@ -1231,6 +1235,9 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   if (a->cta_pair < -1 || a->cta_pair > 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: cta_pair must be -1, 0 or 1");
   if (a->wg_tail < -1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: wg_tail must be -1, 0 or a tile count");
   if (a->stream_k < -1 || a->stream_k > 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: stream_k must be -1, 0 or 1");
+  if (a->rank_first < 0 || a->rank_count < 0 || a->rank_first + a->rank_count > W || (a->rank_count == 0 && a->rank_first != 0))
+    return fail(IRIS_ERR_ARG, "gemm_all_scatter: rank range [%d, %d) outside [0, %d)", a->rank_first, a->rank_first + a->rank_count, W);
+  const int rank_first = a->rank_first, rank_count = a->rank_count ? a->rank_count : W;   // 0, 0 = every rank
   const int64_t nt = num_tiles(a->M, a->N, W);
   const uint64_t bpr = h->bytes_per_rank;
   const uint64_t c_bytes = (uint64_t)a->M * a->N * 2;
@@ -1253,7 +1260,7 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   if (!a->A && a->K > 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: A is NULL");
   if (!a->B_shards) return fail(IRIS_ERR_ARG, "gemm_all_scatter: B_shards is NULL");
   if ((uint64_t)a->A % 16 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: A must be 16-byte aligned");
-  for (int r = 0; r < W; ++r)
+  for (int r = rank_first; r < rank_first + rank_count; ++r)
     if (a->K > 0 && (!a->B_shards[r] || (uint64_t)a->B_shards[r] % 16 != 0)) return fail(IRIS_ERR_ARG, "gemm_all_scatter: B_shards[%d] is NULL or not 16-byte aligned", r);
 
   // The launch plan (tile geometry, grid split, tensor maps) depends on everything but the epoch; timing loops
@@ -1319,8 +1326,9 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     p.tiles_m = pair ? (a->M + 2 * BM - 1) / (2 * BM) : p.ptiles_m;
     p.ctiles_per_rank = (nl + bn - 1) / bn;
     p.ptiles_per_rank = (nl + IRIS_TILE - 1) / IRIS_TILE;
-    p.total_ctiles = p.tiles_m * W * p.ctiles_per_rank;
-    p.total_ptiles = p.ptiles_m * W * p.ptiles_per_rank;
+    p.rank_first = rank_first; p.rank_count = rank_count;
+    p.total_ctiles = p.tiles_m * rank_count * p.ctiles_per_rank;
+    p.total_ptiles = p.ptiles_m * rank_count * p.ptiles_per_rank;
     p.kblocks = (a->K + BK - 1) / BK;
     // 2048 rows per raster group: with tiles claimed in raster order the running tiles then cover about
     // 8 x 9 pair tiles, the near-square footprint that minimises operand re-reads from HBM (measured).
@@ -1335,8 +1343,8 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
         int comm = a->comm_ctas;
         // (with consumer warps in the producer CTAs their ports are busy with OUT = C + bias: the communication CTAs
         // then get the whole scatter, as they do without the takeover rule)
-        if (!comm) comm = a->wg_tail == 0 && !fused_consumer ? auto_comm_ctas_pair(p.total_ctiles, p.kblocks, (double)(W - 1) * a->M * a->N * 2.0, grid)
-                                                              : auto_comm_ctas(a->M, a->N, a->K, W, grid);
+        if (!comm) comm = a->wg_tail == 0 && !fused_consumer ? auto_comm_ctas_pair(p.total_ctiles, p.kblocks, (double)(W - 1) * a->M * nl * rank_count * 2.0, grid)
+                                                              : auto_comm_ctas(a->M, nl * rank_count, a->K, W, grid);
         comm = std::max(2, std::min((comm + 1) & ~1, grid - 2));   // whole pairs on both sides
         p.comm_ctas = comm;
         p.gemm_ctas = 2 * std::min((grid - comm) / 2, p.total_ctiles);
@@ -1346,7 +1354,7 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
       }
     } else if (wg) {
       if (grid < 2) return fail(IRIS_ERR_ARG, "gemm_all_scatter: workgroup_specialized needs at least 2 CTAs");
-      int comm = a->comm_ctas ? a->comm_ctas : auto_comm_ctas(a->M, a->N, a->K, W, grid);
+      int comm = a->comm_ctas ? a->comm_ctas : auto_comm_ctas(a->M, nl * rank_count, a->K, W, grid);
       comm = std::min(comm, std::min(grid - 1, p.total_ptiles));
       p.comm_ctas = comm;
       p.gemm_ctas = std::min(grid - comm, p.total_ctiles);
@@ -1399,7 +1407,7 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
       const cuuint32_t boxA[2] = {BK, BM};
       int rc = make_map(&p.tmA, a->dtype, 2, const_cast<void*>(a->A), dimsA, strA, boxA, CU_TENSOR_MAP_SWIZZLE_128B, "A");
       if (rc != IRIS_OK) return rc;
-      for (int r = 0; r < W; ++r) {
+      for (int r = rank_first; r < rank_first + rank_count; ++r) {
         const cuuint64_t dimsB[2] = {(cuuint64_t)a->K, (cuuint64_t)nl};
         const cuuint32_t boxB[2] = {BK, (cuuint32_t)(pair ? kPairBN / 2 : bn)};   // a pair's CTA loads its half of the tile
         rc = make_map(&p.tmB[r], a->dtype, 2, const_cast<void*>(a->B_shards[r]), dimsB, strA, boxB, CU_TENSOR_MAP_SWIZZLE_128B, "B");
@@ -1469,13 +1477,14 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   if (a->mode == IRIS_MODE_BULK_SYNCHRONOUS) {
     // Listing 3: the second kernel on the same stream; the kernel boundary is the synchronisation.
     const int g2 = std::min(p.total_ptiles, h->sm_count * 8);
-    all_scatter_kernel<<<g2, 256, 0, st>>>(p.tab, a->c_off, a->flag_off, a->M, a->N, nl, p.ptiles_m, p.ptiles_per_rank, a->epoch);
+    all_scatter_kernel<<<g2, 256, 0, st>>>(p.tab, a->c_off, a->flag_off, a->M, a->N, nl, p.ptiles_m, p.ptiles_per_rank, rank_first, rank_count, a->epoch);
     IRIS_CUDA_TRY(cudaGetLastError());
   }
   // Where the consumer does not ride inside the GEMM launch (single-CTA tiles, bulk-synchronous) it follows on
   // the same stream: same flags, same result.
   if (fused_consumer && !cons_in_kernel)
-    return iris_consume_bias(h, a->c_off, a->consumer_out_off, a->flag_off, a->consumer_bias, a->M, a->N, W, a->dtype, a->epoch, 0, a->spin_timeout_ns, stream);
+    return iris_consume_bias_ranks(h, a->c_off, a->consumer_out_off, a->flag_off, a->consumer_bias, a->M, a->N, W, rank_first, rank_count, a->dtype, a->epoch, 0,
+                                   a->spin_timeout_ns, stream);
   return IRIS_OK;
 }
 
@@ -1565,34 +1574,48 @@ int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_h
   }
   cudaStream_t s_in = hp->s[0], s_run = hp->s[1], s_out = hp->s[2];
 
-  // Three streams: host-to-device copies, kernels, device-to-host copies.  B (and the bias) go first; A goes in
-  // blocks of rows, and every block is its own gemm_all_scatter over rows [r0, r1) -- C, OUT, flags and locks of a
-  // row block are contiguous in the short form's layout, so a block is the same call with shifted offsets -- whose
-  // rows of C (and OUT) start back to the host as soon as its kernels are done.  PCIe carries both directions at
-  // once, and the GEMM hides behind the copies.
-  const void* dB[IRIS_MAX_WORLD] = {nullptr};
-  for (int r = 0; r < world; ++r) {
-    dB[r] = static_cast<char*>(heap->stage_b) + (size_t)r * shard_bytes;
-    if (shard_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(dB[r]), B_shards_host[r], shard_bytes, cudaMemcpyHostToDevice, s_in));
-  }
-  void* dbias = static_cast<char*>(heap->stage_b) + b_bytes;
-  if (bias_host && N > 0) IRIS_CUDA_TRY(cudaMemcpyAsync(dbias, bias_host, (size_t)N * 2, cudaMemcpyHostToDevice, s_in));
-  IRIS_CUDA_TRY(cudaEventRecord(hp->b_ready, s_in));
-  IRIS_CUDA_TRY(cudaStreamWaitEvent(s_run, hp->b_ready, 0));
-
+  // Three streams: host-to-device copies, kernels, device-to-host copies.  The smaller operand goes first and whole,
+  // the other one in blocks; every block is its own gemm_all_scatter, and its part of C (and OUT) starts back to the
+  // host as soon as its kernels are done, so the host link carries both directions at once and the GEMM hides behind
+  // the copies.
+  //   by ranks (A is the smaller operand)  block = one rank's shard B_r: the call covers ranks [r, r+1), all rows --
+  //                                        what that rank of a real job would run -- and returns a column block
+  //   by rows  (B is the smaller operand)  block = rows [r0, r1) of A: C, OUT, flags and locks of a row block are
+  //                                        contiguous in the short form's layout, so a block is the same call with
+  //                                        shifted offsets, and returns whole rows
   uint64_t flag_off, lock_off;
   short_form_layout(M, N, world, &flag_off, &lock_off);
   const int nl = world ? N / world : 0;
   const int64_t tiles_per_row = (int64_t)world * ((nl + IRIS_TILE - 1) / IRIS_TILE);
-  int rows_per_block = M;   // whole problem unless it is tall enough to be worth cutting (blocks of whole pair tiles)
-  if (M >= 1024) rows_per_block = std::max(512, (int)align_up((uint64_t)(M + kHostPipeChunks - 1) / kHostPipeChunks, 256));
+  const bool by_ranks = world >= 2 && world <= kHostPipeChunks && a_bytes <= b_bytes && c_bytes > 0;
+  int rows_per_block = M;   // by rows: whole problem unless it is tall enough to be worth cutting (blocks of whole pair tiles)
+  if (!by_ranks && M >= 1024) rows_per_block = std::max(512, (int)align_up((uint64_t)(M + kHostPipeChunks - 1) / kHostPipeChunks, 256));
+  const int blocks = by_ranks ? world : std::max(1, rows_per_block ? (M + rows_per_block - 1) / rows_per_block : 1);
+
+  const void* dB[IRIS_MAX_WORLD] = {nullptr};
+  for (int r = 0; r < world; ++r) dB[r] = static_cast<char*>(heap->stage_b) + (size_t)r * shard_bytes;
+  void* dbias = static_cast<char*>(heap->stage_b) + b_bytes;
+  if (bias_host && N > 0) IRIS_CUDA_TRY(cudaMemcpyAsync(dbias, bias_host, (size_t)N * 2, cudaMemcpyHostToDevice, s_in));
+  if (by_ranks) {
+    if (a_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(heap->stage_a, A_host, a_bytes, cudaMemcpyHostToDevice, s_in));
+  } else {
+    for (int r = 0; r < world; ++r)
+      if (shard_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(dB[r]), B_shards_host[r], shard_bytes, cudaMemcpyHostToDevice, s_in));
+  }
+  IRIS_CUDA_TRY(cudaEventRecord(hp->b_ready, s_in));
+  IRIS_CUDA_TRY(cudaStreamWaitEvent(s_run, hp->b_ready, 0));
+
   char* slot = heap->base + (size_t)out_slot * heap->bytes_per_rank;
   const int32_t epoch = heap->epoch + 1;
-  int blk = 0;
-  for (int r0 = 0; r0 < M || (r0 == 0 && blk == 0); r0 += rows_per_block, ++blk) {
-    const int rows = std::min(rows_per_block, M - r0);
+  for (int blk = 0; blk < blocks; ++blk) {
+    const int r0 = by_ranks ? 0 : blk * rows_per_block;
+    const int rows = by_ranks ? M : std::min(rows_per_block, M - r0);
     const size_t a_off = (size_t)r0 * K * 2, row_off = (size_t)r0 * N * 2;
-    if (rows > 0 && K > 0) IRIS_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(heap->stage_a) + a_off, static_cast<const char*>(A_host) + a_off, (size_t)rows * K * 2, cudaMemcpyHostToDevice, s_in));
+    if (by_ranks) {
+      if (shard_bytes) IRIS_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(dB[blk]), B_shards_host[blk], shard_bytes, cudaMemcpyHostToDevice, s_in));
+    } else if (rows > 0 && K > 0) {
+      IRIS_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(heap->stage_a) + a_off, static_cast<const char*>(A_host) + a_off, (size_t)rows * K * 2, cudaMemcpyHostToDevice, s_in));
+    }
     IRIS_CUDA_TRY(cudaEventRecord(hp->a_ready[blk], s_in));
     IRIS_CUDA_TRY(cudaStreamWaitEvent(s_run, hp->a_ready[blk], 0));
     iris_gemm_args a;
@@ -1604,6 +1627,7 @@ int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_h
     a.flag_off = flag_off + (uint64_t)(r0 / IRIS_TILE) * tiles_per_row * 4;
     a.lock_off = lock_off + (uint64_t)(r0 / IRIS_TILE) * tiles_per_row * 4;
     a.epoch = epoch;
+    if (by_ranks) { a.rank_first = blk; a.rank_count = 1; }
     // with a bias the consumer is part of the same call (inside the GEMM launch where the kernel supports it)
     a.consumer_bias = (bias_host && c_bytes) ? dbias : nullptr;
     a.consumer_out_off = out_off + row_off;
@@ -1612,8 +1636,14 @@ int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_h
     IRIS_CUDA_TRY(cudaEventRecord(hp->c_ready[blk], s_run));
     IRIS_CUDA_TRY(cudaStreamWaitEvent(s_out, hp->c_ready[blk], 0));
     if (rows > 0 && N > 0) {
-      IRIS_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(C_host) + row_off, slot + row_off, (size_t)rows * N * 2, cudaMemcpyDeviceToHost, s_out));
-      if (bias_host) IRIS_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(OUT_host) + row_off, slot + out_off + row_off, (size_t)rows * N * 2, cudaMemcpyDeviceToHost, s_out));
+      if (by_ranks) {   // rank blk's columns of every row
+        const size_t col_off = (size_t)blk * nl * 2, pitch = (size_t)N * 2;
+        IRIS_CUDA_TRY(cudaMemcpy2DAsync(static_cast<char*>(C_host) + col_off, pitch, slot + col_off, pitch, (size_t)nl * 2, (size_t)M, cudaMemcpyDeviceToHost, s_out));
+        if (bias_host) IRIS_CUDA_TRY(cudaMemcpy2DAsync(static_cast<char*>(OUT_host) + col_off, pitch, slot + out_off + col_off, pitch, (size_t)nl * 2, (size_t)M, cudaMemcpyDeviceToHost, s_out));
+      } else {
+        IRIS_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(C_host) + row_off, slot + row_off, (size_t)rows * N * 2, cudaMemcpyDeviceToHost, s_out));
+        if (bias_host) IRIS_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(OUT_host) + row_off, slot + out_off + row_off, (size_t)rows * N * 2, cudaMemcpyDeviceToHost, s_out));
+      }
     }
   }
   heap->epoch = epoch;
@@ -1686,6 +1716,7 @@ int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, co
   p.ptiles_m = p.tiles_m;
   p.ctiles_per_rank = (nl + bn - 1) / bn;
   p.ptiles_per_rank = (nl + IRIS_TILE - 1) / IRIS_TILE;
+  p.rank_first = 0; p.rank_count = world;
   p.total_ctiles = p.tiles_m * world * p.ctiles_per_rank;
   p.total_ptiles = p.tiles_m * world * p.ptiles_per_rank;
   p.kblocks = (K + BK - 1) / BK;

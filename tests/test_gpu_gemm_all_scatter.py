@@ -388,10 +388,13 @@ def test_producers_take_over_what_the_communication_ctas_cannot_finish():
 
 
 @pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
-def test_host_buffer_call_pipelined_over_row_blocks(mode):
-    """M = 1300 is cut into row blocks (512, 512, 276) that are copied, computed and copied back on three streams: the
-    host outputs and the whole heap image must be what the single call on device buffers gives (the oracle's)."""
-    W, M, nl, K, dtype = 4, 1300, 384, 136, "bf16"
+@pytest.mark.parametrize("W,M,nl,K", [(4, 1300, 384, 136),     # A is the smaller operand: one block per rank's shard
+                                      (2, 1300, 256, 136)],    # B is smaller: row blocks of A (512, 512, 276)
+                         ids=["by_ranks", "by_rows"])
+def test_host_buffer_call_pipelined_over_blocks(mode, W, M, nl, K):
+    """The host-buffer call copies, computes and copies back block by block on three streams: the host outputs and
+    the whole heap image must be what the single call on device buffers gives (the oracle's)."""
+    dtype = "bf16"
     N = W * nl
     A = inputs.matrix(61, inputs.STREAM_A, M, K, "ternary:0.5", dtype)
     Bs = [inputs.matrix(61, inputs.STREAM_B0 + r, nl, K, "smallint:2", dtype) for r in range(W)]
@@ -419,3 +422,58 @@ def test_host_buffer_call_pipelined_over_row_blocks(mode):
         c_ref = c_slot(img.mem, g, 0, c_off, M, N)
         assert np.array_equal(C_host, c_ref)
         assert np.array_equal(OUT_host, oracle.consume_bias_rows(c_ref, bias, dtype))
+
+
+RANK_RANGE_SHAPES = [
+    # W, M, N_local, K, kwargs
+    (4, 520, 512, 136, dict()),                              # CTA pairs
+    (8, 384, 256, 192, dict(max_ctas=20, comm_ctas=4)),
+    (3, 130, 136, 72, dict()),                               # single-CTA kernel, ragged everything
+    (4, 640, 512, 1024, dict(cta_pair=-1, stream_k=1, max_ctas=21)),
+]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("W,M,nl,K,kw", RANK_RANGE_SHAPES)
+def test_rank_range_one_call_touches_only_its_ranks(mode, W, M, nl, K, kw):
+    """rank_first / rank_count: one call computes and scatters only those ranks' column shards (what one rank of a real
+    job would run).  After a call for ranks [1, W-1) the other ranks' columns, flags and locks are still the sentinel;
+    after the remaining ranks' calls the heap image is the full call's (the oracle's)."""
+    N, dtype = W * nl, "bf16"
+    A = inputs.matrix(67, inputs.STREAM_A, M, K, "ternary:0.5", dtype)
+    Bs = [inputs.matrix(67, inputs.STREAM_B0 + r, nl, K, "smallint:2", dtype) for r in range(W)]
+    bias = inputs.vector(67, inputs.STREAM_BIAS, N, "smallint:3", dtype)
+    c_off, flag_off, lock_off, out_off, bpr = gemm_layout(M, N, W, with_out=True)
+    nt = oracle.num_tiles(M, N, W)
+    tm_n, ppr = -(-M // 128), -(-nl // 128)
+    c_full = oracle.gemm_block(A, Bs, dtype)
+    out_full = oracle.consume_bias_rows(c_full, bias, dtype)
+    with GpuHeap(W, bpr) as g:
+        img = g.image()
+        for s in range(W):
+            img.view(s, lock_off, nt * 4, np.int32)[:] = 0
+        iris.iris_flags_fill(g.h, lock_off, nt, 0)
+        dA, dbias = dev16(A), dev16(bias)
+
+        def call(first, count):
+            dB = [dev16(Bs[r]) if first <= r < first + count else None for r in range(W)]     # the others are not needed
+            iris.iris_gemm_all_scatter_ex(g.h, dA, dB, M, N, K, W, mode, iris.IRIS_BF16, c_off, flag_off, lock_off, 5, rank_first=first,
+                                          rank_count=count, consumer_bias=dbias, consumer_out_off=out_off, **kw)
+            iris.iris_status_check(g.h)
+            for s in range(W):                                   # the oracle's image, restricted to these ranks
+                cv = img.view(s, c_off, M * N * 2, np.uint16).reshape(M, N)
+                ov = img.view(s, out_off, M * N * 2, np.uint16).reshape(M, N)
+                fv = img.view(s, flag_off, nt * 4, np.int32).reshape(tm_n, W, ppr)
+                for r in range(first, first + count):
+                    cv[:, r * nl:(r + 1) * nl] = c_full[:, r * nl:(r + 1) * nl]
+                    ov[:, r * nl:(r + 1) * nl] = out_full[:, r * nl:(r + 1) * nl]
+                    fv[:, r, :] = 5
+            host = g.to_host()
+            assert np.array_equal(host, img.mem), (first, count, first_diff(host, img.mem))
+
+        call(1, W - 2)
+        call(0, 1)
+        call(W - 1, 1)
+        full, _ = expected_image(g, A, Bs, dtype, mode, epoch=5, c_full=c_full)
+        full.consume_bias(dtype, c_off, out_off, M, N, bias)
+        assert np.array_equal(img.mem, full.mem)                 # the three partial images add up to the oracle's full one
