@@ -300,6 +300,7 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
           ptx::bulk_commit_group();
           IRIS_TR(t2);
           ptx::bulk_wait_group<0>();  // stores performed: the buffer is free and the tile may be published
+          fence_proxy_async();        // async-proxy writes above -> the generic-proxy release of the flags below
 #ifdef IRIS_COMM_TRACE
           const uint64_t t3 = globaltimer_ns();
           tr[0] += 1; tr[1] += t1 - t0; tr[2] += t2 - t1; tr[3] += t3 - t2;
@@ -935,6 +936,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
           ptx::bulk_commit_group();
         }
         ptx::bulk_wait_group<0>();   // stores performed: the boxes are free and the tile may be published
+        fence_proxy_async();         // async-proxy writes above -> the generic-proxy release (flags or lock) after the barrier
       }
       if (p.mode != IRIS_MODE_BULK_SYNCHRONOUS) {
         asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
