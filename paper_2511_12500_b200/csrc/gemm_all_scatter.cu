@@ -1154,10 +1154,14 @@ struct PlanKey {
   uint64_t spin_timeout_ns;
 };
 struct Plan { GemmParams p; int bn, grid; bool pair, streamk; };
+// A few plans are kept (round-robin replacement): a step that alternates between calls -- one per rank shard in the
+// host-buffer pipeline, several schedules in a comparison -- finds each of them again on its next pass.
+constexpr int kPlanSlots = 16;
 static std::mutex g_plan_mutex;
-static Plan g_plan;
-static PlanKey g_plan_key;
-static bool g_plan_valid = false;
+static Plan g_plan[kPlanSlots];
+static PlanKey g_plan_key[kPlanSlots];
+static bool g_plan_valid[kPlanSlots] = {};
+static int g_plan_next = 0;
 
 static void make_key(PlanKey* k, const iris_gemm_args* a, const iris_heap* h) {
   std::memset(k, 0, sizeof(*k));   // padding too: keys are compared with memcmp
@@ -1266,7 +1270,7 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     if (a->K > 0 && (!a->B_shards[r] || (uint64_t)a->B_shards[r] % 16 != 0)) return fail(IRIS_ERR_ARG, "gemm_all_scatter: B_shards[%d] is NULL or not 16-byte aligned", r);
 
   // The launch plan (tile geometry, grid split, tensor maps) depends on everything but the epoch; timing loops
-  // call with the same arguments over and over, so the last plan is kept and re-used when nothing else changed.
+  // call with the same arguments over and over, so recent plans are kept and re-used when nothing else changed.
   GemmParams p;
   int bn = 0, grid = 0;
   bool pair = false, streamk = false;
@@ -1275,9 +1279,11 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   bool hit = false;
   {
     std::lock_guard<std::mutex> lock(g_plan_mutex);
-    if (g_plan_valid && std::memcmp(&key, &g_plan_key, sizeof(key)) == 0) {
-      p = g_plan.p; bn = g_plan.bn; grid = g_plan.grid; pair = g_plan.pair; streamk = g_plan.streamk;
-      hit = true;
+    for (int i = 0; i < kPlanSlots && !hit; ++i) {
+      if (g_plan_valid[i] && std::memcmp(&key, &g_plan_key[i], sizeof(key)) == 0) {
+        p = g_plan[i].p; bn = g_plan[i].bn; grid = g_plan[i].grid; pair = g_plan[i].pair; streamk = g_plan[i].streamk;
+        hit = true;
+      }
     }
   }
   auto build = [&]() -> int {
@@ -1440,9 +1446,11 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     const int brc = build();
     if (brc != IRIS_OK) return brc;
     std::lock_guard<std::mutex> lock(g_plan_mutex);
-    g_plan.p = p; g_plan.bn = bn; g_plan.grid = grid; g_plan.pair = pair; g_plan.streamk = streamk;
-    g_plan_key = key;
-    g_plan_valid = true;
+    const int i = g_plan_next;
+    g_plan_next = (g_plan_next + 1) % kPlanSlots;
+    g_plan[i].p = p; g_plan[i].bn = bn; g_plan[i].grid = grid; g_plan[i].pair = pair; g_plan[i].streamk = streamk;
+    g_plan_key[i] = key;
+    g_plan_valid[i] = true;
   }
   p.epoch = a->epoch;
 
