@@ -22,8 +22,20 @@ def _nvcc() -> str:
     return "nvcc"
 
 
+STAMP = os.path.join(PKG, "lib", "build_flags.txt")
+
+
+def _flags_line() -> str:
+    return " ".join(NVCC_FLAGS + os.environ.get("IRIS_EXTRA_NVCC_FLAGS", "").split())
+
+
 def _stale() -> bool:
     if not os.path.exists(LIB):
+        return True
+    try:
+        if open(STAMP).read() != _flags_line():   # built with other flags (e.g. a debug macro): not this build
+            return True
+    except OSError:
         return True
     t = os.path.getmtime(LIB)
     deps = [os.path.join(CSRC, f) for f in SOURCES + HEADERS] + [os.path.join(ROOT, "include", "iris_b200.h"), __file__]
@@ -59,6 +71,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     tmp = LIB + f".{os.getpid()}.tmp"
     subprocess.check_call([_nvcc(), "-shared", "-o", tmp, *objs, "-cudart", "static"])
     os.replace(tmp, LIB)
+    with open(STAMP, "w") as f:
+        f.write(_flags_line())
     return LIB
 
 
