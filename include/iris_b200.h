@@ -249,6 +249,11 @@ typedef struct iris_gemm_args {
                                   B_shards entries outside the range are not read; tiles, flags and
                                   locks of other ranks are not touched; a consumer that is part of
                                   the call covers the same ranks                                  */
+  int pace_stores;             /* CTA-pair kernel: 0 = the epilogue thread sends a tile's store boxes
+                                  out one by one, spread over three quarters of the time the CTA takes
+                                  per tile, because a burst of W copies holds up the operand loads of
+                                  the tile being multiplied meanwhile (same queue out of the SM);
+                                  -1 = all at once                                                */
   const void* consumer_bias;   /* not NULL: also run the flag-gated consumer OUT = C + bias (see
                                   iris_consume_bias) as part of this call: inside the same launch,
                                   as extra warps that acquire each tile's flag while the GEMM is

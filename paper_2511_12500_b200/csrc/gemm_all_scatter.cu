@@ -92,6 +92,7 @@ struct alignas(64) GemmParams {
   int32_t* backlog;     // publication tiles handed over and not yet published ([0]), tiles kept by that rule ([1])
   uint32_t t_pt_ns;     // estimate: time a communication warp needs for one publication tile, its CTA's port shared by all warps
   uint32_t t_tile_ns;   // estimate: main-loop time of one compute tile
+  int pace_stores;      // pair kernel: 1 = the epilogue spreads a tile's box stores over most of the next tile's main loop
   int raster_group;
   int mode;
   int32_t epoch;
@@ -861,6 +862,8 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
     int acc = 0, fj = 0, fslot = 0;
     uint32_t acc_phase = 0, fph = 0;
     const uint32_t tmem_base = ctrl->tmem_base;
+    uint64_t prev_issue = 0;               // thread 0: when the previous tile's stores started
+    uint32_t period_ns = p.t_tile_ns;      // thread 0: time between two tiles of this CTA (estimate, then measured)
     for (;;) {
       const int tile = feed_take(fj, fph, fslot);
       __syncwarp();
@@ -925,13 +928,33 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         ctrl->keep_tile = seq ? 1 : 0;
         // One thread stores the boxes with TMA: whole 128-byte lines, clipped by the maps at row M and column
         // N_local, to the owner's slot or (Listing 4: for remote_rank in range(world_size): iris.store(...)) to all.
+        // Stores and operand loads leave the SM through one queue: a burst of W x 4 boxes (512 KB, 9 us of the
+        // port) holds up the loads of the tile that is being multiplied meanwhile for longer than the stage ring
+        // covers.  So the boxes go out one at a time, spread over three quarters of the time this CTA takes per
+        // tile (measured from the previous tile; nothing is left to protect in the last wave, which goes at once).
         if (tm < p.ptiles_m) {
+          const uint64_t t0 = globaltimer_ns();
+          if (prev_issue != 0) period_ns = (uint32_t)min((uint64_t)(4u * p.t_tile_ns + 1000u), t0 - prev_issue);
+          prev_issue = t0;
+          int boxes = 0;
+#pragma unroll
+          for (int b = 0; b < kPairBN / 64; ++b) boxes += col_in_shard + 64 * b < p.n_local ? 1 : 0;
+          const bool last_wave = tile >= p.total_ctiles - (p.gemm_ctas >> 1);
+          // (a tile that is handed over goes at once: the communication CTAs are waiting for it)
+          const bool hand_over = !seq && p.mode == IRIS_MODE_WORKGROUP_SPECIALIZED;
+          const uint32_t gap_ns = (p.pace_stores && !last_wave && !hand_over) ? (period_ns / 4u * 3u) / (uint32_t)(boxes * (seq ? W : 1)) : 0u;
+          uint64_t due = t0;
           for (int s = 0; s < W; ++s) {
             if (!seq && s != tc.rank) continue;
 #pragma unroll
             for (int b = 0; b < kPairBN / 64; ++b)
-              if (col_in_shard + 64 * b < p.n_local)
+              if (col_in_shard + 64 * b < p.n_local) {
+                if (gap_ns) {
+                  while (globaltimer_ns() < due) __nanosleep(64);
+                  due += gap_ns;
+                }
                 ptx::tma_store_3d(&p.tmCs[s], col_in_shard + 64 * b, tm * BM, tc.rank, stg + (uint32_t)(b * kStoreBoxBytes));
+              }
           }
           ptx::bulk_commit_group();
         }
@@ -1150,7 +1173,7 @@ struct PlanKey {
   const void* A; const void* B[IRIS_MAX_WORLD];
   int M, N, K, world, mode, dtype;
   uint64_t c_off, flag_off, lock_off;
-  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail, fused_consumer, rank_first, rank_count;
+  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail, fused_consumer, rank_first, rank_count, pace_stores;
   uint64_t spin_timeout_ns;
 };
 struct Plan { GemmParams p; int bn, grid; bool pair, streamk; };
@@ -1173,7 +1196,7 @@ static void make_key(PlanKey* k, const iris_gemm_args* a, const iris_heap* h) {
   k->c_off = a->c_off; k->flag_off = a->flag_off; k->lock_off = a->lock_off;
   k->comm_ctas = a->comm_ctas; k->max_ctas = a->max_ctas; k->raster_group = a->raster_group; k->block_n = a->block_n;
   k->cta_pair = a->cta_pair; k->static_schedule = a->static_schedule; k->stream_k = a->stream_k; k->wg_tail = a->wg_tail;
-  k->rank_first = a->rank_first; k->rank_count = a->rank_count;
+  k->rank_first = a->rank_first; k->rank_count = a->rank_count; k->pace_stores = a->pace_stores;
   k->fused_consumer = a->consumer_bias != nullptr;   // the split between producers and communicators depends on it
   k->spin_timeout_ns = a->spin_timeout_ns;
 }
@@ -1239,6 +1262,7 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   if (a->c_off % 256 != 0 || a->flag_off % 4 != 0 || a->lock_off % 4 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: misaligned heap offsets");
   if (a->comm_ctas < 0 || a->max_ctas < 0 || a->raster_group < 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: negative tuning parameter");
   if (a->cta_pair < -1 || a->cta_pair > 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: cta_pair must be -1, 0 or 1");
+  if (a->pace_stores < -1 || a->pace_stores > 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: pace_stores must be 0 or -1");
   if (a->wg_tail < -1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: wg_tail must be -1, 0 or a tile count");
   if (a->stream_k < -1 || a->stream_k > 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: stream_k must be -1, 0 or 1");
   if (a->rank_first < 0 || a->rank_count < 0 || a->rank_first + a->rank_count > W || (a->rank_count == 0 && a->rank_first != 0))
@@ -1393,6 +1417,8 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     // busy at the end of the kernel: the producers write those tiles to all W slots and publish them, as in
     // fused_sequential mode.  wg_tail: -1 = never (Listing 5 for every tile), n > 0 = the last n compute tiles.
     p.takeover = 0;
+    p.t_tile_ns = (uint32_t)std::min<int64_t>((int64_t)p.kblocks * 260, 1 << 28);   // 512 tensor cycles per k-step at full clocks
+    p.pace_stores = pair && a->pace_stores >= 0 ? 1 : 0;
     if (a->mode == IRIS_MODE_FUSED_SEQUENTIAL) p.seq_from = 0;
     else if (!wg || a->wg_tail < 0) p.seq_from = INT_MAX;
     else {
@@ -1404,7 +1430,6 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
       if (pair && a->wg_tail == 0) {
         p.takeover = 1;
         p.t_pt_ns = (uint32_t)((uint64_t)kCommWarps * kTileBytes * (W - 1) / 45);   // 45 GB/s: what a communication SM sustains
-        p.t_tile_ns = (uint32_t)std::min<int64_t>((int64_t)p.kblocks * 260, 1 << 30);   // at full clocks: errs towards keeping
       }
     }
 
