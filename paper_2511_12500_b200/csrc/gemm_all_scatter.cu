@@ -63,7 +63,10 @@ struct alignas(64) GemmParams {
   CUtensorMap tmA;                    // A [M, K], box 64 x 128, 128B swizzle
   CUtensorMap tmB[IRIS_MAX_WORLD];    // B_r [N_local, K], box 64 x BN, 128B swizzle
   CUtensorMap tmC[IRIS_MAX_WORLD];    // C of slot s viewed as [W][M][N_local], box 128 x 128 x 1, no swizzle
-  CUtensorMap tmCs[IRIS_MAX_WORLD];   // the same view, box 64 x 128 x 1, 128B swizzle: the pair kernel's epilogue stores
+  CUtensorMap tmC4;                   // C of all slots as one tensor [slot][rank][M][N_local] (slots equally spaced: every heap
+                                      // handle), box 128 x 128 x 1 x 1, no swizzle: the communication warps' copies
+  CUtensorMap tmC4s;                  // the same tensor, box 64 x 128 x 1 x 1, 128B swizzle: the pair kernel's epilogue stores
+  int one_map;                        // 1 = tmC4 / tmC4s are valid; 0 = slots at arbitrary addresses, per-slot maps tmC[]
   HeapTable tab;
   uint64_t c_off, flag_off, lock_off;
   uint64_t timeout_ns;
@@ -291,13 +294,17 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
       if (lane == 0) {
         fence_proxy_async();  // producers' generic-proxy stores (acquired above) -> our async-proxy read
         ptx::mbar_arrive_expect_tx(bar, kTileBytes);
-        ptx::tma_load_3d(buf, &p.tmC[rrank], pj * IRIS_TILE, tm * IRIS_TILE, rrank, bar);
+        if (p.one_map) ptx::tma_load_4d(buf, &p.tmC4, pj * IRIS_TILE, tm * IRIS_TILE, rrank, rrank, bar);
+        else ptx::tma_load_3d(buf, &p.tmC[rrank], pj * IRIS_TILE, tm * IRIS_TILE, rrank, bar);
         if (!mbar_wait(bar, bar_phase, p, ctrl, rt)) {
           fail = true;
         } else {
           IRIS_TR(t1);
-          for (int s = 0; s < W; ++s)
-            if (s != rrank) ptx::tma_store_3d(&p.tmC[s], pj * IRIS_TILE, tm * IRIS_TILE, rrank, buf);
+          for (int s = 0; s < W; ++s) {
+            if (s == rrank) continue;
+            if (p.one_map) ptx::tma_store_4d(&p.tmC4, pj * IRIS_TILE, tm * IRIS_TILE, rrank, s, buf);
+            else ptx::tma_store_3d(&p.tmC[s], pj * IRIS_TILE, tm * IRIS_TILE, rrank, buf);
+          }
           ptx::bulk_commit_group();
           IRIS_TR(t2);
           ptx::bulk_wait_group<0>();  // stores performed: the buffer is free and the tile may be published
@@ -399,8 +406,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
       ptx::prefetch_tensormap(&p.tmA);
       for (int r = p.rank_first; r < p.rank_first + p.rank_count; ++r) ptx::prefetch_tensormap(&p.tmB[r]);
     }
-    if (is_comm)
-      for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmC[r]);
+    if (is_comm) {
+      if (p.one_map) ptx::prefetch_tensormap(&p.tmC4);
+      else for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmC[r]);
+    }
   }
   if (warp == 1 && !is_comm) {
     ptx::tmem_alloc(ptx::smem_u32(&ctrl->tmem_base), Cfg::kTmemCols);
@@ -745,10 +754,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
       ptx::prefetch_tensormap(&p.tmA);
       for (int r = p.rank_first; r < p.rank_first + p.rank_count; ++r) ptx::prefetch_tensormap(&p.tmB[r]);
     }
-    if (is_comm)
-      for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmC[r]);
-    else
-      for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmCs[r]);
+    ptx::prefetch_tensormap(is_comm ? &p.tmC4 : &p.tmC4s);
   }
   if (warp == 1 && !is_comm) {
     ptx::tmem_alloc_pair(ptx::smem_u32(&ctrl->tmem_base), 2 * kPairBN);
@@ -953,7 +959,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
                   while (globaltimer_ns() < due) __nanosleep(64);
                   due += gap_ns;
                 }
-                ptx::tma_store_3d(&p.tmCs[s], col_in_shard + 64 * b, tm * BM, tc.rank, stg + (uint32_t)(b * kStoreBoxBytes));
+                ptx::tma_store_4d(&p.tmC4s, col_in_shard + 64 * b, tm * BM, tc.rank, s, stg + (uint32_t)(b * kStoreBoxBytes));
               }
           }
           ptx::bulk_commit_group();
@@ -1065,7 +1071,7 @@ static int make_map(CUtensorMap* m, int dtype, int rank, void* base, const cuuin
                     CUtensorMapSwizzle swz, const char* what) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return fail(IRIS_ERR_CUDA, "cuTensorMapEncodeTiled entry point not available");
-  const cuuint32_t estr[3] = {1, 1, 1};
+  const cuuint32_t estr[5] = {1, 1, 1, 1, 1};
   CUresult r = fn(m, dtype == IRIS_BF16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, (cuuint32_t)rank, base, dims, strides, box,
                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(IRIS_ERR_CUDA, "cuTensorMapEncodeTiled(%s) failed with CUresult %d", what, (int)r);
@@ -1447,21 +1453,18 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
         if (rc != IRIS_OK) return rc;
       }
     }
-    if (pair) {
-      for (int s = 0; s < W; ++s) {
-        const cuuint64_t dimsC[3] = {(cuuint64_t)nl, (cuuint64_t)a->M, (cuuint64_t)W};
-        const cuuint64_t strC[2] = {(cuuint64_t)a->N * 2, (cuuint64_t)nl * 2};
-        const cuuint32_t boxC[3] = {64, BM, 1};
-        int rc = make_map(&p.tmCs[s], a->dtype, 3, h->base + (size_t)s * bpr + a->c_off, dimsC, strC, boxC, CU_TENSOR_MAP_SWIZZLE_128B, "C (epilogue stores)");
+    {
+      // C of every slot as one 4-D tensor [slot][rank][row][column]: the slots of a heap handle are bytes_per_rank apart.
+      const cuuint64_t dims4[4] = {(cuuint64_t)nl, (cuuint64_t)a->M, (cuuint64_t)W, (cuuint64_t)W};
+      const cuuint64_t str4[3] = {(cuuint64_t)a->N * 2, (cuuint64_t)nl * 2, (cuuint64_t)bpr};
+      const cuuint32_t box4[4] = {IRIS_TILE, IRIS_TILE, 1, 1}, box4s[4] = {64, BM, 1, 1};
+      p.one_map = 1;
+      if (wg) {
+        int rc = make_map(&p.tmC4, a->dtype, 4, h->base + a->c_off, dims4, str4, box4, CU_TENSOR_MAP_SWIZZLE_NONE, "C (all slots)");
         if (rc != IRIS_OK) return rc;
       }
-    }
-    if (wg) {
-      for (int s = 0; s < W; ++s) {
-        const cuuint64_t dimsC[3] = {(cuuint64_t)nl, (cuuint64_t)a->M, (cuuint64_t)W};
-        const cuuint64_t strC[2] = {(cuuint64_t)a->N * 2, (cuuint64_t)nl * 2};
-        const cuuint32_t boxC[3] = {IRIS_TILE, IRIS_TILE, 1};
-        int rc = make_map(&p.tmC[s], a->dtype, 3, h->base + (size_t)s * bpr + a->c_off, dimsC, strC, boxC, CU_TENSOR_MAP_SWIZZLE_NONE, "C");
+      if (pair) {
+        int rc = make_map(&p.tmC4s, a->dtype, 4, h->base + a->c_off, dims4, str4, box4s, CU_TENSOR_MAP_SWIZZLE_128B, "C (all slots, epilogue stores)");
         if (rc != IRIS_OK) return rc;
       }
     }

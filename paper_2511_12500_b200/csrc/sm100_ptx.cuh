@@ -63,6 +63,18 @@ __device__ __forceinline__ void tma_store_3d(const void* tmap, int x, int y, int
                ::"l"(tmap), "r"(x), "r"(y), "r"(z), "r"(src)
                : "memory");
 }
+// 4-D forms: C of every slot as one tensor [slot][rank][row][column], so that a kernel that writes all W slots
+// works with one descriptor instead of W.
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const void* tmap, int x, int y, int z, int w, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+               ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tma_store_4d(const void* tmap, int x, int y, int z, int w, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3, %4}], [%5];"
+               ::"l"(tmap), "r"(x), "r"(y), "r"(z), "r"(w), "r"(src)
+               : "memory");
+}
 __device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // Waits until at most N of this thread's bulk groups are still pending; completion here means the
 // global writes have been performed (the non-.read form), not merely that shared memory was read.
