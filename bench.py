@@ -451,11 +451,33 @@ def run_ours(args):
                                       "sample": f"{len(strips)} strips (128 rows x one rank's {nl}-column shard, K={K}) of {args.workload}, "
                                                 f"{fl / flops:.4f} of one step's flops, fp64 accumulation",
                                       "extrapolated_full_step_seconds": flops / (fl / secs)}
+            if args.sweep != "none":
+                result["cpu_baseline"]["all_store"] = oracle_all_store_sample()
         print(json.dumps(result))
     iris.iris_heap_destroy(h)
     if dist_on:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def oracle_all_store_sample(S=4 << 20, W=8):
+    """The oracle's all-store (its copy loops and flag updates on a host image of the heap) at one message size of
+    the sweep, timed as it stands; GB/s counted like the GPU sweep (W*S read + W*W*S written)."""
+    import oracle
+    tile = 32768
+    T = S // tile
+    payload_off, recv_off = 0, align(S)
+    flag_off = recv_off + align(W * S)
+    bpr = align(flag_off + W * T * 4)
+    img = oracle.HeapImage(W, bpr, fill=0)
+    for r in range(W):
+        img.view(r, payload_off, S)[:] = (r + 1)
+    img.all_store(payload_off, recv_off, flag_off, S, tile, 1)          # first touch of the image
+    t0 = time.perf_counter()
+    img.all_store(payload_off, recv_off, flag_off, S, tile, 2)
+    secs = time.perf_counter() - t0
+    moved = float(W * S + W * W * S)
+    return {"S": S, "seconds": secs, "gbs": moved / secs / 1e9, "kind": "oracle"}
 
 
 def all_store_sweep(iris, pk, kind, pull=0):
