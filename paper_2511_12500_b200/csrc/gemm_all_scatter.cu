@@ -1154,8 +1154,9 @@ static int auto_comm_ctas(int M, int N, int K, int W, int sms) {
 // has to balance two things -- every communication pair is a producer pair less (and can add a wave), every byte the
 // communicators do not take is stored through the producers' own ports instead.  Model per candidate count c:
 // waves = ceil(tiles / pairs), t = waves * t_tile + (remote bytes - what c SMs move in that time) / (producer SMs' ports);
-// the smallest t among the counts that leave at least three quarters of the scatter to the communication CTAs
-// (the schedule stays what its name says; measured differences between the candidates are a few per cent).  Constants: 45 GB/s sustained per communication SM (57 at best), 57 GB/s per
+// the smallest t among the counts that leave at least half of the scatter to the communication CTAs (the schedule
+// stays what its name says; measured differences between the candidates are a few per cent).  Kept bytes are paced
+// by the producers' epilogues and cost about two thirds of their raw port time.  Constants: 45 GB/s sustained per communication SM (57 at best), 57 GB/s per
 // producer port, 270 ns per k-step of a pair tile.
 static int auto_comm_ctas_pair(int total_ctiles, int kblocks, double remote_bytes, int grid) {
   int best_c = 2;
@@ -1165,9 +1166,9 @@ static int auto_comm_ctas_pair(int total_ctiles, int kblocks, double remote_byte
     const double waves = std::ceil((double)total_ctiles / pairs);
     const double t_gemm = waves * (kblocks * 0.27e-6 + 2e-6);
     const double cap = c * 45e9 * t_gemm;
-    if (cap < remote_bytes * 0.75 && c < std::min(grid - 2, 64) - 1) continue;
+    if (cap < remote_bytes * 0.5 && c < std::min(grid - 2, 64) - 1) continue;
     const double kept = std::max(0.0, remote_bytes - cap);
-    const double t = t_gemm + kept / (2.0 * pairs * 57e9);
+    const double t = t_gemm + 0.67 * kept / (2.0 * pairs * 57e9);
     if (t < best_t * 0.999) { best_t = t; best_c = c; }
   }
   return best_c;
