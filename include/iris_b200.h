@@ -212,8 +212,11 @@ typedef struct iris_gemm_args {
   int dtype;                   /* IRIS_F16 or IRIS_BF16                                          */
   uint64_t c_off, flag_off, lock_off; /* offsets inside a slot; c_off % 256 == 0, others % 4     */
   int32_t epoch;               /* value written to the flags; callers use 1, 2, 3, ...           */
-  int comm_ctas;               /* workgroup-specialised: communication CTAs (0 = chosen from the
-                                  ratio of scatter bytes to GEMM time; 16 at the largest config) */
+  int comm_ctas;               /* workgroup-specialised: communication CTAs (0 = chosen by the
+                                  library: from a small model of waves and store-path time when
+                                  the producers may take tiles over (wg_tail = 0, CTA-pair kernel:
+                                  10 at the largest config), from the ratio of scatter bytes to
+                                  GEMM time otherwise (16 there))                                */
   int max_ctas;                /* cap on the persistent grid (0 = one CTA per SM)                */
   int raster_group;            /* tile rows per raster group for L2 reuse (0 = 2048 rows)        */
   int block_n;                 /* compute-tile width: 0 = auto, 128 or 256                       */
