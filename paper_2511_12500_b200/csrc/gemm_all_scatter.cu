@@ -720,6 +720,14 @@ __device__ void consumer_warp(const GemmParams& p, CtrlBlock* ctrl, int cwarp, i
 //   tmem_empty[a]  leader only; 8 arrivals = 4 epilogue warps x 2 CTAs (the peer's arrive remotely)
 // ------------------------------------------------------------------------------------------------
 constexpr int kPairBN = 256;
+// Columns the pair's MMA computes for tile column jn of a shard: the full 256, or -- last tile of a ragged shard --
+// what is left, rounded up to 32 (one epilogue chunk; the instruction's N has to be a multiple of 16).  A narrower
+// instruction takes proportionally fewer tensor cycles; the rows of B beyond the shard that it reads are zero-filled
+// by the load and the columns they produce are clipped by the stores.
+__device__ __forceinline__ int pair_tile_cols(const GemmParams& p, int jn) {
+  const int left = p.n_local - jn * kPairBN;
+  return left >= kPairBN ? kPairBN : ((left + 31) & ~31);
+}
 constexpr int kPairStageBytes = 2 * BM * BK * 2;            // 32 KB: A slice + B half
 constexpr int kPairStages = 5;
 constexpr int kStoreBoxBytes = BM * 64 * 2;                 // 16 KB: 128 rows x 64 columns, one TMA store box
@@ -812,6 +820,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         }
         if (tile < 0) break;
         const TileCoord tc = decode_ctile(tile, p);
+        const int ncols = pair_tile_cols(p, tc.jn);   // this CTA keeps rows [cta_rank * ncols / 2, ...) of the B tile
         bool ok = true;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!mbar_wait(ptx::smem_u32(&ctrl->empty[stage]), phase ^ 1, p, ctrl, tile)) { ok = false; break; }
@@ -820,7 +829,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
           const uint32_t full_leader = ptx::mapa(full_local, 0);
           const uint32_t sa = ptx::smem_u32(payload + stage * kPairStageBytes);
           ptx::tma_load_2d_pair(sa, &p.tmA, kb * BK, tc.tm * 2 * BM + cta_rank * BM, full_leader);
-          ptx::tma_load_2d_pair(sa + BM * BK * 2, &p.tmB[tc.rank], kb * BK, tc.jn * kPairBN + cta_rank * (kPairBN / 2), full_leader);
+          ptx::tma_load_2d_pair(sa + BM * BK * 2, &p.tmB[tc.rank], kb * BK, tc.jn * kPairBN + cta_rank * (ncols / 2), full_leader);
           if (++stage == kPairStages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
@@ -829,7 +838,6 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
   } else if (warp == 1) {
     // ---------------- MMA issuer (leader CTA only) ----------------
     if (lane == 0 && leader) {
-      constexpr uint32_t idesc = ptx::idesc_f16(2 * BM, kPairBN, BF16 ? 1 : 0);
       const uint32_t tmem_base = ctrl->tmem_base;
       int stage = 0, acc = 0, fj = 0, fslot = 0;
       uint32_t phase = 0, acc_phase = 0, fph = 0;
@@ -843,6 +851,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         if (tile < 4096) { g_tile_trace[2 * tile] = globaltimer_ns(); unsigned sm; asm("mov.u32 %0, %%smid;" : "=r"(sm)); g_tile_trace[2 * tile + 1] = sm; }
 #endif
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kPairBN);
+        const uint32_t idesc = ptx::idesc_f16(2 * BM, pair_tile_cols(p, decode_ctile(tile, p).jn), BF16 ? 1 : 0);
         bool ok = true;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!mbar_wait(ptx::smem_u32(&ctrl->full[stage]), phase, p, ctrl, tile)) { ok = false; break; }
@@ -891,8 +900,9 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
       // 512 bytes per instruction spread over all banks.  (The previous tile's stores have been waited for
       // before the barrier at the top of this loop, so the boxes are free.)
       const uint32_t stg = ptx::smem_u32(payload + kPairStages * kPairStageBytes);
+      const int chunks = pair_tile_cols(p, tc.jn) / 32;   // 8, fewer for the narrow last tile of a ragged shard
 #pragma unroll 1
-      for (int ch = 0; ch < kPairBN / 32; ++ch) {
+      for (int ch = 0; ch < chunks; ++ch) {
         uint32_t v[32];
         ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kPairBN + ch * 32), v);
         ptx::tmem_wait_ld();
@@ -1329,14 +1339,11 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     }
     if (nl <= 128) bn = 128;
     // CTA pairs (256 x 256 tiles) need at least two tile rows.  A shard that is not a whole number of 256-column
-    // tiles is fine (TMA zero-fills the missing B rows, stores and flags are masked) but spends MMA work on the
-    // padding.  Measured on a 576-column shard (33 % padding) pairs still take 2.44 ms where 128-wide single-CTA
-    // tiles (11 % padding) take 3.26 ms: per padded flop the pair kernel is about 1.6x as fast, so pairs are the
-    // default unless their padding exceeds the narrow tiles' by more than 1.5x.
+    // tiles is fine: TMA zero-fills the missing B rows, stores and flags are masked, and the last tile's MMA is only
+    // as wide as what is left of the shard (rounded up to 32 columns), so the padding costs next to nothing.
     const bool pair_ok = a->M > BM && nl > BM && a->block_n != 128 && h->sm_count >= 4;
     if (a->cta_pair > 0 && !pair_ok) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: cta_pair needs M > 128, N/world > 128 and block_n != 128");
-    const bool pair_pays = (int64_t)((nl + 255) / 256) * 256 * 2 <= (int64_t)((nl + 127) / 128) * 128 * 3;
-    pair = pair_ok && (a->cta_pair > 0 || (a->cta_pair == 0 && pair_pays));
+    pair = pair_ok && a->cta_pair >= 0;
     int max_pairs = 0;
     if (pair) {
       const int rc = a->dtype == IRIS_BF16 ? launch_gemm_pair<true>(p, 0, nullptr, &max_pairs) : launch_gemm_pair<false>(p, 0, nullptr, &max_pairs);
