@@ -91,6 +91,8 @@ def test_random_shapes_exact_heap_image():
             kw["cta_pair"] = 1      # pairs even where the shard is ragged
         if rng.random() < 0.5:
             kw["wg_tail"] = int(rng.choice([-1, 1, 2, 5]))
+        if rng.random() < 0.3:
+            kw["pace_stores"] = -1
         if kw.get("cta_pair") == -1 and rng.random() < 0.6:
             kw["stream_k"] = 1
         dtype = "bf16" if case % 2 else "fp16"
