@@ -1398,6 +1398,14 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
         p.comm_ctas = 0;
         p.gemm_ctas = 2 * std::min(grid / 2, p.total_ctiles);
       }
+      // The fewest producer pairs that still finish in the same number of waves: on this power-capped part an SM
+      // that would only idle through the last, partly filled wave is better left out, the others then clock higher
+      // (W = 8, 1024 x 16384 x 16384: 256 tiles on 64 pairs instead of 74, fused_sequential 0.425 -> 0.398 ms).
+      if (p.total_ctiles > 0) {
+        const int units = p.gemm_ctas / 2;
+        const int waves = (p.total_ctiles + units - 1) / units;
+        p.gemm_ctas = 2 * ((p.total_ctiles + waves - 1) / waves);
+      }
     } else if (wg) {
       if (grid < 2) return fail(IRIS_ERR_ARG, "gemm_all_scatter: workgroup_specialized needs at least 2 CTAs");
       int comm = a->comm_ctas ? a->comm_ctas : auto_comm_ctas(a->M, nl * rank_count, a->K, W, grid);
