@@ -72,13 +72,17 @@ const char* iris_version(void);
 
 /* Create a heap of `world` slots of `bytes_per_rank` bytes each on the current CUDA device.
  * 1 <= world <= IRIS_MAX_WORLD; bytes_per_rank > 0 and a multiple of 256.  The library allocates
- * world * bytes_per_rank bytes of device memory (plus a 256-byte status block) and owns them.
+ * world * bytes_per_rank bytes of device memory (plus a 256-byte status block), clears them to zero
+ * (so flag and lock arrays placed anywhere in it start in their initial state) and owns them.
  * Returns NULL on failure (see iris_last_error). */
 iris_heap* iris_heap_create(int world, size_t bytes_per_rank);
 
 /* Same, with the status code returned and an optional caller-owned backing store:
  * external_base != NULL must be a 256-byte aligned device pointer to world * bytes_per_rank bytes
- * that outlives the heap (e.g. a torch tensor's storage); NULL = the library allocates. */
+ * that outlives the heap (e.g. a torch tensor's storage); NULL = the library allocates.  A caller-owned
+ * backing store is used as it is: before the first iris_gemm_all_scatter_ex on it the caller sets the lock array
+ * to 0 and the flag array below the first epoch (iris_flags_fill); gemm_all_scatter() and
+ * iris_gemm_all_scatter_host() choose their own layout and clear their flag and lock arrays themselves. */
 int iris_heap_create_ex(int world, size_t bytes_per_rank, void* external_base, iris_heap** out);
 
 /* Free the heap (and its memory if the library owns it).  Synchronises the device first. */
@@ -116,9 +120,9 @@ int iris_status_check(iris_heap* heap, void* stream, int32_t* detail);
 /* ------------------------------------------------------------------------------------------ */
 
 /* put: copy a 2-D region from from_rank's memory to to_rank's memory (local -> remote).
- * src and dst are device addresses valid in from_rank's slot, exactly as in Listings 3 and 5
- * (iris.put(C + offset, C + offset, cur_rank, remote_rank)): the region is read at src and
- * written at translate(dst, from_rank, to_rank).  rows x row_bytes bytes; consecutive rows are
+ * src and dst are device addresses valid in from_rank's slot, as in Listings 3 and 5 (where put
+ * receives the same local address for both, with the caller's and the remote rank): the region is
+ * read at src and written at translate(dst, from_rank, to_rank).  rows x row_bytes bytes; consecutive rows are
  * src_pitch / dst_pitch bytes apart (pitch >= row_bytes).  A 16-byte vector path is used when
  * both addresses, both pitches and row_bytes are multiples of 16, a byte path otherwise.
  * IRIS_ERR_RANGE if either region leaves its slot.  rows == 0 or row_bytes == 0: no-op. */
@@ -136,7 +140,7 @@ int iris_copy_tile(iris_heap* heap, const void* src, void* dst, size_t rows, siz
                    size_t dst_pitch, int cur_rank, int from_rank, int to_rank, void* stream);
 
 /* load / store (Table 3, value-based): like get / put, but the local side is a device buffer of the caller's
- * that need not lie in the heap (it stands in for the registers of the paper's tl.load / tl.store).
+ * that need not lie in the heap (it stands in for the registers the paper's value-based calls use).
  * load: read translate(src, from_rank, to_rank) -> out.   store: values -> translate(dst, from_rank, to_rank).
  * Only the heap-side region is range-checked. */
 int iris_load_tile(iris_heap* heap, const void* src, void* out, size_t rows, size_t row_bytes, size_t src_pitch,
@@ -153,6 +157,14 @@ int iris_atomic_add(iris_heap* heap, void* ptr, size_t count, size_t stride_byte
                     int32_t value, int sem, int scope, int32_t* old_out, void* stream);
 int iris_atomic_cas(iris_heap* heap, void* ptr, size_t count, size_t stride_bytes, int from_rank, int to_rank,
                     int32_t compare, int32_t value, int sem, int scope, int32_t* old_out, void* stream);
+
+/* The same two atomics on uint64 words (Table 3's atomic_add / atomic_cas with 64-bit operands; Section 3.3's
+ * sem x scope choice).  ptr and stride_bytes must be multiples of 8; the addition wraps modulo 2^64; old_out is
+ * a device pointer to count uint64 (or NULL). */
+int iris_atomic_add_u64(iris_heap* heap, void* ptr, size_t count, size_t stride_bytes, int from_rank, int to_rank,
+                        uint64_t value, int sem, int scope, uint64_t* old_out, void* stream);
+int iris_atomic_cas_u64(iris_heap* heap, void* ptr, size_t count, size_t stride_bytes, int from_rank, int to_rank,
+                        uint64_t compare, uint64_t value, int sem, int scope, uint64_t* old_out, void* stream);
 
 /* The remaining atomics (atomic_xchg / and / or / xor / min / max; IRIS_OP_ADD is accepted too), vector form
  * as iris_atomic_add: old_out receives the previous values. */
@@ -273,7 +285,9 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* args, void* stream);
 /* The short form named by the problem statement.  bf16; C at offset 0 of every slot, flags at
  * align256(M*N*2), locks right after the flags (align256); epoch = a per-heap counter that starts
  * at 1 and grows by one per call (iris_heap_epoch() returns the last value used); default stream.
- * The heap must have been created with bytes_per_rank >= iris_gemm_heap_bytes(M, N, world). */
+ * The heap must have been created with bytes_per_rank >= iris_gemm_heap_bytes(M, N, world).  On a heap's
+ * first such call, and whenever (M, N) differ from the previous short-form or host-buffer call on it, the
+ * flag and lock arrays of every slot are cleared on the stream before the launch. */
 int gemm_all_scatter(const void* A, const void* const* B_shards, iris_heap* heap, int M, int N, int K, int world,
                      int mode);
 size_t iris_gemm_heap_bytes(int M, int N, int world);
@@ -347,14 +361,18 @@ int iris_gemm_takeover_stats(const iris_heap* heap, int32_t out[2]);
  * are refused with IRIS_ERR_UNSUPPORTED and a message naming the limit; nothing is launched.
  *
  * The first call on a device looks up the device address of that array (with that device current)
- * and remembers it; make this first call outside any stream capture.  Every call clears the words
- * it is going to use (the array keeps the previous call's contents) on `stream`, launches on
- * `stream`, then WAITS for the stream and returns IRIS_OK or IRIS_ERR_TIMEOUT (a bounded device-side
- * wait ran out).  All calls share the one array: two calls whose GPU work overlaps (different
- * streams, different host threads) race on it and must be serialised by the caller.
+ * and remembers it (the per-device record is filled without a lock: concurrent first calls store
+ * the same value).  Every call clears the words it is going to use (the array keeps the previous
+ * call's contents) on `stream`, launches on `stream`, reads the status words back on `stream` and
+ * then WAITS for that stream -- no other stream is touched -- and returns IRIS_OK or
+ * IRIS_ERR_TIMEOUT (a bounded device-side wait ran out).  Because every call waits for its stream,
+ * no call may be made while that stream is being captured.  All calls share the one array: two
+ * calls whose GPU work overlaps (different streams, different host threads) race on it and must be
+ * serialised by the caller.
  * Other arguments, checks, layout and results are those of iris_gemm_all_scatter_ex in
- * IRIS_MODE_WORKGROUP_SPECIALIZED with single-CTA tiles (cta_pair = -1) and default tuning; the
- * results are bit-identical to that call's. */
+ * IRIS_MODE_WORKGROUP_SPECIALIZED with single-CTA tiles (cta_pair = -1) and default tuning: the
+ * launch plan (tile width, grid split, which tiles the producers scatter themselves) is built by
+ * the same code, and the results are bit-identical to that call's. */
 int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, const uint64_t* slot_bases,
                                   size_t bytes_per_rank, int M, int N, int K, int world, int dtype, uint64_t c_off,
                                   uint64_t flag_off, int32_t epoch, void* stream);

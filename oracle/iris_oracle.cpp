@@ -254,6 +254,34 @@ int orc_atomic_cas(uint8_t* image, int world, uint64_t bpr, uint64_t off, int64_
   return 0;
 }
 
+// The same two operations on uint64 words (Table 3's atomics, 64-bit operands): the addition wraps modulo 2^64,
+// the compare-and-swap writes iff the word equals cmp; old_out[i] receives the value before the operation.
+int orc_atomic_add_u64(uint8_t* image, int world, uint64_t bpr, uint64_t off, int64_t count, int64_t stride,
+                       int to_rank, uint64_t val, uint64_t* old_out) {
+  if (bad_rank(to_rank, world)) return -1;
+  if (count > 0 && off + (uint64_t)(count - 1) * stride + 8 > bpr) return -2;
+  for (int64_t i = 0; i < count; ++i) {
+    uint64_t* p = (uint64_t*)(slot(image, bpr, to_rank) + off + i * stride);
+    const uint64_t old = *p;
+    *p = old + val;
+    if (old_out) old_out[i] = old;
+  }
+  return 0;
+}
+
+int orc_atomic_cas_u64(uint8_t* image, int world, uint64_t bpr, uint64_t off, int64_t count, int64_t stride,
+                       int to_rank, uint64_t cmp, uint64_t val, uint64_t* old_out) {
+  if (bad_rank(to_rank, world)) return -1;
+  if (count > 0 && off + (uint64_t)(count - 1) * stride + 8 > bpr) return -2;
+  for (int64_t i = 0; i < count; ++i) {
+    uint64_t* p = (uint64_t*)(slot(image, bpr, to_rank) + off + i * stride);
+    const uint64_t old = *p;
+    if (old == cmp) *p = val;
+    if (old_out) old_out[i] = old;
+  }
+  return 0;
+}
+
 // Consumer: in every slot, OUT = C + bias (bias broadcast over rows), added in fp32 and rounded
 // once to the 16-bit type.  The sum of two 16-bit floats rounded to fp32 and then to 16 bits is
 // computed here as written: float add, then the codec.

@@ -60,6 +60,8 @@ def lib() -> C.CDLL:
                 f.argtypes = [u8p, C.c_int, u64, u64, u64, i64, i64, i64, i64, C.c_int, C.c_int]
             L.orc_atomic_add.argtypes = [u8p, C.c_int, u64, u64, i64, i64, C.c_int, i32, C.POINTER(i32)]
             L.orc_atomic_cas.argtypes = [u8p, C.c_int, u64, u64, i64, i64, C.c_int, i32, i32, C.POINTER(i32)]
+            L.orc_atomic_add_u64.argtypes = [u8p, C.c_int, u64, u64, i64, i64, C.c_int, u64, C.POINTER(u64)]
+            L.orc_atomic_cas_u64.argtypes = [u8p, C.c_int, u64, u64, i64, i64, C.c_int, u64, u64, C.POINTER(u64)]
             L.orc_atomic_rmw.argtypes = [u8p, C.c_int, u64, C.c_int, u64, i64, i64, C.c_int, i32, C.POINTER(i32)]
             L.orc_copy.argtypes = [u8p, C.c_int, u64, u64, u64, i64, i64, i64, i64, C.c_int, C.c_int]
             L.orc_consume_bias.argtypes = [u8p, C.c_int, u64, C.c_int, u64, u64, i64, i64, u16p]
@@ -179,6 +181,18 @@ class HeapImage:
         old = np.empty(count, dtype=np.int32)
         _check(lib().orc_atomic_cas(_u8p(self.mem), self.world, self.bpr, off, count, stride, to_rank, cmp, val,
                                     old.ctypes.data_as(C.POINTER(C.c_int32))), "atomic_cas")
+        return old
+
+    def atomic_add_u64(self, off, count, stride, to_rank, val) -> np.ndarray:
+        old = np.empty(count, dtype=np.uint64)
+        _check(lib().orc_atomic_add_u64(_u8p(self.mem), self.world, self.bpr, off, count, stride, to_rank, val,
+                                        old.ctypes.data_as(C.POINTER(C.c_uint64))), "atomic_add_u64")
+        return old
+
+    def atomic_cas_u64(self, off, count, stride, to_rank, cmp, val) -> np.ndarray:
+        old = np.empty(count, dtype=np.uint64)
+        _check(lib().orc_atomic_cas_u64(_u8p(self.mem), self.world, self.bpr, off, count, stride, to_rank, cmp, val,
+                                        old.ctypes.data_as(C.POINTER(C.c_uint64))), "atomic_cas_u64")
         return old
 
     ATOMIC_OPS = {"add": 0, "xchg": 1, "and": 2, "or": 3, "xor": 4, "min": 5, "max": 6}

@@ -32,7 +32,7 @@ EXPORTS = [
     "iris_atomic_add_contended", "iris_atomic_cas_contended", "iris_flags_fill", "iris_all_store_bench",
     "iris_gemm_all_scatter_ex", "gemm_all_scatter", "iris_gemm_heap_bytes", "iris_heap_epoch", "iris_num_tiles",
     "iris_consume_bias", "iris_consume_bias_ranks", "iris_gemm_all_scatter_host", "iris_gemm_out_offset", "iris_gemm_takeover_stats",
-    "iris_gemm_all_scatter_noalloc", "iris_copy_tile", "iris_load_tile", "iris_store_tile", "iris_atomic_rmw",
+    "iris_gemm_all_scatter_noalloc", "iris_atomic_add_u64", "iris_atomic_cas_u64", "iris_copy_tile", "iris_load_tile", "iris_store_tile", "iris_atomic_rmw",
 ]
 
 
@@ -89,6 +89,8 @@ def lib() -> C.CDLL:
     L.iris_atomic_rmw.argtypes = [vp, ci, vp, sz, sz, ci, ci, i32, ci, ci, vp, vp]
     L.iris_atomic_add.argtypes = [vp, vp, sz, sz, ci, ci, i32, ci, ci, vp, vp]
     L.iris_atomic_cas.argtypes = [vp, vp, sz, sz, ci, ci, i32, i32, ci, ci, vp, vp]
+    L.iris_atomic_add_u64.argtypes = [vp, vp, sz, sz, ci, ci, u64, ci, ci, vp, vp]
+    L.iris_atomic_cas_u64.argtypes = [vp, vp, sz, sz, ci, ci, u64, u64, ci, ci, vp, vp]
     L.iris_atomic_add_contended.argtypes = [vp, vp, sz, ci, ci, i32, ci, ci, vp, vp]
     L.iris_atomic_cas_contended.argtypes = [vp, vp, sz, ci, ci, i32, i32, ci, ci, vp, vp]
     L.iris_flags_fill.argtypes = [vp, u64, sz, i32, vp]
@@ -236,6 +238,16 @@ def iris_atomic_add(heap, ptr, count, stride_bytes, from_rank, to_rank, value, s
 def iris_atomic_cas(heap, ptr, count, stride_bytes, from_rank, to_rank, compare, value, sem=IRIS_SEM_RELAXED,
                     scope=IRIS_SCOPE_GPU, old_out=None, stream=None):
     _ck(lib().iris_atomic_cas(heap, ptr, count, stride_bytes, from_rank, to_rank, compare, value, sem, scope, _ptr(old_out), _stream(stream)))
+
+
+def iris_atomic_add_u64(heap, ptr, count, stride_bytes, from_rank, to_rank, value, sem=IRIS_SEM_RELAXED,
+                        scope=IRIS_SCOPE_GPU, old_out=None, stream=None):
+    _ck(lib().iris_atomic_add_u64(heap, ptr, count, stride_bytes, from_rank, to_rank, value, sem, scope, _ptr(old_out), _stream(stream)))
+
+
+def iris_atomic_cas_u64(heap, ptr, count, stride_bytes, from_rank, to_rank, compare, value, sem=IRIS_SEM_RELAXED,
+                        scope=IRIS_SCOPE_GPU, old_out=None, stream=None):
+    _ck(lib().iris_atomic_cas_u64(heap, ptr, count, stride_bytes, from_rank, to_rank, compare, value, sem, scope, _ptr(old_out), _stream(stream)))
 
 
 def iris_atomic_add_contended(heap, ptr, threads, from_rank, to_rank, value, sem=IRIS_SEM_RELAXED, scope=IRIS_SCOPE_GPU,

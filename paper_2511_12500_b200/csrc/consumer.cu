@@ -1,7 +1,7 @@
 // Flag-gated consumer: waits (acquire, gpu scope) for a publication tile's ready flag in a slot, then
 // reads that tile of C and writes OUT = C + bias.  This is the consumer side of the paper's
-// producer-consumer handshake (Section 4.1): it "spins on these atomic locks (with acquire
-// semantics)" and touches the data only afterwards.  HBM-bound: 16-byte coalesced accesses, one warp
+// producer-consumer handshake (Section 4.1): poll the tile's flag with acquire-ordered loads and touch
+// the data only once it has been seen set.  HBM-bound: 16-byte coalesced accesses, one warp
 // instruction covers 512 contiguous bytes of a row, several CTAs per SM for latency hiding.
 #include "iris_device.cuh"
 

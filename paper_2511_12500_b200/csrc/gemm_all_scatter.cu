@@ -202,15 +202,6 @@ __device__ __forceinline__ int32_t* lock_addr(const GemmParams& p, int rank, int
 //            then waits until the stores have been performed
 //   publish  lanes 0..W-1 write the tile's ready flag in slot `lane` with release semantics
 // ------------------------------------------------------------------------------------------------
-#ifdef IRIS_COMM_TRACE
-// Debug build only: per communicator warp {tiles, ns in: load, store issue, store wait, publish, idle poll, claim}.
-__device__ unsigned long long g_comm_trace[64 * 6 * 8];
-__device__ unsigned long long g_tile_trace[2 * 4096];  // {start ns, smid} per compute tile
-#define IRIS_TR(var) const uint64_t var = globaltimer_ns()
-#else
-#define IRIS_TR(var)
-#endif
-
 template <bool STATIC_LOCKS, int SUBS, int SUBS_M = 1>
 __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload, int warp, int lane) {
   constexpr uint32_t kFull = 0xFFFFFFFFu;
@@ -226,9 +217,6 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
   int widx = lane < n_my ? lane : -1;  // index into this warp's item list that this lane watches
   int next = n_my < 32 ? n_my : 32;
   uint64_t last_progress = globaltimer_ns();
-#ifdef IRIS_COMM_TRACE
-  uint64_t last_poll = last_progress;
-#endif
   uint32_t spins = 0;
   bool ok = true;
   // item -> publication tile, recomputed only when the lane moves to a new item
@@ -254,10 +242,6 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
       ready = t < 0 || state == 1 || state == 2;
     }
     const uint32_t mask = __ballot_sync(kFull, ready);
-#ifdef IRIS_COMM_TRACE
-    unsigned long long* tr = &g_comm_trace[(size_t)cw * 8];
-    if (lane == 0 && mask == 0) { const uint64_t now = globaltimer_ns(); tr[5] += now - last_poll; last_poll = now; }
-#endif
     if (mask == 0) {
       if ((++spins & 15u) == 0) {
         bool expired = false;
@@ -273,13 +257,9 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
       }
       continue;
     }
-    // Listing 5: tl.atomic_cas(locks + tile_id, 1, 0, sem="acquire", scope="gpu"); all ready lanes at once.
-    IRIS_TR(tc0);
+    // claim (Listing 5, communication branch): every ready lane takes its lock, state -> 0, acquire at gpu scope
     if (ready && t >= 0) (void)cas_acquire_gpu(lock_addr<STATIC_LOCKS>(p, rank, t), state, 0);
     __syncwarp();
-#ifdef IRIS_COMM_TRACE
-    if (lane == 0) tr[6] += globaltimer_ns() - tc0;
-#endif
     uint32_t todo = mask;
     while (todo) {
       const int src = __ffs(todo) - 1;
@@ -290,7 +270,6 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
       if (rt < 0 || rstate == 2) continue;   // no such sub-tile, or nothing left to do but the lock reset above
       const int tm = rt / pt_n, pj = (rt % pt_n) % p.ptiles_per_rank;
       bool fail = false;
-      IRIS_TR(t0);
       if (lane == 0) {
         fence_proxy_async();  // producers' generic-proxy stores (acquired above) -> our async-proxy read
         ptx::mbar_arrive_expect_tx(bar, kTileBytes);
@@ -299,31 +278,24 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
         if (!mbar_wait(bar, bar_phase, p, ctrl, rt)) {
           fail = true;
         } else {
-          IRIS_TR(t1);
           for (int s = 0; s < W; ++s) {
             if (s == rrank) continue;
             if (p.one_map) ptx::tma_store_4d(&p.tmC4, pj * IRIS_TILE, tm * IRIS_TILE, rrank, s, buf);
             else ptx::tma_store_3d(&p.tmC[s], pj * IRIS_TILE, tm * IRIS_TILE, rrank, buf);
           }
           ptx::bulk_commit_group();
-          IRIS_TR(t2);
           ptx::bulk_wait_group<0>();  // stores performed: the buffer is free and the tile may be published
           fence_proxy_async();        // async-proxy writes above -> the generic-proxy release of the flags below
-#ifdef IRIS_COMM_TRACE
-          const uint64_t t3 = globaltimer_ns();
-          tr[0] += 1; tr[1] += t1 - t0; tr[2] += t2 - t1; tr[3] += t3 - t2;
-#endif
         }
       }
       bar_phase ^= 1;
       if (__any_sync(kFull, fail)) { ok = false; break; }
-      IRIS_TR(t4);
+      // bar.warp.sync orders lane 0's wait for the bulk stores (and its proxy fence) before the other lanes' flag
+      // releases: a vote converges the warp but is not a memory barrier
+      __syncwarp();
       if (lane < W) st_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[lane] + p.flag_off) + rt, p.epoch);
       if (p.takeover && lane == 0) atomicAdd(p.backlog, -1);
       __syncwarp();
-#ifdef IRIS_COMM_TRACE
-      if (lane == 0) { tr[4] += globaltimer_ns() - t4; last_poll = globaltimer_ns(); }
-#endif
     }
     // lanes whose item was handled move on to the next unwatched items, in lane order
     if (mask & (1u << lane)) {
@@ -514,7 +486,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
         if (row < p.M) {
           const int c0 = col_in_shard + ch * 32;
           if (seq) {
-            // Listing 4: for remote_rank in range(world_size): iris.store(C + offset, c, cur_rank, remote_rank)
+            // Listing 4: the tile goes to every rank, the owner included, at the same symmetric offset
             for (int s = 0; s < W; ++s) {
               const uint64_t dst = p.tab.base[s] + row_off + (uint64_t)c0 * 2;  // translate(C + offset, rank -> s)
 #pragma unroll
@@ -611,7 +583,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
           const int pj = tc.jn * subs + et;
           if (pj < p.ptiles_per_rank) {
             const int t = tc.tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
-            // Listing 5: tl.atomic_cas(locks + tile_id, 0, 1, sem="release", scope="gpu")
+            // hand-over (Listing 5, producer branch): lock 0 -> 1, release at gpu scope
             (void)cas_release_gpu(lock_addr<STATIC_LOCKS>(p, tc.rank, t), 0, 1);
           }
         }
@@ -672,7 +644,8 @@ __device__ void consumer_warp(const GemmParams& p, CtrlBlock* ctrl, int cwarp, i
         }
       }
     }
-    ok = __shfl_sync(kFull, ok, 0);  // warp-level synchronisation: lane 0's acquire precedes every lane's reads
+    ok = __shfl_sync(kFull, ok, 0);
+    __syncwarp();   // bar.warp.sync orders lane 0's acquire of the flag before every lane's reads of the tile
     if (!ok) return;
     const int rows = min(IRIS_TILE, p.M - tm * IRIS_TILE);
     const uint64_t col0 = (uint64_t)tc.rank * p.n_local + (uint64_t)pj * IRIS_TILE;
@@ -847,9 +820,6 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         if (tile < 0) break;
         if (!mbar_wait(ptx::smem_u32(&ctrl->tmem_empty[acc]), acc_phase ^ 1, p, ctrl, tile)) break;
         ptx::tc_fence_after();
-#ifdef IRIS_COMM_TRACE
-        if (tile < 4096) { g_tile_trace[2 * tile] = globaltimer_ns(); unsigned sm; asm("mov.u32 %0, %%smid;" : "=r"(sm)); g_tile_trace[2 * tile + 1] = sm; }
-#endif
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kPairBN);
         const uint32_t idesc = ptx::idesc_f16(2 * BM, pair_tile_cols(p, decode_ctile(tile, p).jn), BF16 ? 1 : 0);
         bool ok = true;
@@ -943,7 +913,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         }
         ctrl->keep_tile = seq ? 1 : 0;
         // One thread stores the boxes with TMA: whole 128-byte lines, clipped by the maps at row M and column
-        // N_local, to the owner's slot or (Listing 4: for remote_rank in range(world_size): iris.store(...)) to all.
+        // N_local, to the owner's slot or (Listing 4's loop over all ranks) to all.
         // Stores and operand loads leave the SM through one queue: a burst of W x 4 boxes (512 KB, 9 us of the
         // port) holds up the loads of the tile that is being multiplied meanwhile for longer than the stage ring
         // covers.  So the boxes go out one at a time, spread over three quarters of the time this CTA takes per
@@ -1088,14 +1058,23 @@ static int make_map(CUtensorMap* m, int dtype, int rank, void* base, const cuuin
   return IRIS_OK;
 }
 
+// The dynamic shared-memory limit is an attribute of (function, device): set it once per device a kernel is
+// launched on.  `done` is that kernel's per-device record; the device is the current one.
+constexpr int kMaxDevices = 64;
+static int ensure_smem_limit(const void* kern, int bytes, bool (&done)[kMaxDevices]) {
+  int dev = 0;
+  IRIS_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev >= 0 && dev < kMaxDevices && done[dev]) return IRIS_OK;
+  IRIS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+  if (dev >= 0 && dev < kMaxDevices) done[dev] = true;
+  return IRIS_OK;
+}
+
 template <int BN, bool BF16, bool STATIC_LOCKS = false>
 static int launch_gemm(const GemmParams& p, int grid, bool cooperative, cudaStream_t st) {
   auto kern = gemm_all_scatter_kernel<BN, BF16, STATIC_LOCKS>;
-  static bool configured = false;
-  if (!configured) {
-    IRIS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemTotal));
-    configured = true;
-  }
+  static bool configured[kMaxDevices] = {};
+  if (int rc = ensure_smem_limit(reinterpret_cast<const void*>(kern), kSmemTotal, configured)) return rc;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)grid);
   cfg.blockDim = dim3(kGemmThreads);
@@ -1121,11 +1100,8 @@ static int launch_gemm(const GemmParams& p, int grid, bool cooperative, cudaStre
 template <bool BF16, bool STATIC_LOCKS = false, bool CONSUMER = false>
 static int launch_gemm_pair(const GemmParams& p, int grid, cudaStream_t st, int* max_pairs_out) {
   auto kern = gemm_all_scatter_pair_kernel<BF16, STATIC_LOCKS, CONSUMER>;
-  static bool configured = false;
-  if (!configured) {
-    IRIS_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kPairSmemTotal));
-    configured = true;
-  }
+  static bool configured[kMaxDevices] = {};
+  if (int rc = ensure_smem_limit(reinterpret_cast<const void*>(kern), kPairSmemTotal, configured)) return rc;
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3((unsigned)(max_pairs_out ? 2 : grid));
   cfg.blockDim = dim3(CONSUMER ? kGemmThreadsFused : kGemmThreads);
@@ -1184,7 +1160,29 @@ static int auto_comm_ctas_pair(int total_ctiles, int kblocks, double remote_byte
   return best_c;
 }
 
-// ---- launch-plan cache -------------------------------------------------------------------------------
+// ---- launch plans ---------------------------------------------------------------------------------------
+// What a plan needs to know about where the slots are: a heap handle's (equally spaced from `base`, status block in
+// the handle) or raw addresses (base == NULL: one tensor map per slot, single-CTA kernel only).
+struct PlanEnv {
+  HeapTable tab;
+  char* base;
+  uint64_t bpr;
+  int sm_count;
+  int32_t* status;
+};
+struct Plan { GemmParams p; int bn, grid; bool pair, streamk; };
+
+// Compute-tile width of the single-CTA kernel when the caller does not choose one.
+static int default_block_n(int M, int nl, int W, int sm_count) {
+  int bn = (nl % 256 == 0 || nl > 1024) ? 256 : 128;
+  // Few tiles (the skinny shapes): when the 128-wide tiles all fit in one wave they put more SMs to work on the
+  // B panels; when they need a second, partly filled wave (config 4: 224 tiles on 148 SMs) one wave of 256-wide
+  // tiles is faster (measured 0.127 vs 0.142 ms) although a quarter of the SMs then idle.
+  if ((int64_t)((M + BM - 1) / BM) * W * ((nl + 127) / 128) <= sm_count) bn = 128;
+  if (nl <= 128) bn = 128;
+  return bn;
+}
+
 struct PlanKey {
   const void* heap; const void* base; const void* status; uint64_t bytes_per_rank;
   const void* A; const void* B[IRIS_MAX_WORLD];
@@ -1193,7 +1191,6 @@ struct PlanKey {
   int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail, fused_consumer, rank_first, rank_count, pace_stores;
   uint64_t spin_timeout_ns;
 };
-struct Plan { GemmParams p; int bn, grid; bool pair, streamk; };
 // A few plans are kept (round-robin replacement): a step that alternates between calls -- one per rank shard in the
 // host-buffer pipeline, several schedules in a comparison -- finds each of them again on its next pass.
 constexpr int kPlanSlots = 16;
@@ -1222,6 +1219,179 @@ int64_t num_tiles(int M, int N, int world) {
   if (M < 0 || N < 0 || world < 1 || world > IRIS_MAX_WORLD || N % world != 0) return -1;
   const int64_t nl = N / world;
   return (int64_t)((M + IRIS_TILE - 1) / IRIS_TILE) * world * ((nl + IRIS_TILE - 1) / IRIS_TILE);
+}
+
+// Tile geometry, grid split and tensor maps of one call: everything but the epoch.  The arguments have been checked.
+static int build_plan(const iris_gemm_args* a, const PlanEnv& env, Plan& out) {
+  GemmParams& p = out.p;
+  int& bn = out.bn;
+  int& grid = out.grid;
+  bool& pair = out.pair;
+  bool& streamk = out.streamk;
+  const int W = a->world, nl = a->N / W;
+  const int rank_first = a->rank_first, rank_count = a->rank_count ? a->rank_count : W;   // 0, 0 = every rank
+  const bool wg = a->mode == IRIS_MODE_WORKGROUP_SPECIALIZED;
+  const bool fused_consumer = a->consumer_bias != nullptr;
+  std::memset(&p, 0, sizeof(p));
+  bn = a->block_n ? a->block_n : default_block_n(a->M, nl, W, env.sm_count);
+  if (nl <= 128) bn = 128;
+  // CTA pairs (256 x 256 tiles) need at least two tile rows.  A shard that is not a whole number of 256-column
+  // tiles is fine: TMA zero-fills the missing B rows, stores and flags are masked, and the last tile's MMA is only
+  // as wide as what is left of the shard (rounded up to 32 columns), so the padding costs next to nothing.
+  const bool pair_ok = a->M > BM && nl > BM && a->block_n != 128 && env.sm_count >= 4 && env.base != nullptr;
+  if (a->cta_pair > 0 && !pair_ok) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: cta_pair needs M > 128, N/world > 128 and block_n != 128");
+  pair = pair_ok && a->cta_pair >= 0;
+  int max_pairs = 0;
+  if (pair) {
+    const int rc = a->dtype == IRIS_BF16 ? launch_gemm_pair<true>(p, 0, nullptr, &max_pairs) : launch_gemm_pair<false>(p, 0, nullptr, &max_pairs);
+    if (rc != IRIS_OK) return rc;
+    if (max_pairs < 2) {
+      if (a->cta_pair > 0) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: no room for CTA pairs on this device");
+      pair = false;
+    }
+  }
+  if (pair) {   // a cap on the grid that leaves no room for whole pairs: fall back to single-CTA tiles unless pairs were demanded
+    const int cap = a->max_ctas ? std::min(a->max_ctas, env.sm_count) : env.sm_count;
+    if ((cap & ~1) < (wg ? 4 : 2)) {
+      if (a->cta_pair > 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: max_ctas too small for CTA pairs");
+      pair = false;
+    }
+  }
+  if (pair) bn = kPairBN;
+  p.tab = env.tab;
+  p.c_off = a->c_off;
+  p.flag_off = a->flag_off;
+  p.lock_off = a->lock_off;
+  p.timeout_ns = a->spin_timeout_ns ? a->spin_timeout_ns : kDefaultTimeoutNs;
+  p.status = env.status;
+  p.M = a->M; p.N = a->N; p.K = a->K; p.n_local = nl;
+  p.ptiles_m = (a->M + BM - 1) / BM;
+  p.tiles_m = pair ? (a->M + 2 * BM - 1) / (2 * BM) : p.ptiles_m;
+  p.ctiles_per_rank = (nl + bn - 1) / bn;
+  p.ptiles_per_rank = (nl + IRIS_TILE - 1) / IRIS_TILE;
+  p.rank_first = rank_first; p.rank_count = rank_count;
+  p.total_ctiles = p.tiles_m * rank_count * p.ctiles_per_rank;
+  p.total_ptiles = p.ptiles_m * rank_count * p.ptiles_per_rank;
+  p.kblocks = (a->K + BK - 1) / BK;
+  // 2048 rows per raster group: with tiles claimed in raster order the running tiles then cover about
+  // 8 x 9 pair tiles, the near-square footprint that minimises operand re-reads from HBM (measured).
+  p.raster_group = a->raster_group ? a->raster_group : (pair ? 8 : 16);
+  p.mode = a->mode;
+  p.epoch = a->epoch;
+  grid = a->max_ctas ? std::min(a->max_ctas, env.sm_count) : env.sm_count;
+  if (pair) {
+    grid = std::min(grid & ~1, 2 * max_pairs);
+    if (grid < (wg ? 4 : 2)) return fail(IRIS_ERR_ARG, "gemm_all_scatter: max_ctas too small for CTA pairs");
+    if (wg) {
+      int comm = a->comm_ctas;
+      // (with consumer warps in the producer CTAs their ports are busy with OUT = C + bias: the communication CTAs
+      // then get the whole scatter, as they do without the takeover rule)
+      if (!comm) comm = a->wg_tail == 0 && !fused_consumer ? auto_comm_ctas_pair(p.total_ctiles, p.kblocks, (double)(W - 1) * a->M * nl * rank_count * 2.0, grid)
+                                                            : auto_comm_ctas(a->M, nl * rank_count, a->K, W, grid);
+      comm = std::max(2, std::min((comm + 1) & ~1, grid - 2));   // whole pairs on both sides
+      p.comm_ctas = comm;
+      p.gemm_ctas = 2 * std::min((grid - comm) / 2, p.total_ctiles);
+    } else {
+      p.comm_ctas = 0;
+      p.gemm_ctas = 2 * std::min(grid / 2, p.total_ctiles);
+    }
+    // The fewest producer pairs that still finish in the same number of waves: on this power-capped part an SM
+    // that would only idle through the last, partly filled wave is better left out, the others then clock higher
+    // (W = 8, 1024 x 16384 x 16384: 256 tiles on 64 pairs instead of 74, fused_sequential 0.425 -> 0.398 ms).
+    if (p.total_ctiles > 0) {
+      const int units = p.gemm_ctas / 2;
+      const int waves = (p.total_ctiles + units - 1) / units;
+      p.gemm_ctas = 2 * ((p.total_ctiles + waves - 1) / waves);
+    }
+  } else if (wg) {
+    if (grid < 2) return fail(IRIS_ERR_ARG, "gemm_all_scatter: workgroup_specialized needs at least 2 CTAs");
+    int comm = a->comm_ctas ? a->comm_ctas : auto_comm_ctas(a->M, nl * rank_count, a->K, W, grid);
+    comm = std::min(comm, std::min(grid - 1, p.total_ptiles));
+    p.comm_ctas = comm;
+    p.gemm_ctas = std::min(grid - comm, p.total_ctiles);
+  } else {
+    p.comm_ctas = 0;
+    p.gemm_ctas = std::min(grid, p.total_ctiles);
+  }
+  // stream-K (single-CTA kernel): when the tile count leaves the last wave badly filled, cut the k-steps of all
+  // tiles into equal ranges instead, one per producer CTA.
+  streamk = false;
+  if (!pair && a->stream_k >= 0 && p.kblocks > 0) {
+    const int producers = wg ? std::max(1, std::min(grid, env.sm_count) - p.comm_ctas) : grid;
+    const int64_t waves = (p.total_ctiles + producers - 1) / producers;
+    const bool badly_filled = (int64_t)p.total_ctiles * 10 < waves * producers * 9;      // < 90 % of the slots used
+    const bool enough_k = (int64_t)p.total_ctiles * p.kblocks >= (int64_t)producers * 4 && p.kblocks >= 8;
+    (void)badly_filled;   // measured: on the skinny shapes this was meant for, operand streaming -- not the wave fill -- is the
+                          // limit and the parts' round trip through the workspace costs more than it saves: on request only
+    if (enough_k && a->stream_k > 0) {
+      streamk = true;
+      p.gemm_ctas = producers;
+    }
+  }
+  p.streamk = streamk ? 1 : 0;
+  grid = p.gemm_ctas + p.comm_ctas;
+  // Which tiles the producers scatter themselves.  In workgroup_specialized mode the tiles of the last wave
+  // (raster ids >= total - producer units; every unit's final tile is one of them) have no GEMM work left to
+  // overlap with, so handing them to a few communication CTAs would leave their store ports as the only ones
+  // busy at the end of the kernel: the producers write those tiles to all W slots and publish them, as in
+  // fused_sequential mode.  wg_tail: -1 = never (Listing 5 for every tile), n > 0 = the last n compute tiles.
+  p.takeover = 0;
+  p.t_tile_ns = (uint32_t)std::min<int64_t>((int64_t)p.kblocks * 260, 1 << 28);   // 512 tensor cycles per k-step at full clocks
+  p.pace_stores = pair && a->pace_stores >= 0 ? 1 : 0;
+  if (a->mode == IRIS_MODE_FUSED_SEQUENTIAL) p.seq_from = 0;
+  else if (!wg || a->wg_tail < 0) p.seq_from = INT_MAX;
+  else {
+    const int units = pair ? p.gemm_ctas / 2 : p.gemm_ctas;
+    p.seq_from = std::max(0, p.total_ctiles - (a->wg_tail > 0 ? a->wg_tail : units));
+    // wg_tail = 0 on the pair kernel: producers also keep tiles the communication CTAs could not finish in time.
+    // Estimates: one SM's port stores at most 57 GB/s, shared by the CTA's communicator warps; a k-step of a pair
+    // tile takes 512 tensor cycles.
+    if (pair && a->wg_tail == 0) {
+      p.takeover = 1;
+      p.t_pt_ns = (uint32_t)((uint64_t)kCommWarps * kTileBytes * (W - 1) / 45);   // 45 GB/s: what a communication SM sustains
+    }
+  }
+
+  // Tensor maps.  K == 0 has no operand to describe; the kernel then never issues a load.
+  if (a->K > 0) {
+    const cuuint64_t dimsA[2] = {(cuuint64_t)a->K, (cuuint64_t)a->M};
+    const cuuint64_t strA[1] = {(cuuint64_t)a->K * 2};
+    const cuuint32_t boxA[2] = {BK, BM};
+    int rc = make_map(&p.tmA, a->dtype, 2, const_cast<void*>(a->A), dimsA, strA, boxA, CU_TENSOR_MAP_SWIZZLE_128B, "A");
+    if (rc != IRIS_OK) return rc;
+    for (int r = rank_first; r < rank_first + rank_count; ++r) {
+      const cuuint64_t dimsB[2] = {(cuuint64_t)a->K, (cuuint64_t)nl};
+      const cuuint32_t boxB[2] = {BK, (cuuint32_t)(pair ? kPairBN / 2 : bn)};   // a pair's CTA loads its half of the tile
+      rc = make_map(&p.tmB[r], a->dtype, 2, const_cast<void*>(a->B_shards[r]), dimsB, strA, boxB, CU_TENSOR_MAP_SWIZZLE_128B, "B");
+      if (rc != IRIS_OK) return rc;
+    }
+  }
+  if (env.base) {
+    // C of every slot as one 4-D tensor [slot][rank][row][column]: the slots of a heap handle are bytes_per_rank apart.
+    const cuuint64_t dims4[4] = {(cuuint64_t)nl, (cuuint64_t)a->M, (cuuint64_t)W, (cuuint64_t)W};
+    const cuuint64_t str4[3] = {(cuuint64_t)a->N * 2, (cuuint64_t)nl * 2, (cuuint64_t)env.bpr};
+    const cuuint32_t box4[4] = {IRIS_TILE, IRIS_TILE, 1, 1}, box4s[4] = {64, BM, 1, 1};
+    p.one_map = 1;
+    if (wg) {
+      int rc = make_map(&p.tmC4, a->dtype, 4, env.base + a->c_off, dims4, str4, box4, CU_TENSOR_MAP_SWIZZLE_NONE, "C (all slots)");
+      if (rc != IRIS_OK) return rc;
+    }
+    if (pair) {
+      int rc = make_map(&p.tmC4s, a->dtype, 4, env.base + a->c_off, dims4, str4, box4s, CU_TENSOR_MAP_SWIZZLE_128B, "C (all slots, epilogue stores)");
+      if (rc != IRIS_OK) return rc;
+    }
+  } else {
+    // slots at arbitrary addresses: C of slot s as [rank][row][column], one map per slot (communication CTAs only)
+    p.one_map = 0;
+    for (int s = 0; wg && s < W; ++s) {
+      const cuuint64_t dimsC[3] = {(cuuint64_t)nl, (cuuint64_t)a->M, (cuuint64_t)W};
+      const cuuint64_t strC[2] = {(cuuint64_t)a->N * 2, (cuuint64_t)nl * 2};
+      const cuuint32_t boxC[3] = {IRIS_TILE, IRIS_TILE, 1};
+      int rc = make_map(&p.tmC[s], a->dtype, 3, reinterpret_cast<void*>(env.tab.base[s] + a->c_off), dimsC, strC, boxC, CU_TENSOR_MAP_SWIZZLE_NONE, "C");
+      if (rc != IRIS_OK) return rc;
+    }
+  }
+  return IRIS_OK;
 }
 
 // Streams and events of iris_gemm_all_scatter_host's copy / compute / copy-back pipeline.
@@ -1328,163 +1498,11 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     }
   }
   auto build = [&]() -> int {
-    std::memset(&p, 0, sizeof(p));
-    bn = a->block_n;
-    if (bn == 0) {
-      bn = (nl % 256 == 0 || nl > 1024) ? 256 : 128;
-      // Few tiles (the skinny shapes): when the 128-wide tiles all fit in one wave they put more SMs to work on the
-      // B panels; when they need a second, partly filled wave (config 4: 224 tiles on 148 SMs) one wave of 256-wide
-      // tiles is faster (measured 0.127 vs 0.142 ms) although a quarter of the SMs then idle.
-      if ((int64_t)((a->M + BM - 1) / BM) * W * ((nl + 127) / 128) <= h->sm_count) bn = 128;
-    }
-    if (nl <= 128) bn = 128;
-    // CTA pairs (256 x 256 tiles) need at least two tile rows.  A shard that is not a whole number of 256-column
-    // tiles is fine: TMA zero-fills the missing B rows, stores and flags are masked, and the last tile's MMA is only
-    // as wide as what is left of the shard (rounded up to 32 columns), so the padding costs next to nothing.
-    const bool pair_ok = a->M > BM && nl > BM && a->block_n != 128 && h->sm_count >= 4;
-    if (a->cta_pair > 0 && !pair_ok) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: cta_pair needs M > 128, N/world > 128 and block_n != 128");
-    pair = pair_ok && a->cta_pair >= 0;
-    int max_pairs = 0;
-    if (pair) {
-      const int rc = a->dtype == IRIS_BF16 ? launch_gemm_pair<true>(p, 0, nullptr, &max_pairs) : launch_gemm_pair<false>(p, 0, nullptr, &max_pairs);
-      if (rc != IRIS_OK) return rc;
-      if (max_pairs < 2) {
-        if (a->cta_pair > 0) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: no room for CTA pairs on this device");
-        pair = false;
-      }
-    }
-    if (pair) {   // a cap on the grid that leaves no room for whole pairs: fall back to single-CTA tiles unless pairs were demanded
-      const int cap = a->max_ctas ? std::min(a->max_ctas, h->sm_count) : h->sm_count;
-      if ((cap & ~1) < (wg ? 4 : 2)) {
-        if (a->cta_pair > 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: max_ctas too small for CTA pairs");
-        pair = false;
-      }
-    }
-    if (pair) bn = kPairBN;
-    p.tab = h->table();
-    p.c_off = a->c_off;
-    p.flag_off = a->flag_off;
-    p.lock_off = a->lock_off;
-    p.timeout_ns = a->spin_timeout_ns ? a->spin_timeout_ns : kDefaultTimeoutNs;
-    p.status = h->status;
-    p.M = a->M; p.N = a->N; p.K = a->K; p.n_local = nl;
-    p.ptiles_m = (a->M + BM - 1) / BM;
-    p.tiles_m = pair ? (a->M + 2 * BM - 1) / (2 * BM) : p.ptiles_m;
-    p.ctiles_per_rank = (nl + bn - 1) / bn;
-    p.ptiles_per_rank = (nl + IRIS_TILE - 1) / IRIS_TILE;
-    p.rank_first = rank_first; p.rank_count = rank_count;
-    p.total_ctiles = p.tiles_m * rank_count * p.ctiles_per_rank;
-    p.total_ptiles = p.ptiles_m * rank_count * p.ptiles_per_rank;
-    p.kblocks = (a->K + BK - 1) / BK;
-    // 2048 rows per raster group: with tiles claimed in raster order the running tiles then cover about
-    // 8 x 9 pair tiles, the near-square footprint that minimises operand re-reads from HBM (measured).
-    p.raster_group = a->raster_group ? a->raster_group : (pair ? 8 : 16);
-    p.mode = a->mode;
-    p.epoch = a->epoch;
-    grid = a->max_ctas ? std::min(a->max_ctas, h->sm_count) : h->sm_count;
-    if (pair) {
-      grid = std::min(grid & ~1, 2 * max_pairs);
-      if (grid < (wg ? 4 : 2)) return fail(IRIS_ERR_ARG, "gemm_all_scatter: max_ctas too small for CTA pairs");
-      if (wg) {
-        int comm = a->comm_ctas;
-        // (with consumer warps in the producer CTAs their ports are busy with OUT = C + bias: the communication CTAs
-        // then get the whole scatter, as they do without the takeover rule)
-        if (!comm) comm = a->wg_tail == 0 && !fused_consumer ? auto_comm_ctas_pair(p.total_ctiles, p.kblocks, (double)(W - 1) * a->M * nl * rank_count * 2.0, grid)
-                                                              : auto_comm_ctas(a->M, nl * rank_count, a->K, W, grid);
-        comm = std::max(2, std::min((comm + 1) & ~1, grid - 2));   // whole pairs on both sides
-        p.comm_ctas = comm;
-        p.gemm_ctas = 2 * std::min((grid - comm) / 2, p.total_ctiles);
-      } else {
-        p.comm_ctas = 0;
-        p.gemm_ctas = 2 * std::min(grid / 2, p.total_ctiles);
-      }
-      // The fewest producer pairs that still finish in the same number of waves: on this power-capped part an SM
-      // that would only idle through the last, partly filled wave is better left out, the others then clock higher
-      // (W = 8, 1024 x 16384 x 16384: 256 tiles on 64 pairs instead of 74, fused_sequential 0.425 -> 0.398 ms).
-      if (p.total_ctiles > 0) {
-        const int units = p.gemm_ctas / 2;
-        const int waves = (p.total_ctiles + units - 1) / units;
-        p.gemm_ctas = 2 * ((p.total_ctiles + waves - 1) / waves);
-      }
-    } else if (wg) {
-      if (grid < 2) return fail(IRIS_ERR_ARG, "gemm_all_scatter: workgroup_specialized needs at least 2 CTAs");
-      int comm = a->comm_ctas ? a->comm_ctas : auto_comm_ctas(a->M, nl * rank_count, a->K, W, grid);
-      comm = std::min(comm, std::min(grid - 1, p.total_ptiles));
-      p.comm_ctas = comm;
-      p.gemm_ctas = std::min(grid - comm, p.total_ctiles);
-    } else {
-      p.comm_ctas = 0;
-      p.gemm_ctas = std::min(grid, p.total_ctiles);
-    }
-    // stream-K (single-CTA kernel): when the tile count leaves the last wave badly filled, cut the k-steps of all
-    // tiles into equal ranges instead, one per producer CTA.
-    streamk = false;
-    if (!pair && a->stream_k >= 0 && p.kblocks > 0) {
-      const int producers = wg ? std::max(1, std::min(grid, h->sm_count) - p.comm_ctas) : grid;
-      const int64_t waves = (p.total_ctiles + producers - 1) / producers;
-      const bool badly_filled = (int64_t)p.total_ctiles * 10 < waves * producers * 9;      // < 90 % of the slots used
-      const bool enough_k = (int64_t)p.total_ctiles * p.kblocks >= (int64_t)producers * 4 && p.kblocks >= 8;
-      (void)badly_filled;   // measured: on the skinny shapes this was meant for, operand streaming -- not the wave fill -- is the
-                            // limit and the parts' round trip through the workspace costs more than it saves: on request only
-      if (enough_k && a->stream_k > 0) {
-        streamk = true;
-        p.gemm_ctas = producers;
-      }
-    }
-    p.streamk = streamk ? 1 : 0;
-    grid = p.gemm_ctas + p.comm_ctas;
-    // Which tiles the producers scatter themselves.  In workgroup_specialized mode the tiles of the last wave
-    // (raster ids >= total - producer units; every unit's final tile is one of them) have no GEMM work left to
-    // overlap with, so handing them to a few communication CTAs would leave their store ports as the only ones
-    // busy at the end of the kernel: the producers write those tiles to all W slots and publish them, as in
-    // fused_sequential mode.  wg_tail: -1 = never (Listing 5 for every tile), n > 0 = the last n compute tiles.
-    p.takeover = 0;
-    p.t_tile_ns = (uint32_t)std::min<int64_t>((int64_t)p.kblocks * 260, 1 << 28);   // 512 tensor cycles per k-step at full clocks
-    p.pace_stores = pair && a->pace_stores >= 0 ? 1 : 0;
-    if (a->mode == IRIS_MODE_FUSED_SEQUENTIAL) p.seq_from = 0;
-    else if (!wg || a->wg_tail < 0) p.seq_from = INT_MAX;
-    else {
-      const int units = pair ? p.gemm_ctas / 2 : p.gemm_ctas;
-      p.seq_from = std::max(0, p.total_ctiles - (a->wg_tail > 0 ? a->wg_tail : units));
-      // wg_tail = 0 on the pair kernel: producers also keep tiles the communication CTAs could not finish in time.
-      // Estimates: one SM's port stores at most 57 GB/s, shared by the CTA's communicator warps; a k-step of a pair
-      // tile takes 512 tensor cycles.
-      if (pair && a->wg_tail == 0) {
-        p.takeover = 1;
-        p.t_pt_ns = (uint32_t)((uint64_t)kCommWarps * kTileBytes * (W - 1) / 45);   // 45 GB/s: what a communication SM sustains
-      }
-    }
-
-    // Tensor maps.  K == 0 has no operand to describe; the kernel then never issues a load.
-    if (a->K > 0) {
-      const cuuint64_t dimsA[2] = {(cuuint64_t)a->K, (cuuint64_t)a->M};
-      const cuuint64_t strA[1] = {(cuuint64_t)a->K * 2};
-      const cuuint32_t boxA[2] = {BK, BM};
-      int rc = make_map(&p.tmA, a->dtype, 2, const_cast<void*>(a->A), dimsA, strA, boxA, CU_TENSOR_MAP_SWIZZLE_128B, "A");
-      if (rc != IRIS_OK) return rc;
-      for (int r = rank_first; r < rank_first + rank_count; ++r) {
-        const cuuint64_t dimsB[2] = {(cuuint64_t)a->K, (cuuint64_t)nl};
-        const cuuint32_t boxB[2] = {BK, (cuuint32_t)(pair ? kPairBN / 2 : bn)};   // a pair's CTA loads its half of the tile
-        rc = make_map(&p.tmB[r], a->dtype, 2, const_cast<void*>(a->B_shards[r]), dimsB, strA, boxB, CU_TENSOR_MAP_SWIZZLE_128B, "B");
-        if (rc != IRIS_OK) return rc;
-      }
-    }
-    {
-      // C of every slot as one 4-D tensor [slot][rank][row][column]: the slots of a heap handle are bytes_per_rank apart.
-      const cuuint64_t dims4[4] = {(cuuint64_t)nl, (cuuint64_t)a->M, (cuuint64_t)W, (cuuint64_t)W};
-      const cuuint64_t str4[3] = {(cuuint64_t)a->N * 2, (cuuint64_t)nl * 2, (cuuint64_t)bpr};
-      const cuuint32_t box4[4] = {IRIS_TILE, IRIS_TILE, 1, 1}, box4s[4] = {64, BM, 1, 1};
-      p.one_map = 1;
-      if (wg) {
-        int rc = make_map(&p.tmC4, a->dtype, 4, h->base + a->c_off, dims4, str4, box4, CU_TENSOR_MAP_SWIZZLE_NONE, "C (all slots)");
-        if (rc != IRIS_OK) return rc;
-      }
-      if (pair) {
-        int rc = make_map(&p.tmC4s, a->dtype, 4, h->base + a->c_off, dims4, str4, box4s, CU_TENSOR_MAP_SWIZZLE_128B, "C (all slots, epilogue stores)");
-        if (rc != IRIS_OK) return rc;
-      }
-    }
-    return IRIS_OK;
+    PlanEnv env{h->table(), h->base, h->bytes_per_rank, h->sm_count, h->status};
+    Plan pl;
+    const int rc = build_plan(a, env, pl);
+    p = pl.p; bn = pl.bn; grid = pl.grid; pair = pl.pair; streamk = pl.streamk;
+    return rc;
   };
   if (!hit) {
     const int brc = build();
@@ -1548,6 +1566,25 @@ static void short_form_layout(int M, int N, int world, uint64_t* flag_off, uint6
   *lock_off = *flag_off + align_up((uint64_t)(nt > 0 ? nt : 0) * 4, 256);
 }
 
+// The short form and the host-buffer entry point choose where flags and locks live, so they also initialise them:
+// on the heap's first such call, and whenever (M, N) -- hence the layout -- changes, both arrays are zeroed in every
+// slot on `st` before the launch (stale locks would break Listing 5's handshake, stale flags >= epoch would let a
+// consumer read early).  The epoch keeps growing, so zeroed flags are always "not yet published".
+static int short_form_init(iris_heap* heap, int M, int N, int world, cudaStream_t st) {
+  if (heap->sf_M == M && heap->sf_N == N) return IRIS_OK;
+  const int64_t nt = num_tiles(M, N, world);
+  uint64_t flag_off, lock_off;
+  short_form_layout(M, N, world, &flag_off, &lock_off);
+  const uint64_t bytes = (lock_off - flag_off) * 2;   // both arrays, each rounded up to 256 bytes
+  if (nt > 0) {
+    if (flag_off > heap->bytes_per_rank || bytes > heap->bytes_per_rank - flag_off) return fail(IRIS_ERR_RANGE, "gemm_all_scatter: flags and locks leave the slot");
+    for (int s = 0; s < world; ++s)
+      IRIS_CUDA_TRY(cudaMemsetAsync(heap->base + (size_t)s * heap->bytes_per_rank + flag_off, 0, bytes, st));
+  }
+  heap->sf_M = M; heap->sf_N = N;
+  return IRIS_OK;
+}
+
 static int short_form(const void* A, const void* const* B_shards, iris_heap* heap, int M, int N, int K, int world, int mode, int dtype, void* stream,
                       const void* bias = nullptr, uint64_t out_off = 0) {
   if (!heap_ok(heap)) return fail(IRIS_ERR_STATE, "gemm_all_scatter: bad heap handle");
@@ -1561,7 +1598,9 @@ static int short_form(const void* A, const void* const* B_shards, iris_heap* hea
   a.epoch = heap->epoch + 1;
   a.consumer_bias = bias;
   a.consumer_out_off = out_off;
-  const int rc = iris_gemm_all_scatter_ex(&a, stream);
+  int rc = short_form_init(heap, M, N, world, static_cast<cudaStream_t>(stream));
+  if (rc != IRIS_OK) return rc;
+  rc = iris_gemm_all_scatter_ex(&a, stream);
   if (rc == IRIS_OK) heap->epoch = a.epoch;
   return rc;
 }
@@ -1660,6 +1699,7 @@ int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_h
   IRIS_CUDA_TRY(cudaStreamWaitEvent(s_run, hp->b_ready, 0));
 
   char* slot = heap->base + (size_t)out_slot * heap->bytes_per_rank;
+  if (int irc = short_form_init(heap, M, N, world, s_run)) return irc;
   const int32_t epoch = heap->epoch + 1;
   for (int blk = 0; blk < blocks; ++blk) {
     const int r0 = by_ranks ? 0 : blk * rows_per_block;
@@ -1737,11 +1777,13 @@ int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, co
       if (!B_shards[r] || (uint64_t)B_shards[r] % 16 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter_noalloc: B_shards[%d] is NULL or not 16-byte aligned", r);
   }
 
-  // Set-up, once per device, with that device current: the device address of the static scratch.
-  static int32_t* scratch_of_device[64] = {nullptr};
+  // Set-up, once per device, with that device current: the device address of the static scratch.  (The record is
+  // filled without a lock: two threads making a device's first call at the same time both look the address up and
+  // store the same value.)
+  static int32_t* scratch_of_device[kMaxDevices] = {nullptr};
   int dev = -1, sms = 0;
   IRIS_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter_noalloc: device ordinal %d not supported", dev);
+  if (dev < 0 || dev >= kMaxDevices) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter_noalloc: device ordinal %d not supported", dev);
   if (!scratch_of_device[dev]) {
     void* sym = nullptr;
     cudaError_t e = cudaGetSymbolAddress(&sym, g_noalloc_scratch);
@@ -1755,78 +1797,40 @@ int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, co
   // The array keeps the previous call's contents: the status block and the locks in use must start at zero.
   IRIS_CUDA_TRY(cudaMemsetAsync(scratch, 0, (size_t)(kNoAllocStatusWords + nt) * 4, st));
 
-  GemmParams p;
-  std::memset(&p, 0, sizeof(p));
-  const int bn = (nl <= 128) ? 128 : ((nl % 256 == 0 || nl > 1024) ? 256 : 128);
-  for (int r = 0; r < world; ++r) p.tab.base[r] = slot_bases[r];
-  p.tab.bytes_per_rank = bytes_per_rank;
-  p.tab.world = world;
-  p.c_off = c_off;
-  p.flag_off = flag_off;
-  p.timeout_ns = kDefaultTimeoutNs;
-  p.status = scratch;
-  p.M = M; p.N = N; p.K = K; p.n_local = nl;
-  p.tiles_m = (M + BM - 1) / BM;
-  p.ptiles_m = p.tiles_m;
-  p.ctiles_per_rank = (nl + bn - 1) / bn;
-  p.ptiles_per_rank = (nl + IRIS_TILE - 1) / IRIS_TILE;
-  p.rank_first = 0; p.rank_count = world;
-  p.total_ctiles = p.tiles_m * world * p.ctiles_per_rank;
-  p.total_ptiles = p.tiles_m * world * p.ptiles_per_rank;
-  p.kblocks = (K + BK - 1) / BK;
-  p.raster_group = 16;
-  p.mode = IRIS_MODE_WORKGROUP_SPECIALIZED;
-  p.epoch = epoch;
-  p.comm_ctas = std::min(auto_comm_ctas(M, N, K, world, sms), std::min(sms - 1, p.total_ptiles));
-  p.gemm_ctas = std::min(sms - p.comm_ctas, p.total_ctiles);
-  p.seq_from = std::max(0, p.total_ctiles - p.gemm_ctas);   // the last wave is scattered by its producers
-  if (K > 0) {
-    const cuuint64_t dimsA[2] = {(cuuint64_t)K, (cuuint64_t)M};
-    const cuuint64_t strA[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t boxA[2] = {BK, BM};
-    int rc = make_map(&p.tmA, dtype, 2, const_cast<void*>(A), dimsA, strA, boxA, CU_TENSOR_MAP_SWIZZLE_128B, "A");
-    if (rc != IRIS_OK) return rc;
-    for (int r = 0; r < world; ++r) {
-      const cuuint64_t dimsB[2] = {(cuuint64_t)K, (cuuint64_t)nl};
-      const cuuint32_t boxB[2] = {BK, (cuuint32_t)bn};
-      rc = make_map(&p.tmB[r], dtype, 2, const_cast<void*>(B_shards[r]), dimsB, strA, boxB, CU_TENSOR_MAP_SWIZZLE_128B, "B");
-      if (rc != IRIS_OK) return rc;
-    }
-  }
-  for (int s = 0; s < world; ++s) {
-    const cuuint64_t dimsC[3] = {(cuuint64_t)nl, (cuuint64_t)M, (cuuint64_t)world};
-    const cuuint64_t strC[2] = {(cuuint64_t)N * 2, (cuuint64_t)nl * 2};
-    const cuuint32_t boxC[3] = {IRIS_TILE, IRIS_TILE, 1};
-    int rc = make_map(&p.tmC[s], dtype, 3, reinterpret_cast<void*>(slot_bases[s] + c_off), dimsC, strC, boxC, CU_TENSOR_MAP_SWIZZLE_NONE, "C");
-    if (rc != IRIS_OK) return rc;
-  }
-  const int grid = p.gemm_ctas + p.comm_ctas;
-  const bool bf = dtype == IRIS_BF16;
-  int rc;
-  if (bn == 256) rc = bf ? launch_gemm<256, true, true>(p, grid, true, st) : launch_gemm<256, false, true>(p, grid, true, st);
-  else           rc = bf ? launch_gemm<128, true, true>(p, grid, true, st) : launch_gemm<128, false, true>(p, grid, true, st);
+  // The plan is the one iris_gemm_all_scatter_ex builds for workgroup_specialized with single-CTA tiles and default
+  // tuning (same function), with the slots at the caller's addresses and the locks and status block in the scratch.
+  iris_gemm_args a;
+  std::memset(&a, 0, sizeof(a));
+  a.A = A; a.B_shards = B_shards;
+  a.M = M; a.N = N; a.K = K; a.world = world; a.mode = IRIS_MODE_WORKGROUP_SPECIALIZED; a.dtype = dtype;
+  a.c_off = c_off; a.flag_off = flag_off; a.epoch = epoch;
+  a.cta_pair = -1;
+  PlanEnv env{};
+  for (int r = 0; r < world; ++r) env.tab.base[r] = slot_bases[r];
+  env.tab.bytes_per_rank = bytes_per_rank;
+  env.tab.world = world;
+  env.base = nullptr;
+  env.bpr = bytes_per_rank;
+  env.sm_count = sms;
+  env.status = scratch;
+  Plan pl;
+  int rc = build_plan(&a, env, pl);
   if (rc != IRIS_OK) return rc;
+  if (pl.pair || pl.streamk) return fail(IRIS_ERR_STATE, "gemm_all_scatter_noalloc: unexpected plan");
+  pl.p.epoch = epoch;
+  const bool bf = dtype == IRIS_BF16;
+  if (pl.bn == 256) rc = bf ? launch_gemm<256, true, true>(pl.p, pl.grid, true, st) : launch_gemm<256, false, true>(pl.p, pl.grid, true, st);
+  else              rc = bf ? launch_gemm<128, true, true>(pl.p, pl.grid, true, st) : launch_gemm<128, false, true>(pl.p, pl.grid, true, st);
+  if (rc != IRIS_OK) return rc;
+  // the status words come back on the caller's stream (no other stream is touched), then one wait for that stream
+  int32_t host_status[kStatusWords] = {0};
+  IRIS_CUDA_TRY(cudaMemcpyAsync(host_status, scratch, sizeof(host_status), cudaMemcpyDeviceToHost, st));
   IRIS_CUDA_TRY(cudaStreamSynchronize(st));
-  int32_t host_status[kStatusWords];
-  IRIS_CUDA_TRY(cudaMemcpy(host_status, scratch, sizeof(host_status), cudaMemcpyDeviceToHost));
   if (host_status[0] != 0)
     return fail(host_status[0], "gemm_all_scatter_noalloc: device-side wait expired: block=%d tile=%d", host_status[2], host_status[3]);
   return IRIS_OK;
 }
 
 
-#ifdef IRIS_COMM_TRACE
-int iris_debug_comm_trace(unsigned long long* host_out, int clear) {
-  cudaDeviceSynchronize();
-  if (host_out) cudaMemcpyFromSymbol(host_out, g_comm_trace, sizeof(g_comm_trace));
-  if (clear) { static unsigned long long z[64 * 6 * 8]; cudaMemcpyToSymbol(g_comm_trace, z, sizeof(z)); }
-  return 0;
-}
-int iris_debug_tile_trace(unsigned long long* host_out) {
-  cudaDeviceSynchronize();
-  cudaMemcpyFromSymbol(host_out, g_tile_trace, sizeof(g_tile_trace));
-  return 0;
-}
-#endif
 
 }  // extern "C"

@@ -72,7 +72,16 @@ int iris_heap_create_ex(int world, size_t bytes_per_rank, void* external_base, i
     }
     h->base = static_cast<char*>(p);
     h->owns = true;
+    // flags, locks and everything else start at zero (a caller-owned backing store is left as the caller prepared it)
+    e = cudaMemset(p, 0, (size_t)world * bytes_per_rank);
+    if (e != cudaSuccess) {
+      cudaFree(p);
+      delete h;
+      cudaGetLastError();
+      return fail(IRIS_ERR_CUDA, "iris_heap_create: cudaMemset: %s", cudaGetErrorString(e));
+    }
   }
+  h->sf_M = h->sf_N = -1;
   cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&h->status), 256);
   if (e == cudaSuccess) e = cudaMemset(h->status, 0, 256);
   if (e != cudaSuccess) {

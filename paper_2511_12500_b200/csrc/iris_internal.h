@@ -49,6 +49,7 @@ struct iris_heap {
   uint64_t bump;       // next free offset
   int32_t* status;     // device, kStatusWords int32
   int32_t epoch;       // last epoch used by the short-form call
+  int sf_M, sf_N;      // short form / host entry point: the (M, N) whose flag and lock arrays have been zeroed (-1: none yet)
   int sm_count;
   // staging for the host-buffer entry point
   void* stage_a;

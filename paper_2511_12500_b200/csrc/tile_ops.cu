@@ -85,6 +85,46 @@ __global__ void __launch_bounds__(256) atomic_op_kernel(const __grid_constant__ 
   }
 }
 
+// ---- 64-bit atomic_add / atomic_cas (Table 3's atomics on uint64 words), same sem x scope choice -----------
+#define IRIS_ATOM64_CASE(SEMV, SCOPEV, SEMS, SCOPES)                                                         \
+  if (sem == SEMV && scope == SCOPEV) {                                                                      \
+    if (IS_CAS)                                                                                              \
+      asm volatile("atom." SEMS "." SCOPES ".global.cas.b64 %0, [%1], %2, %3;"                               \
+                   : "=l"(old) : "l"(p), "l"(cmp), "l"(val) : "memory");                                     \
+    else                                                                                                     \
+      asm volatile("atom." SEMS "." SCOPES ".global.add.u64 %0, [%1], %2;" : "=l"(old) : "l"(p), "l"(val) : "memory"); \
+    return old;                                                                                              \
+  }
+
+template <bool IS_CAS>
+__device__ __forceinline__ uint64_t atomic_rmw64(uint64_t* p, uint64_t cmp, uint64_t val, int sem, int scope) {
+  uint64_t old = 0;
+  IRIS_ATOM64_CASE(IRIS_SEM_RELAXED, IRIS_SCOPE_BLOCK, "relaxed", "cta")
+  IRIS_ATOM64_CASE(IRIS_SEM_RELAXED, IRIS_SCOPE_GPU, "relaxed", "gpu")
+  IRIS_ATOM64_CASE(IRIS_SEM_RELAXED, IRIS_SCOPE_SYS, "relaxed", "sys")
+  IRIS_ATOM64_CASE(IRIS_SEM_ACQUIRE, IRIS_SCOPE_BLOCK, "acquire", "cta")
+  IRIS_ATOM64_CASE(IRIS_SEM_ACQUIRE, IRIS_SCOPE_GPU, "acquire", "gpu")
+  IRIS_ATOM64_CASE(IRIS_SEM_ACQUIRE, IRIS_SCOPE_SYS, "acquire", "sys")
+  IRIS_ATOM64_CASE(IRIS_SEM_RELEASE, IRIS_SCOPE_BLOCK, "release", "cta")
+  IRIS_ATOM64_CASE(IRIS_SEM_RELEASE, IRIS_SCOPE_GPU, "release", "gpu")
+  IRIS_ATOM64_CASE(IRIS_SEM_RELEASE, IRIS_SCOPE_SYS, "release", "sys")
+  IRIS_ATOM64_CASE(IRIS_SEM_ACQ_REL, IRIS_SCOPE_BLOCK, "acq_rel", "cta")
+  IRIS_ATOM64_CASE(IRIS_SEM_ACQ_REL, IRIS_SCOPE_GPU, "acq_rel", "gpu")
+  IRIS_ATOM64_CASE(IRIS_SEM_ACQ_REL, IRIS_SCOPE_SYS, "acq_rel", "sys")
+  return old;
+}
+#undef IRIS_ATOM64_CASE
+
+template <bool IS_CAS>
+__global__ void __launch_bounds__(256) atomic_vec64_kernel(const __grid_constant__ HeapTable tab, uint64_t ptr, size_t count, size_t stride, int from_rank,
+                                                           int to_rank, uint64_t cmp, uint64_t val, int sem, int scope, uint64_t* old_out) {
+  const uint64_t p = translate(ptr, from_rank, to_rank, tab);
+  for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < count; i += (size_t)gridDim.x * blockDim.x) {
+    const uint64_t old = atomic_rmw64<IS_CAS>(reinterpret_cast<uint64_t*>(p + i * stride), cmp, val, sem, scope);
+    if (old_out) old_out[i] = old;
+  }
+}
+
 template <bool IS_CAS>
 __global__ void __launch_bounds__(256) atomic_contended_kernel(const __grid_constant__ HeapTable tab, uint64_t ptr, size_t threads, int from_rank, int to_rank,
                                                                int32_t cmp, int32_t val, int sem, int scope, int32_t* old_out) {
@@ -164,8 +204,11 @@ static int check_region(const iris_heap* h, const void* p, int rank, size_t rows
   const uint64_t base = (uint64_t)(h->base + (size_t)rank * h->bytes_per_rank);
   const uint64_t a = (uint64_t)p;
   if (a < base || a - base >= h->bytes_per_rank) return fail(IRIS_ERR_RANGE, "%s: address is outside rank %d's heap", what, rank);
-  const uint64_t span = (rows - 1) * pitch + row_bytes;
-  if (span > h->bytes_per_rank - (a - base)) return fail(IRIS_ERR_RANGE, "%s: region leaves rank %d's heap", what, rank);
+  // span = (rows - 1) * pitch + row_bytes must fit in what is left of the slot; compared by division so that huge
+  // rows / pitch values cannot wrap the product
+  const uint64_t avail = h->bytes_per_rank - (a - base);
+  if (row_bytes > avail || (rows > 1 && pitch > 0 && (uint64_t)(rows - 1) > (avail - row_bytes) / pitch))
+    return fail(IRIS_ERR_RANGE, "%s: region leaves rank %d's heap", what, rank);
   return IRIS_OK;
 }
 
@@ -212,13 +255,15 @@ static int move2d(iris_heap* h, const void* src, void* dst, size_t rows, size_t 
   return IRIS_OK;
 }
 
-static int atomic_common(iris_heap* h, void* ptr, size_t count, size_t stride, int from_rank, int to_rank, int sem, int scope, const char* name) {
+static int atomic_common(iris_heap* h, void* ptr, size_t count, size_t stride, int from_rank, int to_rank, int sem, int scope, const char* name,
+                         size_t word = 4) {
   if (!heap_ok(h)) return fail(IRIS_ERR_STATE, "%s: bad heap handle", name);
   if (from_rank < 0 || from_rank >= h->world || to_rank < 0 || to_rank >= h->world) return fail(IRIS_ERR_ARG, "%s: rank out of range", name);
   if (sem < IRIS_SEM_RELAXED || sem > IRIS_SEM_ACQ_REL || scope < IRIS_SCOPE_BLOCK || scope > IRIS_SCOPE_SYS) return fail(IRIS_ERR_ARG, "%s: bad sem/scope", name);
   if (count == 0) return 1;  // nothing to do
-  if (!ptr || (uint64_t)ptr % 4 != 0 || stride % 4 != 0 || (count > 1 && stride == 0)) return fail(IRIS_ERR_ARG, "%s: pointer/stride must be 4-byte aligned", name);
-  return check_region(h, ptr, from_rank, count, 4, stride ? stride : 4, name);
+  if (!ptr || (uint64_t)ptr % word != 0 || stride % word != 0 || (count > 1 && stride == 0))
+    return fail(IRIS_ERR_ARG, "%s: pointer/stride must be %zu-byte aligned", name, word);
+  return check_region(h, ptr, from_rank, count, word, stride ? stride : word, name);
 }
 
 }  // namespace iris
@@ -276,6 +321,24 @@ int iris_atomic_cas(iris_heap* h, void* ptr, size_t count, size_t stride, int fr
   int rc = atomic_common(h, ptr, count, stride, from_rank, to_rank, sem, scope, "iris_atomic_cas");
   if (rc != IRIS_OK) return rc > 0 ? IRIS_OK : rc;
   atomic_vec_kernel<true><<<grid_for(h, count, 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(h->table(), (uint64_t)ptr, count, stride, from_rank, to_rank, compare, value, sem, scope, old_out);
+  IRIS_CUDA_TRY(cudaGetLastError());
+  return IRIS_OK;
+}
+
+int iris_atomic_add_u64(iris_heap* h, void* ptr, size_t count, size_t stride, int from_rank, int to_rank, uint64_t value, int sem, int scope,
+                        uint64_t* old_out, void* stream) {
+  int rc = atomic_common(h, ptr, count, stride, from_rank, to_rank, sem, scope, "iris_atomic_add_u64", 8);
+  if (rc != IRIS_OK) return rc > 0 ? IRIS_OK : rc;
+  atomic_vec64_kernel<false><<<grid_for(h, count, 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(h->table(), (uint64_t)ptr, count, stride, from_rank, to_rank, 0, value, sem, scope, old_out);
+  IRIS_CUDA_TRY(cudaGetLastError());
+  return IRIS_OK;
+}
+
+int iris_atomic_cas_u64(iris_heap* h, void* ptr, size_t count, size_t stride, int from_rank, int to_rank, uint64_t compare, uint64_t value, int sem,
+                        int scope, uint64_t* old_out, void* stream) {
+  int rc = atomic_common(h, ptr, count, stride, from_rank, to_rank, sem, scope, "iris_atomic_cas_u64", 8);
+  if (rc != IRIS_OK) return rc > 0 ? IRIS_OK : rc;
+  atomic_vec64_kernel<true><<<grid_for(h, count, 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(h->table(), (uint64_t)ptr, count, stride, from_rank, to_rank, compare, value, sem, scope, old_out);
   IRIS_CUDA_TRY(cudaGetLastError());
   return IRIS_OK;
 }

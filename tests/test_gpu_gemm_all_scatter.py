@@ -261,9 +261,8 @@ def test_short_form_and_host_entry_point():
     flag_off = (M * N * 2 + 255) // 256 * 256
     lock_off = flag_off + (nt * 4 + 255) // 256 * 256
     assert bpr == lock_off + (nt * 4 + 255) // 256 * 256 + 256
-    with GpuHeap(W, bpr) as g:
+    with GpuHeap(W, bpr) as g:                                         # backing bytes pre-filled with 0xA5: stale flags and locks
         dA, dB = dev16(A), [dev16(b) for b in Bs]
-        iris.iris_flags_fill(g.h, lock_off, nt, 0)
         for i, mode in enumerate(MODES):
             iris.gemm_all_scatter(dA, dB, g.h, M, N, K, W, mode)       # default stream
             iris.iris_status_check(g.h, 0)
@@ -283,11 +282,37 @@ def test_short_form_and_host_entry_point():
     assert out_off == bpr - 256
     bias = inputs.vector(9, inputs.STREAM_BIAS, N, "smallint:2", "bf16")
     with GpuHeap(W, out_off + M * N * 2) as g:
-        iris.iris_flags_fill(g.h, lock_off, nt, 0)
         C_host, OUT_host = np.empty((M, N), dtype=np.uint16), np.empty((M, N), dtype=np.uint16)
         iris.iris_gemm_all_scatter_host(A, Bs, C_host, None, bias, OUT_host, g.h, M, N, K, W, iris.IRIS_MODE_FUSED_SEQUENTIAL,
                                         iris.IRIS_BF16, 0)
         assert np.array_equal(C_host, c_ref) and np.array_equal(OUT_host, oracle.consume_bias_rows(c_ref, bias, "bf16"))
+
+
+def test_short_form_clears_stale_flags_and_locks_when_its_layout_changes():
+    """The short form places flags and locks itself, so it also initialises them: on a heap whose bytes are a non-zero
+    pattern (locks that are neither 0, 1 nor 2; flags far above any epoch), in the workgroup-specialised schedule, first
+    for one shape and then for a smaller one whose lock array lands inside the first shape's C."""
+    W, K = 2, 128
+    shapes = [(512, 1024), (256, 512)]
+    bpr = iris.iris_gemm_heap_bytes(*shapes[0], W)
+    with GpuHeap(W, bpr, fill=0x7B) as g:
+        epoch = 0
+        for M, N in shapes:
+            A, Bs = inputs.gemm_inputs(13, W, M, N, K, "smallint:2", "bf16")
+            c_ref = oracle.gemm_block(A, Bs, "bf16")
+            nt = oracle.num_tiles(M, N, W)
+            flag_off = (M * N * 2 + 255) // 256 * 256
+            lock_off = flag_off + (nt * 4 + 255) // 256 * 256
+            dA, dB = dev16(A), [dev16(b) for b in Bs]
+            for _ in range(2):
+                iris.gemm_all_scatter(dA, dB, g.h, M, N, K, W, iris.IRIS_MODE_WORKGROUP_SPECIALIZED)
+                iris.iris_status_check(g.h, 0)
+                epoch += 1
+                host = g.to_host()
+                for s in range(W):
+                    assert np.array_equal(c_slot(host, g, s, 0, M, N), c_ref)
+                    assert np.all(host[s * bpr + flag_off: s * bpr + flag_off + nt * 4].view(np.int32) == epoch)
+                    assert np.all(host[s * bpr + lock_off: s * bpr + lock_off + nt * 4].view(np.int32) == 0)
 
 
 STREAMK_SHAPES = [
@@ -407,9 +432,8 @@ def test_host_buffer_call_pipelined_over_blocks(mode, W, M, nl, K):
     bpr = out_off + (M * N * 2 + 255) // 256 * 256 + 256
     with GpuHeap(W, bpr) as g:
         img = g.image()
-        for s in range(W):
-            img.view(s, lock_off, nt * 4, np.int32)[:] = 0
-        iris.iris_flags_fill(g.h, lock_off, nt, 0)
+        for s in range(W):                       # the call clears its own flag and lock arrays (in whole 256-byte units)
+            img.view(s, flag_off, out_off - flag_off)[:] = 0
         C_host, OUT_host = np.zeros((M, N), dtype=np.uint16), np.zeros((M, N), dtype=np.uint16)
         flags = np.zeros((W, nt), dtype=np.int32)
         for call in (1, 2):                      # the second call reuses the handle's streams, events and staging

@@ -116,6 +116,61 @@ def test_atomic_vector_forms_match_oracle(sem, scope):
         assert np.array_equal(g.to_host(), img.mem)
 
 
+@pytest.mark.parametrize("sem", [iris.IRIS_SEM_RELAXED, iris.IRIS_SEM_ACQUIRE, iris.IRIS_SEM_RELEASE, iris.IRIS_SEM_ACQ_REL])
+@pytest.mark.parametrize("scope", [iris.IRIS_SCOPE_BLOCK, iris.IRIS_SCOPE_GPU, iris.IRIS_SCOPE_SYS])
+def test_u64_atomic_vector_forms_match_oracle(sem, scope):
+    """atomic_add / atomic_cas on uint64 words: previous values and the whole heap image equal the oracle's, with
+    operands that carry out of the low 32 bits and wrap at 2**64."""
+    with GpuHeap(3, 1 << 16, fill=0) as g:
+        img = g.image(fill=0)
+        n, stride, off = 777, 16, 512
+        rng = np.random.default_rng(21)
+        init = rng.integers(0, 2**64, n, dtype=np.uint64)
+        init[:3] = [2**64 - 1, 2**32 - 1, 0]
+        words = np.zeros(n * 2, dtype=np.uint64)
+        words[::2] = init
+        g.write(2, off, words)
+        img.view(2, off, n * stride, np.uint64)[:] = words
+        old = torch.empty(n, dtype=torch.int64, device="cuda")
+        for val in (1, 2**32 + 3, 2**64 - 1):
+            iris.iris_atomic_add_u64(g.h, g.addr(0, off), n, stride, 0, 2, val, sem, scope, old)
+            assert np.array_equal(old.cpu().numpy().view(np.uint64), img.atomic_add_u64(off, n, stride, 2, val))
+        cur = img.view(2, off, n * stride, np.uint64)[::2].copy()
+        target = int(cur[5])
+        iris.iris_atomic_cas_u64(g.h, g.addr(1, off), n, stride, 1, 2, target, 42, sem, scope, old)   # hits where the word equals cur[5]
+        assert np.array_equal(old.cpu().numpy().view(np.uint64), img.atomic_cas_u64(off, n, stride, 2, target, 42))
+        iris.iris_atomic_cas_u64(g.h, g.addr(1, off), n, stride, 1, 2, target ^ (1 << 40), 43, sem, scope, old)   # differs in the high half only
+        assert np.array_equal(old.cpu().numpy().view(np.uint64), img.atomic_cas_u64(off, n, stride, 2, target ^ (1 << 40), 43))
+        assert np.array_equal(g.to_host(), img.mem)
+        for bad in (dict(ptr=g.addr(0, off + 4)), dict(stride=12)):        # 8-byte alignment of address and stride
+            with pytest.raises(iris.IrisError) as e:
+                iris.iris_atomic_add_u64(g.h, bad.get("ptr", g.addr(0, off)), 2, bad.get("stride", 8), 0, 1, 1)
+            assert e.value.code == iris.IRIS_ERR_ARG
+        with pytest.raises(iris.IrisError) as e:
+            iris.iris_atomic_cas_u64(g.h, g.addr(0, (1 << 16) - 8), 2, 8, 0, 1, 0, 1)
+        assert e.value.code == iris.IRIS_ERR_RANGE
+        assert np.array_equal(g.to_host(), img.mem)
+
+
+def test_region_checks_do_not_wrap_on_huge_sizes():
+    """rows, pitch and count large enough to wrap a 64-bit product are refused with IRIS_ERR_RANGE before any launch."""
+    with GpuHeap(2, 4096) as g:
+        before = g.to_host().copy()
+        with pytest.raises(iris.IrisError) as e:
+            iris.iris_put_tile(g.h, g.addr(0, 0), g.addr(0, 2048), 2**62, 4, 4, 4, 0, 1)
+        assert e.value.code == iris.IRIS_ERR_RANGE
+        with pytest.raises(iris.IrisError) as e:
+            iris.iris_get_tile(g.h, g.addr(0, 0), g.addr(0, 2048), 2**61 + 1, 8, 8, 8, 0, 1)
+        assert e.value.code == iris.IRIS_ERR_RANGE
+        with pytest.raises(iris.IrisError) as e:
+            iris.iris_atomic_add(g.h, g.addr(0, 0), 2**62, 4, 0, 1, 1)
+        assert e.value.code == iris.IRIS_ERR_RANGE
+        with pytest.raises(iris.IrisError) as e:
+            iris.iris_atomic_add_u64(g.h, g.addr(0, 0), 2**61, 8, 0, 1, 1)
+        assert e.value.code == iris.IRIS_ERR_RANGE
+        assert np.array_equal(g.to_host(), before)
+
+
 def test_contended_atomics_invariants():
     with GpuHeap(2, 4096, fill=0) as g:
         n = 100000

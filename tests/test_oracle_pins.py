@@ -279,6 +279,32 @@ def test_atomics_sequential_semantics():
     assert list(olds) == [0, 0, 0, 0] and list(img.view(0, 32, 32, np.int32)[::2]) == [-2] * 4
 
 
+def test_u64_atomics_against_python_integers():
+    """64-bit add wraps modulo 2**64 and returns the previous word; cas writes only on a match.  Checked against python's
+    unbounded integers (reduced mod 2**64) on values that overflow 32 bits and 64 bits, strided, in one rank only."""
+    rng = np.random.default_rng(11)
+    n, stride, off = 33, 16, 64
+    init = [int(x) for x in rng.integers(0, 2**64, n, dtype=np.uint64)]
+    init[0], init[1], init[2] = 2**64 - 1, 2**32 - 1, 0
+    img = oracle.HeapImage(3, 1024)
+    img.view(2, off, n * stride, np.uint64)[::2] = np.array(init, dtype=np.uint64)
+    for val in (1, 2**32, 2**63 + 5, 2**64 - 1):
+        old = img.atomic_add_u64(off, n, stride, 2, val)
+        assert [int(x) for x in old] == init
+        init = [(x + val) % 2**64 for x in init]
+        assert [int(x) for x in img.view(2, off, n * stride, np.uint64)[::2]] == init
+    assert not img.view(2, off, n * stride, np.uint64)[1::2].any()          # the words between the strided ones
+    assert not img.slot(0).any() and not img.slot(1).any()                  # other ranks untouched
+    # cas: the high half alone must not match
+    word = 0x1234_5678_9ABC_DEF0
+    img.view(1, 8, 8, np.uint64)[0] = word
+    assert int(img.atomic_cas_u64(8, 1, 8, 1, word & 0xFFFFFFFF, 7)[0]) == word and int(img.view(1, 8, 8, np.uint64)[0]) == word
+    assert int(img.atomic_cas_u64(8, 1, 8, 1, word ^ (1 << 63), 7)[0]) == word and int(img.view(1, 8, 8, np.uint64)[0]) == word
+    assert int(img.atomic_cas_u64(8, 1, 8, 1, word, 2**64 - 2)[0]) == word and int(img.view(1, 8, 8, np.uint64)[0]) == 2**64 - 2
+    with pytest.raises(ValueError):
+        img.atomic_add_u64(1024 - 4, 1, 8, 0, 1)                            # the word would leave the slot
+
+
 def test_remaining_atomics_against_numpy_semantics():
     rng = np.random.default_rng(9)
     init = rng.integers(-2**31, 2**31 - 1, 64, dtype=np.int64).astype(np.int32)

@@ -35,8 +35,12 @@ def _reference_run(W, M, N, K, dtype, A, Bs, epoch):
         return (host[:, c_off:c_off + M * N * 2].copy(), host[:, flag_off:flag_off + nt * 4].copy())
 
 
-def test_noalloc_matches_regular_entry_point_twice_in_a_row():
-    W, M, nl, K, dtype = 4, 520, 392, 328, "bf16"          # several tiles, ragged in M, N_local and K
+@pytest.mark.parametrize("W,M,nl,K,dtype", [
+    (4, 520, 392, 328, "bf16"),      # 128-wide compute tiles; several tiles, ragged in M, N_local and K
+    (8, 640, 512, 192, "fp16"),      # N_local a multiple of 256 and more tiles than SMs: the 256-wide kernel, five tile rows
+    (2, 900, 1280, 136, "bf16"),     # 256-wide kernel (160 narrow tiles would not fit one wave), ragged M and K
+], ids=["bn128_bf16", "bn256_fp16", "bn256_bf16_ragged"])
+def test_noalloc_matches_regular_entry_point_twice_in_a_row(W, M, nl, K, dtype):
     N = W * nl
     c_off, flag_off, _, _, bpr = gemm_layout(M, N, W)
     nt = oracle.num_tiles(M, N, W)
