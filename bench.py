@@ -53,9 +53,39 @@ DEFAULT_WORKLOAD = "cfg5_w8_m8192_n16384_k16384"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 METRIC = "gemm_all_scatter_tflops"
 UNIT = "TFLOP/s"
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one workgroup_specialized launch on the default
-# workload, from a 1-pass ncu capture at full size: 4.74 GB read + 2.10 GB written.
-NCU_TRAFFIC_BYTES = {"cfg5_w8_m8192_n16384_k16384": 6.84e9}
+# DRAM traffic of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum per launch) is not typed in here: it is
+# read from the ncu summary under profiles/ that records it together with a digest of the kernel sources it was taken on.
+TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "gemm_all_scatter_dram_traffic.md")
+KERNEL_SOURCES = ["gemm_all_scatter.cu", "sm100_ptx.cuh", "iris_device.cuh", "iris_internal.h"]
+
+
+def kernel_sources_digest() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2511_12500_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(workload: str, mode: str):
+    """(bytes per launch or None, note) from the tracked ncu record; None when there is no record for this workload and
+    schedule or when the kernel sources have changed since it was captured."""
+    try:
+        text = open(TRAFFIC_RECORD).read()
+    except OSError:
+        return None, "no ncu record under profiles/"
+    for block in text.split("\n## ")[1:]:
+        kv = {}
+        for line in block.splitlines():
+            if ":" in line and line.startswith("- "):
+                k, v = line[2:].split(":", 1)
+                kv[k.strip()] = v.strip()
+        if kv.get("workload") == workload and kv.get("mode") == mode:
+            if kv.get("kernel_sources_sha256") != kernel_sources_digest():
+                return None, f"ncu record is for older kernel sources (commit {kv.get('commit', '?')}); not carried over"
+            return float(kv["dram_bytes_read"]) + float(kv["dram_bytes_write"]), f"ncu 1-pass capture at commit {kv.get('commit', '?')}"
+    return None, "no ncu record for this workload and schedule"
 
 
 def peaks():
@@ -242,6 +272,7 @@ def run_ours(args):
     store_bytes = float(W) * M * N * 2
 
     def gemm(epoch, m=mode, fused=False, wg_tail=None, **kw):
+        kw.setdefault("stream", None)
         iris.iris_gemm_all_scatter_ex(h, dA, dB, M, N, K, W, m, dt, 0, flag_off, lock_off, epoch, comm_ctas=args.comm_ctas,
                                       raster_group=args.raster_group, block_n=args.block_n, cta_pair=args.cta_pair, static_schedule=args.static_schedule, stream_k=args.stream_k,
                                       wg_tail=args.wg_tail if wg_tail is None else wg_tail,
@@ -312,15 +343,46 @@ def run_ours(args):
         t_store = store_bytes / (pk["hbm_gbs"] * 1e9) * 1e3
         t_bytes = ((M * K + N * K) * 2.0 + store_bytes) / (pk["hbm_gbs"] * 1e9) * 1e3   # operand reads + replicated stores
         achieved = flops / (gemm_ms * 1e-3) / 1e12
+        traffic, traffic_note = recorded_traffic(args.workload, args.mode)
         result["roofline"] = {"kernel": f"gemm_all_scatter_pair_kernel<bf16> ({args.mode}); single-CTA kernel when --cta-pair -1 or the shape needs it", "bound": "tensor", "achieved": achieved,
                               "peak": pk["bf16_tflops"], "unit": "TFLOP/s", "frac": achieved / pk["bf16_tflops"],
                               "peak_kind": f"{pk_kind} burst (of {pk_kind})", "peak_sustained": pk["bf16_tflops_sustained"],
-                              "frac_sustained": achieved / pk["bf16_tflops_sustained"], "traffic": NCU_TRAFFIC_BYTES.get(args.workload) if args.mode == "workgroup_specialized" else None,
+                              "traffic": traffic, "traffic_note": traffic_note,
                               "algorithmic_bytes": (M * K + N * K) * 2.0 + store_bytes,
                               "kernel_ms": gemm_ms, "combined_roofline_ms": max(t_tensor, t_store),
                               "frac_of_combined_roofline": max(t_tensor, t_store) / gemm_ms,
                               "full_traffic_roofline_ms": max(t_tensor, t_bytes), "frac_of_full_traffic_roofline": max(t_tensor, t_bytes) / gemm_ms,
                               "replicated_store_gbs": store_bytes / (gemm_ms * 1e-3) / 1e9}
+        # ---------------- the same kernel in steady state: >= 1 s of back-to-back launches under the power cap ----------------
+        # (the timed region above may last well under 100 ms, during which the clocks are still on their way down)
+        if args.steady_seconds > 0:
+            n_steady = max(10, int(np.ceil(args.steady_seconds * 1e3 / max(gemm_ms, 1e-3))))
+            s2 = ClockSampler(local_rank)
+            s2.start()
+            for _ in range(3):
+                epoch += 1
+                gemm(epoch)
+            time.sleep(0.3)               # nvidia-smi needs a moment before its first line
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            s2.mark()
+            e0.record(stream)
+            for _ in range(n_steady):
+                epoch += 1
+                gemm(epoch)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ck = s2.stop()
+            iris.iris_status_check(h)
+            sms = e0.elapsed_time(e1) / n_steady
+            st_ach = flops / (sms * 1e-3) / 1e12
+            result["roofline"]["steady"] = {"launches": n_steady, "seconds": sms * n_steady * 1e-3, "kernel_ms": sms, "achieved": st_ach,
+                                            "frac": st_ach / pk["bf16_tflops"], "frac_vs_sustained": st_ach / pk["bf16_tflops_sustained"],
+                                            "sm_mhz": ck.get("sm_mhz"), "clock_samples": ck.get("samples"), "reasons": ck.get("reasons"),
+                                            "power_w_max": ck.get("power_w_max"),
+                                            "ms_times_mhz": (sms * ck["sm_mhz"]) if ck.get("sm_mhz") else None,
+                                            "note": "back-to-back launches of the dominant kernel alone; frac against the burst peak, frac_vs_sustained "
+                                                    "against the peak measured the same way (a seconds-long loop)"}
         cons_bytes = 2.0 * store_bytes + N * 2
         if fused:   # time the stand-alone consumer kernel too, for its own HBM figure
             ts = []
@@ -343,7 +405,9 @@ def run_ours(args):
         variants = list(iris.MODES.items()) + [("workgroup_specialized_every_tile_via_comm_ctas", iris.IRIS_MODE_WORKGROUP_SPECIALIZED)]
         tA = dA.view(torch.bfloat16 if dtype == "bf16" else torch.float16).view(M, K)
         tB = torch.cat([b.view(tA.dtype).view(nl, K) for b in dB], dim=0)
+        variants.append(("unfused_two_streams", "unfused"))   # Section 4.1: producers and communication kernel as two launches
         variants.append(("library_gemm_no_scatter", None))   # context: cuBLAS through torch.matmul, same operands, same moment
+        comm_stream = torch.cuda.Stream()
         series = {name: [] for name, _ in variants}
         for it in range(1 + args.mode_iters if args.mode_iters > 0 else 0):
             for name, m in variants:
@@ -352,6 +416,8 @@ def run_ours(args):
                 e0.record(stream)
                 if m is None:
                     tC = tA @ tB.t()
+                elif m == "unfused":
+                    gemm(epoch, iris.IRIS_MODE_WORKGROUP_SPECIALIZED, stream=stream, comm_stream=comm_stream)   # `stream` joins the second one
                 else:
                     gemm(epoch, m, wg_tail=-1 if name.endswith("comm_ctas") else None)
                 e1.record(stream)
@@ -374,6 +440,34 @@ def run_ours(args):
                 modes[name]["half_tiles_kept_by_producers_before_the_last_wave"] = kept[name]
         iris.iris_status_check(h)
         result["modes"] = modes
+
+        # ---------------- consumer launched on a second stream right after the producer (it overlaps the GEMM) ----------------
+        # End-to-end time from the producer's launch to the end of the last kernel, next to the same two kernels on one stream.
+        if args.mode_iters > 0:
+            cons_stream = torch.cuda.Stream()
+            joined = torch.cuda.Event()
+            ts2, ts1 = [], []
+            for it in range(1 + args.mode_iters):
+                for overlapped in (True, False):
+                    epoch += 1
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    torch.cuda.synchronize()
+                    e0.record(stream)
+                    gemm(epoch)
+                    if overlapped:
+                        iris.iris_consume_bias(h, 0, out_off, flag_off, dbias, M, N, W, dt, epoch, stream=cons_stream)
+                        joined.record(cons_stream)
+                        stream.wait_event(joined)
+                    else:
+                        consume(epoch)
+                    e1.record(stream)
+                    torch.cuda.synchronize()
+                    if it > 0:
+                        (ts2 if overlapped else ts1).append(e0.elapsed_time(e1))
+            iris.iris_status_check(h)
+            result["consumer_on_second_stream"] = {"ms": float(np.median(ts2)), "ms_min": float(min(ts2)), "tflops": flops / float(np.median(ts2)) / 1e9,
+                                                   "same_two_kernels_on_one_stream_ms": float(np.median(ts1)),
+                                                   "note": "producer kernel on one stream, iris_consume_bias on a second stream right after it; first launch to last kernel done"}
 
         # ---------------- the same step with the consumer's warps inside the GEMM launch ----------------
         if not fused and args.mode != "bulk_synchronous":
@@ -482,7 +576,8 @@ def oracle_all_store_sample(S=4 << 20, W=8):
 
 def all_store_sweep(iris, pk, kind, pull=0):
     """W=8 all-store (push) or all-load (pull): message sizes 1 KiB .. (64 MiB | 1 GiB) in powers of 4.
-    GB/s counts W*S read + W*W*S written (push) or W*W*S read + W*W*S written (pull)."""
+    GB/s counts the HBM-side bytes, W*S read + W*W*S written, in both forms; the pull form also reports the bytes its
+    loads request (W*W*S read + W*W*S written) as the L2-side rate."""
     import torch
     W = 8
     top = 15 if kind == "full" else 13
@@ -515,9 +610,20 @@ def all_store_sweep(iris, pk, kind, pull=0):
         torch.cuda.synchronize()
         iris.iris_status_check(h)
         ms = e0.elapsed_time(e1) / iters
-        moved = float((W * W * S if pull else W * S) + W * W * S)
-        out.append({"S": S, "ms": ms, "gbs": moved / ms / 1e6, "frac_of_hbm_peak": moved / ms / 1e6 / pk["hbm_gbs"],
-                    "l2": "warm (working set below L2)" if W * W * S < (100 << 20) else "exceeds L2"})
+        # HBM-side bytes: every source block is fetched from DRAM once (W*S) however many ranks read it; W*W*S are written.
+        # The pull form issues W*W*S of reads, of which all but W*S are served by L2: reported separately as l2_side_gbs.
+        hbm_bytes = float(W * S + W * W * S)
+        row = {"S": S, "ms": ms, "gbs": hbm_bytes / ms / 1e6, "frac_of_hbm_peak": hbm_bytes / ms / 1e6 / pk["hbm_gbs"],
+               "l2": "warm (working set below L2)" if W * W * S < (100 << 20) else "exceeds L2"}
+        if pull:
+            l2_bytes = float(2 * W * W * S)
+            row["l2_side_gbs"] = l2_bytes / ms / 1e6
+            row["l2_side_frac_of_hbm_peak"] = l2_bytes / ms / 1e6 / pk["hbm_gbs"]
+            if row["l2_side_frac_of_hbm_peak"] > 1.0:
+                row["l2_side_note"] = "L2-served: W-1 of the W reads of each block hit in L2, so this figure is not an HBM rate"
+        if row["frac_of_hbm_peak"] > 1.0:
+            row["note"] = "L2-served (working set fits the 126 MB L2): not an HBM rate"
+        out.append(row)
         iris.iris_heap_destroy(h)
         del mem
         torch.cuda.empty_cache()
@@ -588,6 +694,7 @@ def main():
     ap.add_argument("--stream-k", type=int, default=0)
     ap.add_argument("--wg-tail", type=int, default=0, help="workgroup_specialized: 0 = producers scatter the last wave themselves, -1 = never, n = last n tiles")
     ap.add_argument("--mode-iters", type=int, default=3)
+    ap.add_argument("--steady-seconds", type=float, default=1.0, help="length of the back-to-back loop behind roofline.steady (0 = skip)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--cpu-strips", type=int, default=32)
     ap.add_argument("--sweep", default="short", choices=["none", "short", "full"])

@@ -58,6 +58,12 @@ enum { IRIS_SCOPE_BLOCK = 0, IRIS_SCOPE_GPU = 1, IRIS_SCOPE_SYS = 2 };
 /* Read-modify-write atomics of Table 3 (atomic_cas has its own call). min / max compare as signed int32. */
 enum { IRIS_OP_ADD = 0, IRIS_OP_XCHG = 1, IRIS_OP_AND = 2, IRIS_OP_OR = 3, IRIS_OP_XOR = 4, IRIS_OP_MIN = 5, IRIS_OP_MAX = 6 };
 
+/* Storage of a B shard (iris_gemm_args.b_layout). */
+enum {
+  IRIS_B_N_BY_K = 0, /* [N/W, K], K contiguous: the K x N_local operand stored column-major            */
+  IRIS_B_K_BY_N = 1  /* [K, N/W] row-major, N contiguous: Listing 2's K x N_local operand as printed   */
+};
+
 #define IRIS_MAX_WORLD 8
 #define IRIS_TILE 128 /* publication tile edge: one ready flag per 128 x 128 block of C */
 
@@ -213,9 +219,9 @@ int iris_all_store_bench(iris_heap* heap, uint64_t payload_off, uint64_t recv_of
  */
 typedef struct iris_gemm_args {
   const void* A;               /* device: [M, K] row-major, K contiguous, 16-byte aligned        */
-  const void* const* B_shards; /* HOST array of `world` DEVICE pointers; shard r is [N/W, K] with
-                                  K contiguous (= the K x N_local operand of Listing 2 stored
-                                  column-major), 16-byte aligned                                 */
+  const void* const* B_shards; /* HOST array of `world` DEVICE pointers, each 16-byte aligned; shard r
+                                  is [N/W, K] with K contiguous (= the K x N_local operand of
+                                  Listing 2 stored column-major) unless b_layout says otherwise  */
   iris_heap* heap;
   int M, N, K;                 /* N = global width; N % world == 0, (N/world) % 8 == 0, K % 8 == 0;
                                   M, N, K >= 0 (an empty problem publishes nothing and succeeds) */
@@ -276,11 +282,34 @@ typedef struct iris_gemm_args {
                                   workgroup_specialized), or as a following kernel otherwise.
                                   Device pointer to N elements, 16-byte aligned                  */
   uint64_t consumer_out_off;   /* offset of OUT [M, N] in every slot (with consumer_bias)        */
+  int b_layout;                /* IRIS_B_N_BY_K (0): shards are [N/W, K], K contiguous;
+                                  IRIS_B_K_BY_N (1): shards are [K, N/W] row-major as Listing 2 prints
+                                  its B operand.  The tensor cores then read B as an MN-major
+                                  operand (transpose bit of the instruction descriptor, 64 x 64
+                                  shared-memory blocks); results are bit-identical to the other
+                                  layout's on the transposed data                                */
 } iris_gemm_args;
 
 /* Enqueue the whole operation on `stream` (bulk-synchronous: two kernels; otherwise one).
  * IRIS_ERR_ARG / IRIS_ERR_RANGE / IRIS_ERR_UNSUPPORTED are returned before any launch. */
 int iris_gemm_all_scatter_ex(const iris_gemm_args* args, void* stream);
+
+/* Unfused producer-consumer (Section 4.1 "Unfused producer-consumer"; Section 5.2 reports it as the best pattern on
+ * the paper's hardware): the workgroup-specialised schedule as TWO kernels on TWO streams with a partition of the
+ * SMs.  The GEMM kernel (producer CTAs only: tile -> owner slot -> lock 0 -> 1, release) is launched on
+ * producer_stream; the communication kernel (lock 1 -> 0, acquire; copy to the other W-1 slots; publish the flags),
+ * with comm_ctas CTAs -- at most what the producers leave free -- is launched right after it on comm_stream.
+ * args->mode must be IRIS_MODE_WORKGROUP_SPECIALIZED; comm_ctas, wg_tail and every other field mean what they mean
+ * for iris_gemm_all_scatter_ex, and the final heap image is the same.  consumer_bias is refused
+ * (IRIS_ERR_UNSUPPORTED): a consumer goes on a stream of its own (iris_consume_bias), where it overlaps both.
+ * Ordering: comm_stream first waits for what was enqueued on producer_stream before this call; after the call
+ * producer_stream waits for the communication kernel, so work enqueued on producer_stream afterwards (and
+ * iris_status_check on it) sees the finished scatter.  The two streams must differ.
+ * The dependency between the kernels runs one way (the second waits for locks the first sets, never the reverse)
+ * and every wait has the usual deadline: if the hardware starts the second kernel late the scatter merely
+ * overlaps less, and if it cannot run at all within spin_timeout_ns the call ends with IRIS_ERR_TIMEOUT in the
+ * status block, never with a hang. */
+int iris_gemm_all_scatter_unfused(const iris_gemm_args* args, void* producer_stream, void* comm_stream);
 
 /* The short form named by the problem statement.  bf16; C at offset 0 of every slot, flags at
  * align256(M*N*2), locks right after the flags (align256); epoch = a per-heap counter that starts

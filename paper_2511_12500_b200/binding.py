@@ -19,6 +19,7 @@ IRIS_SEM_RELAXED, IRIS_SEM_ACQUIRE, IRIS_SEM_RELEASE, IRIS_SEM_ACQ_REL = 0, 1, 2
 IRIS_SCOPE_BLOCK, IRIS_SCOPE_GPU, IRIS_SCOPE_SYS = 0, 1, 2
 IRIS_OP_ADD, IRIS_OP_XCHG, IRIS_OP_AND, IRIS_OP_OR, IRIS_OP_XOR, IRIS_OP_MIN, IRIS_OP_MAX = range(7)
 ATOMIC_OPS = {"add": 0, "xchg": 1, "and": 2, "or": 3, "xor": 4, "min": 5, "max": 6}
+IRIS_B_N_BY_K, IRIS_B_K_BY_N = 0, 1
 IRIS_MAX_WORLD = 8
 IRIS_TILE = 128
 
@@ -30,7 +31,7 @@ EXPORTS = [
     "iris_heap_bytes_per_rank", "iris_heap_base", "iris_heap_bases", "iris_malloc", "iris_heap_reset", "iris_translate",
     "iris_status_check", "iris_put_tile", "iris_get_tile", "iris_atomic_add", "iris_atomic_cas",
     "iris_atomic_add_contended", "iris_atomic_cas_contended", "iris_flags_fill", "iris_all_store_bench",
-    "iris_gemm_all_scatter_ex", "gemm_all_scatter", "iris_gemm_heap_bytes", "iris_heap_epoch", "iris_num_tiles",
+    "iris_gemm_all_scatter_ex", "iris_gemm_all_scatter_unfused", "gemm_all_scatter", "iris_gemm_heap_bytes", "iris_heap_epoch", "iris_num_tiles",
     "iris_consume_bias", "iris_consume_bias_ranks", "iris_gemm_all_scatter_host", "iris_gemm_out_offset", "iris_gemm_takeover_stats",
     "iris_gemm_all_scatter_noalloc", "iris_atomic_add_u64", "iris_atomic_cas_u64", "iris_copy_tile", "iris_load_tile", "iris_store_tile", "iris_atomic_rmw",
 ]
@@ -49,7 +50,7 @@ class GemmArgs(C.Structure):
         ("c_off", C.c_uint64), ("flag_off", C.c_uint64), ("lock_off", C.c_uint64),
         ("epoch", C.c_int32), ("comm_ctas", C.c_int), ("max_ctas", C.c_int), ("raster_group", C.c_int),
         ("block_n", C.c_int), ("spin_timeout_ns", C.c_uint64), ("cta_pair", C.c_int), ("static_schedule", C.c_int), ("stream_k", C.c_int), ("wg_tail", C.c_int), ("rank_first", C.c_int), ("rank_count", C.c_int), ("pace_stores", C.c_int),
-        ("consumer_bias", C.c_void_p), ("consumer_out_off", C.c_uint64),
+        ("consumer_bias", C.c_void_p), ("consumer_out_off", C.c_uint64), ("b_layout", C.c_int),
     ]
 
 
@@ -96,6 +97,7 @@ def lib() -> C.CDLL:
     L.iris_flags_fill.argtypes = [vp, u64, sz, i32, vp]
     L.iris_all_store_bench.argtypes = [vp, u64, u64, u64, sz, sz, i32, ci, ci, vp]
     L.iris_gemm_all_scatter_ex.argtypes = [C.POINTER(GemmArgs), vp]
+    L.iris_gemm_all_scatter_unfused.argtypes = [C.POINTER(GemmArgs), vp, vp]
     L.gemm_all_scatter.argtypes = [vp, C.POINTER(vp), vp, ci, ci, ci, ci, ci]
     L.iris_gemm_heap_bytes.restype = sz
     L.iris_gemm_heap_bytes.argtypes = [ci, ci, ci]
@@ -290,11 +292,20 @@ def _shards(B_shards):
 
 
 def iris_gemm_all_scatter_ex(heap, A, B_shards, M, N, K, world, mode, dtype, c_off, flag_off, lock_off=0, epoch=1,
-                             comm_ctas=0, max_ctas=0, raster_group=0, block_n=0, spin_timeout_ns=0, cta_pair=0, static_schedule=0, stream_k=0, wg_tail=0, rank_first=0, rank_count=0, pace_stores=0, consumer_bias=None, consumer_out_off=0, stream=None):
+                             comm_ctas=0, max_ctas=0, raster_group=0, block_n=0, spin_timeout_ns=0, cta_pair=0, static_schedule=0, stream_k=0, wg_tail=0, rank_first=0, rank_count=0, pace_stores=0, consumer_bias=None, consumer_out_off=0, b_layout=0, stream=None, comm_stream=None):
     arr = _shards(B_shards)
     a = GemmArgs(_ptr(A), C.cast(arr, C.POINTER(C.c_void_p)), heap, M, N, K, world, mode, dtype, c_off, flag_off, lock_off,
-                 epoch, comm_ctas, max_ctas, raster_group, block_n, spin_timeout_ns, cta_pair, static_schedule, stream_k, wg_tail, rank_first, rank_count, pace_stores, _ptr(consumer_bias), consumer_out_off)
-    _ck(lib().iris_gemm_all_scatter_ex(C.byref(a), _stream(stream)))
+                 epoch, comm_ctas, max_ctas, raster_group, block_n, spin_timeout_ns, cta_pair, static_schedule, stream_k, wg_tail, rank_first, rank_count, pace_stores, _ptr(consumer_bias), consumer_out_off, b_layout)
+    if comm_stream is not None:     # the two-kernel, two-stream form (producers on `stream`, communication kernel on `comm_stream`)
+        _ck(lib().iris_gemm_all_scatter_unfused(C.byref(a), _stream(stream), _stream(comm_stream)))
+    else:
+        _ck(lib().iris_gemm_all_scatter_ex(C.byref(a), _stream(stream)))
+
+
+def iris_gemm_all_scatter_unfused(heap, A, B_shards, M, N, K, world, dtype, c_off, flag_off, lock_off, epoch, producer_stream, comm_stream, **kw):
+    """Workgroup-specialised schedule as two kernels on two streams (see the header)."""
+    iris_gemm_all_scatter_ex(heap, A, B_shards, M, N, K, world, IRIS_MODE_WORKGROUP_SPECIALIZED, dtype, c_off, flag_off, lock_off, epoch,
+                             stream=producer_stream, comm_stream=comm_stream, **kw)
 
 
 def gemm_all_scatter(A, B_shards, heap, M, N, K, world, mode):

@@ -31,6 +31,7 @@ __global__ void __launch_bounds__(kConsThreads) consume_bias_kernel(const __grid
         const uint64_t start = globaltimer_ns();
         uint32_t spins = 0;
         while ((seen = ld_acquire_gpu(flag)) < epoch) {
+          __nanosleep(256);   // the tile is still being produced: leave the issue slots to whoever shares this SM
           if ((++spins & 31u) == 0 && globaltimer_ns() - start > timeout_ns) {
             report_timeout(status, KID_CONSUMER, t, s, seen, epoch);
             failed = 1;

@@ -48,9 +48,14 @@ constexpr int kPairBNc = 256;     // pair tile width (also used by the fused con
 constexpr int kSchedDepth = 4;    // pair kernel: tile ids in flight between the claiming thread and the other roles
 constexpr int kCommWarps = 6;     // communication CTA: every warp is a communicator with a 32 KB tile buffer
 constexpr int kTileBytes = IRIS_TILE * IRIS_TILE * 2;
+constexpr int kMnBlockBytes = 64 * BK * 2;   // B_r [K, N_local]: one [64 k][64 n] block of a stage, as its TMA box lands
 constexpr int kSmemPayload = 192 * 1024;
 constexpr int kSmemCtrl = 1024;
-constexpr int kSmemTotal = kSmemPayload + kSmemCtrl + 1024;  // + slack to align the base to 1024
+constexpr int kStoreBoxBytes = BM * 64 * 2;                 // 16 KB: 128 rows x 64 columns, one TMA store box (128B-swizzled rows)
+constexpr int kEpiStageBytes = 2 * kStoreBoxBytes;          // single-CTA kernel: 128 converted columns of a tile on their way out
+constexpr int kSmemTotal = kSmemPayload + kEpiStageBytes + kSmemCtrl + 1024;  // + slack to align the base to 1024
+constexpr int kCommSmemTotal = kSmemPayload + kSmemCtrl + 1024;               // the communication kernel of the two-stream form
+static_assert(kSmemTotal <= 232448, "shared memory per CTA");
 
 template <int BN>
 struct TileCfg {
@@ -61,11 +66,12 @@ struct TileCfg {
 
 struct alignas(64) GemmParams {
   CUtensorMap tmA;                    // A [M, K], box 64 x 128, 128B swizzle
-  CUtensorMap tmB[IRIS_MAX_WORLD];    // B_r [N_local, K], box 64 x BN, 128B swizzle
+  CUtensorMap tmB[IRIS_MAX_WORLD];    // B_r [N_local, K], box 64 x BN, 128B swizzle; or B_r [K, N_local], box 64 (n) x 64 (k), 128B swizzle
   CUtensorMap tmC[IRIS_MAX_WORLD];    // C of slot s viewed as [W][M][N_local], box 128 x 128 x 1, no swizzle
   CUtensorMap tmC4;                   // C of all slots as one tensor [slot][rank][M][N_local] (slots equally spaced: every heap
                                       // handle), box 128 x 128 x 1 x 1, no swizzle: the communication warps' copies
-  CUtensorMap tmC4s;                  // the same tensor, box 64 x 128 x 1 x 1, 128B swizzle: the pair kernel's epilogue stores
+  CUtensorMap tmC4s;                  // the same tensor, box 64 x 128 x 1 x 1, 128B swizzle: the epilogues' stores
+  CUtensorMap tmCs[IRIS_MAX_WORLD];   // slots at arbitrary addresses: C of slot s as [W][M][N_local], box 64 x 128 x 1, 128B swizzle
   int one_map;                        // 1 = tmC4 / tmC4s are valid; 0 = slots at arbitrary addresses, per-slot maps tmC[]
   HeapTable tab;
   uint64_t c_off, flag_off, lock_off;
@@ -95,6 +101,7 @@ struct alignas(64) GemmParams {
   int32_t* backlog;     // publication tiles handed over and not yet published ([0]), tiles kept by that rule ([1])
   uint32_t t_pt_ns;     // estimate: time a communication warp needs for one publication tile, its CTA's port shared by all warps
   uint32_t t_tile_ns;   // estimate: main-loop time of one compute tile
+  int b_mn;             // 1 = B_r is [K, N_local] row-major (N contiguous): 64 x 64 boxes, MN-major descriptor; 0 = [N_local, K]
   int pace_stores;      // pair kernel: 1 = the epilogue spreads a tile's box stores over most of the next tile's main loop
   int raster_group;
   int mode;
@@ -203,11 +210,11 @@ __device__ __forceinline__ int32_t* lock_addr(const GemmParams& p, int rank, int
 //   publish  lanes 0..W-1 write the tile's ready flag in slot `lane` with release semantics
 // ------------------------------------------------------------------------------------------------
 template <bool STATIC_LOCKS, int SUBS, int SUBS_M = 1>
-__device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload, int warp, int lane) {
+__device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload, int warp, int lane, int comm_block) {
   constexpr uint32_t kFull = 0xFFFFFFFFu;
   const int W = p.tab.world;
   const int ncw = p.comm_ctas * kCommWarps;
-  const int cw = ((int)blockIdx.x - p.gemm_ctas) * kCommWarps + warp;
+  const int cw = comm_block * kCommWarps + warp;   // comm_block: this CTA's index among the communication CTAs
   const int items = min(p.total_ctiles, p.seq_from) * SUBS * SUBS_M;   // the tail wave's tiles are scattered by their producers
   const int n_my = cw < items ? (items - cw + ncw - 1) / ncw : 0;  // items cw, cw + ncw, ...
   const int pt_n = W * p.ptiles_per_rank;
@@ -362,7 +369,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
   using Cfg = TileCfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* payload = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  CtrlBlock* ctrl = reinterpret_cast<CtrlBlock*>(payload + kSmemPayload);
+  CtrlBlock* ctrl = reinterpret_cast<CtrlBlock*>(payload + kSmemPayload + kEpiStageBytes);
   const int warp = (int)threadIdx.x / 32, lane = (int)threadIdx.x % 32;
   const bool is_comm = (int)blockIdx.x >= p.gemm_ctas;
   const int W = p.tab.world;
@@ -381,6 +388,9 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
     if (is_comm) {
       if (p.one_map) ptx::prefetch_tensormap(&p.tmC4);
       else for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmC[r]);
+    } else {
+      if (p.one_map) ptx::prefetch_tensormap(&p.tmC4s);
+      else for (int r = 0; r < W; ++r) ptx::prefetch_tensormap(&p.tmCs[r]);
     }
   }
   if (warp == 1 && !is_comm) {
@@ -392,7 +402,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
   ptx::tc_fence_after();
 
   if (is_comm) {
-    comm_cta<STATIC_LOCKS, BN / IRIS_TILE>(p, ctrl, payload, warp, lane);
+    comm_cta<STATIC_LOCKS, BN / IRIS_TILE>(p, ctrl, payload, warp, lane, (int)blockIdx.x - p.gemm_ctas);
   } else if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
@@ -409,7 +419,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
           uint8_t* sa = payload + stage * Cfg::kStageBytes;
           ptx::mbar_arrive_expect_tx(bar, Cfg::kStageBytes);
           ptx::tma_load_2d(ptx::smem_u32(sa), &p.tmA, kb * BK, tc.tm * BM, bar);
-          ptx::tma_load_2d(ptx::smem_u32(sa + BM * BK * 2), &p.tmB[tc.rank], kb * BK, tc.jn * BN, bar);
+          if (p.b_mn) {   // B_r [K, N_local]: one [64 k][64 n] block per 64 columns of the tile
+#pragma unroll
+            for (int nb = 0; nb < BN / 64; ++nb)
+              ptx::tma_load_2d(ptx::smem_u32(sa + BM * BK * 2 + nb * kMnBlockBytes), &p.tmB[tc.rank], tc.jn * BN + nb * 64, kb * BK, bar);
+          } else {
+            ptx::tma_load_2d(ptx::smem_u32(sa + BM * BK * 2), &p.tmB[tc.rank], kb * BK, tc.jn * BN, bar);
+          }
           if (++stage == Cfg::kStages) { stage = 0; phase ^= 1; }
         }
       }
@@ -417,7 +433,8 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-      constexpr uint32_t idesc = ptx::idesc_f16(BM, BN, BF16 ? 1 : 0);
+      const uint32_t idesc = ptx::idesc_f16(BM, BN, BF16 ? 1 : 0) | (p.b_mn ? ptx::kIdescBMnMajor : 0u);
+      const uint64_t b_kstep = p.b_mn ? (uint64_t)(2 * 1024 >> 4) : 2u;   // 16 k: two 8-row swizzle atoms (MN-major), or +32 bytes in the row (K-major)
       const uint32_t tmem_base = ctrl->tmem_base;
       int stage = 0, acc = 0;
       uint32_t phase = 0, acc_phase = 0;
@@ -433,10 +450,10 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
           ptx::tc_fence_after();
           const uint32_t sa = ptx::smem_u32(payload + stage * Cfg::kStageBytes);
           const uint64_t adesc = ptx::smem_desc_k_sw128(sa);
-          const uint64_t bdesc = ptx::smem_desc_k_sw128(sa + BM * BK * 2);
+          const uint64_t bdesc = p.b_mn ? ptx::smem_desc_mn_sw128(sa + BM * BK * 2, kMnBlockBytes) : ptx::smem_desc_k_sw128(sa + BM * BK * 2);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k)  // +32 bytes per K step: +2 in the (>>4) address field
-            ptx::mma_f16_ss(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb > sg.kb0) || k != 0);
+            ptx::mma_f16_ss(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)k * b_kstep, idesc, (kb > sg.kb0) || k != 0);
           ptx::mma_commit(ptx::smem_u32(&ctrl->empty[stage]));  // stage reusable once these MMAs have read it
           if (++stage == Cfg::kStages) { stage = 0; phase ^= 1; }
         }
@@ -464,43 +481,58 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
       const bool whole = sg.kb0 == 0 && sg.kb1 == p.kblocks;   // this CTA computed the tile's entire k range
       const bool seq = tile >= p.seq_from;                      // scatter from registers (Listing 4) or hand over (Listing 5)
       const int row_in_tile = quad * 32 + lane;
-      const int row = tc.tm * BM + row_in_tile;
       const int col_in_shard = tc.jn * BN;
-      const uint64_t row_off = p.c_off + ((uint64_t)row * p.N + (uint64_t)tc.rank * p.n_local) * 2;
       const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN);
 
-      // converts 32 fp32 columns of this thread's row and stores them where the schedule wants them
-      auto emit = [&](const uint32_t (&v)[32], int ch) {
-        uint4 q[4];
+      // The converted tile leaves through shared memory: a lane owns a row, so a store straight from its registers would
+      // put 16 bytes into each of 32 different lines per instruction (measured: twice the payload crosses the SM's port).
+      // Instead 128 columns at a time are staged as two 64-column boxes in the 128B-swizzle layout of the store maps
+      // (16-byte piece j of row r at position j ^ (r % 8): a warp's 512 bytes per instruction spread over all banks)
+      // and one thread sends them out with TMA -- whole 128-byte lines, clipped by the maps at row M and column N_local.
+      const uint32_t stg = ptx::smem_u32(payload + kSmemPayload);
+      auto stage_chunk = [&](const uint32_t (&v)[32], int ch) {
+        const uint32_t row_base = stg + (uint32_t)(((ch >> 1) & 1) * kStoreBoxBytes + row_in_tile * 128);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
+          uint4 q;
           if (p.kblocks == 0) {
-            q[i] = make_uint4(0, 0, 0, 0);  // K == 0: the sum is empty
+            q = make_uint4(0, 0, 0, 0);  // K == 0: the sum is empty
           } else {
-            q[i].x = pack2<BF16>(v[8 * i + 0], v[8 * i + 1]);
-            q[i].y = pack2<BF16>(v[8 * i + 2], v[8 * i + 3]);
-            q[i].z = pack2<BF16>(v[8 * i + 4], v[8 * i + 5]);
-            q[i].w = pack2<BF16>(v[8 * i + 6], v[8 * i + 7]);
+            q.x = pack2<BF16>(v[8 * i + 0], v[8 * i + 1]);
+            q.y = pack2<BF16>(v[8 * i + 2], v[8 * i + 3]);
+            q.z = pack2<BF16>(v[8 * i + 4], v[8 * i + 5]);
+            q.w = pack2<BF16>(v[8 * i + 6], v[8 * i + 7]);
           }
+          const int piece = (ch & 1) * 4 + i;
+          ptx::st_shared_v4(row_base + (uint32_t)((piece ^ (row_in_tile & 7)) << 4), q);
         }
-        if (row < p.M) {
-          const int c0 = col_in_shard + ch * 32;
-          if (seq) {
-            // Listing 4: the tile goes to every rank, the owner included, at the same symmetric offset
-            for (int s = 0; s < W; ++s) {
-              const uint64_t dst = p.tab.base[s] + row_off + (uint64_t)c0 * 2;  // translate(C + offset, rank -> s)
+      };
+      // Sends the staged columns [128 * half, 128 * half + 128) of the tile to every slot (Listing 4) or to the owner's
+      // (Listings 3 and 5).  After the last half the stores have been performed (the tile may be published); after an
+      // earlier one the boxes have been read and may be refilled.
+      auto flush_half = [&](int half, bool last) {
+        fence_proxy_async();   // this thread's shared-memory writes -> the TMA unit's reads
+        asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
+        if (et == 0) {
+          for (int s = 0; s < W; ++s) {
+            if (!seq && s != tc.rank) continue;
 #pragma unroll
-              for (int i = 0; i < 4; ++i)
-                if (c0 + 8 * i < p.n_local) st_global_v4(reinterpret_cast<void*>(dst + 16 * i), q[i]);
+            for (int b = 0; b < 2; ++b) {
+              const int col = col_in_shard + half * IRIS_TILE + 64 * b;
+              if (col >= p.n_local) continue;
+              if (p.one_map) ptx::tma_store_4d(&p.tmC4s, col, tc.tm * BM, tc.rank, s, stg + (uint32_t)(b * kStoreBoxBytes));
+              else ptx::tma_store_3d(&p.tmCs[s], col, tc.tm * BM, tc.rank, stg + (uint32_t)(b * kStoreBoxBytes));
             }
+          }
+          ptx::bulk_commit_group();
+          if (last) {
+            ptx::bulk_wait_group<0>();
+            fence_proxy_async();   // async-proxy writes above -> the generic-proxy release (flags or lock) after the barrier
           } else {
-            // Listings 3 and 5: store to the local (owner) rank's memory
-            const uint64_t dst = p.tab.base[tc.rank] + row_off + (uint64_t)c0 * 2;
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-              if (c0 + 8 * i < p.n_local) st_global_v4(reinterpret_cast<void*>(dst + 16 * i), q[i]);
+            ptx::bulk_wait_group_read<0>();
           }
         }
+        asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
       };
       auto release_accumulator = [&]() {
         ptx::tc_fence_before();
@@ -508,28 +540,34 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
         if (lane == 0) ptx::mbar_arrive(ptx::smem_u32(&ctrl->tmem_empty[acc]));
         if (++acc == 2) { acc = 0; acc_phase ^= 1; }
       };
+      constexpr int kChunks = BN / 32;
 
       bool publish = true;
       if (whole) {
 #pragma unroll 1
-        for (int ch = 0; ch < BN / 32; ++ch) {
+        for (int ch = 0; ch < kChunks; ++ch) {
           uint32_t v[32];
           ptx::tmem_ld_32x32(t_addr + (uint32_t)(ch * 32), v);
           ptx::tmem_wait_ld();
-          emit(v, ch);
+          stage_chunk(v, ch);
+          if ((ch & 3) == 3) {
+            if (ch == kChunks - 1) release_accumulator();   // accumulator drained: hand it back to the MMA warp
+            flush_half(ch >> 2, ch == kChunks - 1);
+          }
         }
-        release_accumulator();   // accumulator drained: hand it back to the MMA warp
       } else {
         // ---- stream-K: a part of the tile.  Park the fp32 partial sums, then see whether we are the last part. ----
-        float* mine = p.ws + (size_t)(2 * (int)blockIdx.x + (sg.first ? 0 : 1)) * (BM * BN) + (size_t)row_in_tile * BN;
+        // Workspace layout of a part: [chunk of 32 columns][row][32 floats], so a lane writes 128 contiguous bytes and a
+        // warp 4 KB.
+        float* mine = p.ws + (size_t)(2 * (int)blockIdx.x + (sg.first ? 0 : 1)) * (BM * BN) + (size_t)row_in_tile * 32;
 #pragma unroll 1
-        for (int ch = 0; ch < BN / 32; ++ch) {
+        for (int ch = 0; ch < kChunks; ++ch) {
           uint32_t v[32];
           ptx::tmem_ld_32x32(t_addr + (uint32_t)(ch * 32), v);
           ptx::tmem_wait_ld();
 #pragma unroll
           for (int i = 0; i < 8; ++i)
-            st_global_v4(mine + ch * 32 + 4 * i, make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
+            st_global_v4(mine + (size_t)ch * (BM * 32) + 4 * i, make_uint4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]));
         }
         release_accumulator();
         const int c_lo = streamk_cta_of((long long)tile * p.kblocks, units, p.gemm_ctas);
@@ -542,13 +580,13 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
         if (publish) {
           __threadfence();
 #pragma unroll 1
-          for (int ch = 0; ch < BN / 32; ++ch) {
+          for (int ch = 0; ch < kChunks; ++ch) {
             float sum[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) sum[i] = 0.0f;
             for (int c = c_lo; c <= c_hi; ++c) {   // parts in k order: CTA c_lo holds the lowest k range
               const bool its_first = streamk_begin(c, units, p.gemm_ctas) >= (long long)tile * p.kblocks;
-              const float* part = p.ws + (size_t)(2 * c + (its_first ? 0 : 1)) * (BM * BN) + (size_t)row_in_tile * BN + ch * 32;
+              const float* part = p.ws + (size_t)(2 * c + (its_first ? 0 : 1)) * (BM * BN) + (size_t)ch * (BM * 32) + (size_t)row_in_tile * 32;
 #pragma unroll
               for (int i = 0; i < 8; ++i) {
                 const uint4 w = ld_global_v4(part + 4 * i);
@@ -561,13 +599,14 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
             uint32_t v[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) v[i] = __float_as_uint(sum[i]);
-            emit(v, ch);
+            stage_chunk(v, ch);
+            if ((ch & 3) == 3) flush_half(ch >> 2, ch == kChunks - 1);
           }
         }
       }
       if (publish && p.mode != IRIS_MODE_BULK_SYNCHRONOUS) {
-        // every epilogue thread's stores happen-before the barrier; the release below is cumulative
-        asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
+        // the tile's stores have been performed and fenced by the issuing thread before the barrier that ended
+        // flush_half; the releases below are cumulative over them
         const int subs = BN / IRIS_TILE;
         const int pt_n = W * p.ptiles_per_rank;
         if (seq) {
@@ -703,7 +742,6 @@ __device__ __forceinline__ int pair_tile_cols(const GemmParams& p, int jn) {
 }
 constexpr int kPairStageBytes = 2 * BM * BK * 2;            // 32 KB: A slice + B half
 constexpr int kPairStages = 5;
-constexpr int kStoreBoxBytes = BM * 64 * 2;                 // 16 KB: 128 rows x 64 columns, one TMA store box
 constexpr int kPairStoreBytes = (kPairBN / 64) * kStoreBoxBytes;   // 64 KB: this CTA's 128 x 256 half of the converted tile
 constexpr int kPairSmemPayload = kPairStages * kPairStageBytes + kPairStoreBytes;   // 224 KB
 constexpr int kPairSmemTotal = kPairSmemPayload + kSmemCtrl + 1024;
@@ -762,7 +800,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
   if (warp >= kGemmThreads / 32) {
     if (CONSUMER && !is_comm) consumer_warp<BF16>(p, ctrl, warp - kGemmThreads / 32, lane);
   } else if (is_comm) {
-    comm_cta<STATIC_LOCKS, kPairBN / IRIS_TILE, 2>(p, ctrl, payload, warp, lane);
+    comm_cta<STATIC_LOCKS, kPairBN / IRIS_TILE, 2>(p, ctrl, payload, warp, lane, (int)blockIdx.x - p.gemm_ctas);
   } else if (warp == 0) {
     // ---------------- TMA producer (both CTAs); the leader's also claims and publishes the tiles ----------------
     if (lane == 0) {
@@ -802,7 +840,13 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
           const uint32_t full_leader = ptx::mapa(full_local, 0);
           const uint32_t sa = ptx::smem_u32(payload + stage * kPairStageBytes);
           ptx::tma_load_2d_pair(sa, &p.tmA, kb * BK, tc.tm * 2 * BM + cta_rank * BM, full_leader);
-          ptx::tma_load_2d_pair(sa + BM * BK * 2, &p.tmB[tc.rank], kb * BK, tc.jn * kPairBN + cta_rank * (ncols / 2), full_leader);
+          if (p.b_mn) {   // this CTA's half of the tile's columns as two [64 k][64 n] blocks
+            const int n0 = tc.jn * kPairBN + cta_rank * (ncols / 2);
+            ptx::tma_load_2d_pair(sa + BM * BK * 2, &p.tmB[tc.rank], n0, kb * BK, full_leader);
+            ptx::tma_load_2d_pair(sa + BM * BK * 2 + kMnBlockBytes, &p.tmB[tc.rank], n0 + 64, kb * BK, full_leader);
+          } else {
+            ptx::tma_load_2d_pair(sa + BM * BK * 2, &p.tmB[tc.rank], kb * BK, tc.jn * kPairBN + cta_rank * (ncols / 2), full_leader);
+          }
           if (++stage == kPairStages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
@@ -821,17 +865,18 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         if (!mbar_wait(ptx::smem_u32(&ctrl->tmem_empty[acc]), acc_phase ^ 1, p, ctrl, tile)) break;
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kPairBN);
-        const uint32_t idesc = ptx::idesc_f16(2 * BM, pair_tile_cols(p, decode_ctile(tile, p).jn), BF16 ? 1 : 0);
+        const uint32_t idesc = ptx::idesc_f16(2 * BM, pair_tile_cols(p, decode_ctile(tile, p).jn), BF16 ? 1 : 0) | (p.b_mn ? ptx::kIdescBMnMajor : 0u);
+        const uint64_t b_kstep = p.b_mn ? (uint64_t)(2 * 1024 >> 4) : 2u;
         bool ok = true;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!mbar_wait(ptx::smem_u32(&ctrl->full[stage]), phase, p, ctrl, tile)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t sa = ptx::smem_u32(payload + stage * kPairStageBytes);
           const uint64_t adesc = ptx::smem_desc_k_sw128(sa);
-          const uint64_t bdesc = ptx::smem_desc_k_sw128(sa + BM * BK * 2);
+          const uint64_t bdesc = p.b_mn ? ptx::smem_desc_mn_sw128(sa + BM * BK * 2, kMnBlockBytes) : ptx::smem_desc_k_sw128(sa + BM * BK * 2);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k)
-            ptx::mma_f16_ss_pair(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)(k * 2), idesc, (kb | k) != 0);
+            ptx::mma_f16_ss_pair(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)k * b_kstep, idesc, (kb | k) != 0);
           ptx::mma_commit_pair(ptx::smem_u32(&ctrl->empty[stage]), 3);  // both CTAs may refill this stage
           if (++stage == kPairStages) { stage = 0; phase ^= 1; }
         }
@@ -991,6 +1036,33 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
 }
 
 // ------------------------------------------------------------------------------------------------
+// Unfused producer-consumer (Section 4.1): the communication role as a kernel of its own.  The GEMM kernel runs with
+// producer CTAs only on one stream; this kernel, launched right after it on a second stream with as many CTAs as the
+// producers leave SMs free, is the consumer of the lock handshake: the same 32-lane acquire poll, claim, TMA copy to
+// the other W-1 slots and flag publication as the communication CTAs of the single launch (comm_cta above).
+// The dependency runs one way only: nothing in the GEMM kernel waits for this one, and every wait here has its
+// deadline, so the pair completes (or reports a timeout) whichever kernel the hardware happens to start first.
+// SUBS x SUBS_M: publication tiles per compute tile of the producing kernel (its work-item order).
+// ------------------------------------------------------------------------------------------------
+template <int SUBS, int SUBS_M>
+__global__ void __launch_bounds__(kCommWarps * 32, 1) scatter_comm_kernel(const __grid_constant__ GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* payload = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  CtrlBlock* ctrl = reinterpret_cast<CtrlBlock*>(payload + kSmemPayload);   // (kCommSmemTotal: no epilogue staging here)
+  const int warp = (int)threadIdx.x / 32, lane = (int)threadIdx.x % 32;
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kCommWarps; ++i) ptx::mbar_init(ptx::smem_u32(&ctrl->comm_full[i]), 1);
+    ctrl->abort = 0;
+    ptx::fence_mbar_init();
+    fence_proxy_async();
+    if (p.one_map) ptx::prefetch_tensormap(&p.tmC4);
+    else for (int r = 0; r < p.tab.world; ++r) ptx::prefetch_tensormap(&p.tmC[r]);
+  }
+  __syncthreads();
+  comm_cta<false, SUBS, SUBS_M>(p, ctrl, payload, warp, lane, (int)blockIdx.x);
+}
+
+// ------------------------------------------------------------------------------------------------
 // Bulk-synchronous second kernel (Listing 3, all_scatter): per publication tile, iris.put the owner's
 // tile to every other rank, then publish the W ready flags.
 // ------------------------------------------------------------------------------------------------
@@ -1122,6 +1194,16 @@ static int launch_gemm_pair(const GemmParams& p, int grid, cudaStream_t st, int*
   return IRIS_OK;
 }
 
+template <int SUBS, int SUBS_M>
+static int launch_scatter_comm(const GemmParams& p, cudaStream_t st) {
+  auto kern = scatter_comm_kernel<SUBS, SUBS_M>;
+  static bool configured[kMaxDevices] = {};
+  if (int rc = ensure_smem_limit(reinterpret_cast<const void*>(kern), kCommSmemTotal, configured)) return rc;
+  kern<<<p.comm_ctas, kCommWarps * 32, kCommSmemTotal, st>>>(p);
+  IRIS_CUDA_TRY(cudaGetLastError());
+  return IRIS_OK;
+}
+
 // How many CTAs to reserve for communication when the caller does not say.  A communication CTA moves
 // one tile read plus W-1 tile writes per publication tile; one SM sustains about 55 GB/s of such TMA
 // traffic while the other SMs run the GEMM (measured with per-phase %globaltimer stamps in the
@@ -1188,7 +1270,7 @@ struct PlanKey {
   const void* A; const void* B[IRIS_MAX_WORLD];
   int M, N, K, world, mode, dtype;
   uint64_t c_off, flag_off, lock_off;
-  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail, fused_consumer, rank_first, rank_count, pace_stores;
+  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail, fused_consumer, rank_first, rank_count, pace_stores, b_layout;
   uint64_t spin_timeout_ns;
 };
 // A few plans are kept (round-robin replacement): a step that alternates between calls -- one per rank shard in the
@@ -1210,7 +1292,7 @@ static void make_key(PlanKey* k, const iris_gemm_args* a, const iris_heap* h) {
   k->c_off = a->c_off; k->flag_off = a->flag_off; k->lock_off = a->lock_off;
   k->comm_ctas = a->comm_ctas; k->max_ctas = a->max_ctas; k->raster_group = a->raster_group; k->block_n = a->block_n;
   k->cta_pair = a->cta_pair; k->static_schedule = a->static_schedule; k->stream_k = a->stream_k; k->wg_tail = a->wg_tail;
-  k->rank_first = a->rank_first; k->rank_count = a->rank_count; k->pace_stores = a->pace_stores;
+  k->rank_first = a->rank_first; k->rank_count = a->rank_count; k->pace_stores = a->pace_stores; k->b_layout = a->b_layout;
   k->fused_consumer = a->consumer_bias != nullptr;   // the split between producers and communicators depends on it
   k->spin_timeout_ns = a->spin_timeout_ns;
 }
@@ -1278,6 +1360,7 @@ static int build_plan(const iris_gemm_args* a, const PlanEnv& env, Plan& out) {
   p.raster_group = a->raster_group ? a->raster_group : (pair ? 8 : 16);
   p.mode = a->mode;
   p.epoch = a->epoch;
+  p.b_mn = a->b_layout == IRIS_B_K_BY_N ? 1 : 0;
   grid = a->max_ctas ? std::min(a->max_ctas, env.sm_count) : env.sm_count;
   if (pair) {
     grid = std::min(grid & ~1, 2 * max_pairs);
@@ -1360,9 +1443,16 @@ static int build_plan(const iris_gemm_args* a, const PlanEnv& env, Plan& out) {
     int rc = make_map(&p.tmA, a->dtype, 2, const_cast<void*>(a->A), dimsA, strA, boxA, CU_TENSOR_MAP_SWIZZLE_128B, "A");
     if (rc != IRIS_OK) return rc;
     for (int r = rank_first; r < rank_first + rank_count; ++r) {
-      const cuuint64_t dimsB[2] = {(cuuint64_t)a->K, (cuuint64_t)nl};
-      const cuuint32_t boxB[2] = {BK, (cuuint32_t)(pair ? kPairBN / 2 : bn)};   // a pair's CTA loads its half of the tile
-      rc = make_map(&p.tmB[r], a->dtype, 2, const_cast<void*>(a->B_shards[r]), dimsB, strA, boxB, CU_TENSOR_MAP_SWIZZLE_128B, "B");
+      if (a->b_layout == IRIS_B_K_BY_N) {   // Listing 2's operand as printed: [K, N_local], N contiguous
+        const cuuint64_t dimsB[2] = {(cuuint64_t)nl, (cuuint64_t)a->K};
+        const cuuint64_t strB[1] = {(cuuint64_t)nl * 2};
+        const cuuint32_t boxB[2] = {64, BK};
+        rc = make_map(&p.tmB[r], a->dtype, 2, const_cast<void*>(a->B_shards[r]), dimsB, strB, boxB, CU_TENSOR_MAP_SWIZZLE_128B, "B [K, N_local]");
+      } else {
+        const cuuint64_t dimsB[2] = {(cuuint64_t)a->K, (cuuint64_t)nl};
+        const cuuint32_t boxB[2] = {BK, (cuuint32_t)(pair ? kPairBN / 2 : bn)};   // a pair's CTA loads its half of the tile
+        rc = make_map(&p.tmB[r], a->dtype, 2, const_cast<void*>(a->B_shards[r]), dimsB, strA, boxB, CU_TENSOR_MAP_SWIZZLE_128B, "B");
+      }
       if (rc != IRIS_OK) return rc;
     }
   }
@@ -1376,18 +1466,19 @@ static int build_plan(const iris_gemm_args* a, const PlanEnv& env, Plan& out) {
       int rc = make_map(&p.tmC4, a->dtype, 4, env.base + a->c_off, dims4, str4, box4, CU_TENSOR_MAP_SWIZZLE_NONE, "C (all slots)");
       if (rc != IRIS_OK) return rc;
     }
-    if (pair) {
-      int rc = make_map(&p.tmC4s, a->dtype, 4, env.base + a->c_off, dims4, str4, box4s, CU_TENSOR_MAP_SWIZZLE_128B, "C (all slots, epilogue stores)");
-      if (rc != IRIS_OK) return rc;
-    }
+    int rc = make_map(&p.tmC4s, a->dtype, 4, env.base + a->c_off, dims4, str4, box4s, CU_TENSOR_MAP_SWIZZLE_128B, "C (all slots, epilogue stores)");
+    if (rc != IRIS_OK) return rc;
   } else {
-    // slots at arbitrary addresses: C of slot s as [rank][row][column], one map per slot (communication CTAs only)
+    // slots at arbitrary addresses: C of slot s as [rank][row][column], per slot one map for the communication CTAs'
+    // copies and one for the epilogue's stores
     p.one_map = 0;
-    for (int s = 0; wg && s < W; ++s) {
+    for (int s = 0; s < W; ++s) {
       const cuuint64_t dimsC[3] = {(cuuint64_t)nl, (cuuint64_t)a->M, (cuuint64_t)W};
       const cuuint64_t strC[2] = {(cuuint64_t)a->N * 2, (cuuint64_t)nl * 2};
-      const cuuint32_t boxC[3] = {IRIS_TILE, IRIS_TILE, 1};
-      int rc = make_map(&p.tmC[s], a->dtype, 3, reinterpret_cast<void*>(env.tab.base[s] + a->c_off), dimsC, strC, boxC, CU_TENSOR_MAP_SWIZZLE_NONE, "C");
+      const cuuint32_t boxC[3] = {IRIS_TILE, IRIS_TILE, 1}, boxCs[3] = {64, BM, 1};
+      int rc = wg ? make_map(&p.tmC[s], a->dtype, 3, reinterpret_cast<void*>(env.tab.base[s] + a->c_off), dimsC, strC, boxC, CU_TENSOR_MAP_SWIZZLE_NONE, "C") : IRIS_OK;
+      if (rc != IRIS_OK) return rc;
+      rc = make_map(&p.tmCs[s], a->dtype, 3, reinterpret_cast<void*>(env.tab.base[s] + a->c_off), dimsC, strC, boxCs, CU_TENSOR_MAP_SWIZZLE_128B, "C (epilogue stores)");
       if (rc != IRIS_OK) return rc;
     }
   }
@@ -1431,7 +1522,9 @@ size_t iris_gemm_heap_bytes(int M, int N, int world) {
   return (size_t)(align_up((uint64_t)M * N * 2, 256) + 2 * align_up((uint64_t)nt * 4, 256) + 256);
 }
 
-int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
+// Checks, plan and launches of one call.  unfused: the workgroup-specialised schedule as two kernels, producers on
+// `stream` and the communication kernel on `comm_stream` (Section 4.1's unfused producer-consumer pattern).
+static int enqueue_gemm_all_scatter(const iris_gemm_args* a, void* stream, bool unfused, void* comm_stream) {
   if (!a) return fail(IRIS_ERR_ARG, "gemm_all_scatter: NULL args");
   iris_heap* h = a->heap;
   if (!heap_ok(h)) return fail(IRIS_ERR_STATE, "gemm_all_scatter: bad heap handle");
@@ -1452,6 +1545,7 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   if (a->pace_stores < -1 || a->pace_stores > 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: pace_stores must be 0 or -1");
   if (a->wg_tail < -1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: wg_tail must be -1, 0 or a tile count");
   if (a->stream_k < -1 || a->stream_k > 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: stream_k must be -1, 0 or 1");
+  if (a->b_layout != IRIS_B_N_BY_K && a->b_layout != IRIS_B_K_BY_N) return fail(IRIS_ERR_ARG, "gemm_all_scatter: unknown b_layout %d", a->b_layout);
   if (a->rank_first < 0 || a->rank_count < 0 || a->rank_first + a->rank_count > W || (a->rank_count == 0 && a->rank_first != 0))
     return fail(IRIS_ERR_ARG, "gemm_all_scatter: rank range [%d, %d) outside [0, %d)", a->rank_first, a->rank_first + a->rank_count, W);
   const int rank_first = a->rank_first, rank_count = a->rank_count ? a->rank_count : W;   // 0, 0 = every rank
@@ -1466,6 +1560,12 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   if (overlaps(a->c_off, c_bytes, a->flag_off, (uint64_t)nt * 4) || (wg && (overlaps(a->c_off, c_bytes, a->lock_off, (uint64_t)nt * 4) || overlaps(a->flag_off, (uint64_t)nt * 4, a->lock_off, (uint64_t)nt * 4))))
     return fail(IRIS_ERR_ARG, "gemm_all_scatter: C, flag and lock regions overlap");
   const bool fused_consumer = a->consumer_bias != nullptr;
+  if (unfused) {
+    if (!wg) return fail(IRIS_ERR_ARG, "gemm_all_scatter_unfused: the two-kernel form is the workgroup_specialized schedule (mode %d given)", a->mode);
+    // consumer warps inside the producer kernel would wait for flags that the second kernel publishes, while that one
+    // waits for the producers: two launches waiting on one another.  The consumer goes on a stream of its own instead.
+    if (fused_consumer) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter_unfused: consumer_bias is not supported here; launch iris_consume_bias on its own stream");
+  }
   if (fused_consumer) {
     if ((uint64_t)a->consumer_bias % 16 != 0 || a->consumer_out_off % 16 != 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: consumer bias / OUT offset must be 16-byte aligned");
     if (a->consumer_out_off > bpr || c_bytes > bpr - a->consumer_out_off) return fail(IRIS_ERR_RANGE, "gemm_all_scatter: OUT leaves the slot");
@@ -1541,11 +1641,33 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
   }
   const bool cons_in_kernel = pair && fused_consumer && a->mode != IRIS_MODE_BULK_SYNCHRONOUS;  // BSP publishes in its 2nd kernel
   if (cons_in_kernel) { p.bias = static_cast<const uint8_t*>(a->consumer_bias); p.out_off = a->consumer_out_off; }
-  if (cons_in_kernel) rc = bf ? launch_gemm_pair<true, false, true>(p, grid, st, nullptr) : launch_gemm_pair<false, false, true>(p, grid, st, nullptr);
-  else if (pair)      rc = bf ? launch_gemm_pair<true>(p, grid, st, nullptr) : launch_gemm_pair<false>(p, grid, st, nullptr);
-  else if (bn == 256) rc = bf ? launch_gemm<256, true>(p, grid, wg, st) : launch_gemm<256, false>(p, grid, wg, st);
-  else                rc = bf ? launch_gemm<128, true>(p, grid, wg, st) : launch_gemm<128, false>(p, grid, wg, st);
+  // unfused: the producers alone; they wait on nothing outside their own CTA (pair), so no cooperative launch is needed
+  const int ggrid = unfused ? p.gemm_ctas : grid;
+  const bool coop = wg && !unfused;
+  if (unfused) {   // fork: the second stream starts after whatever precedes the producers on the first (the counter resets above)
+    if (!h->ev_fork) {
+      IRIS_CUDA_TRY(cudaEventCreateWithFlags(reinterpret_cast<cudaEvent_t*>(&h->ev_fork), cudaEventDisableTiming));
+      IRIS_CUDA_TRY(cudaEventCreateWithFlags(reinterpret_cast<cudaEvent_t*>(&h->ev_join), cudaEventDisableTiming));
+    }
+    IRIS_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(h->ev_fork), st));
+  }
+  if (cons_in_kernel) rc = bf ? launch_gemm_pair<true, false, true>(p, ggrid, st, nullptr) : launch_gemm_pair<false, false, true>(p, ggrid, st, nullptr);
+  else if (pair)      rc = bf ? launch_gemm_pair<true>(p, ggrid, st, nullptr) : launch_gemm_pair<false>(p, ggrid, st, nullptr);
+  else if (bn == 256) rc = bf ? launch_gemm<256, true>(p, ggrid, coop, st) : launch_gemm<256, false>(p, ggrid, coop, st);
+  else                rc = bf ? launch_gemm<128, true>(p, ggrid, coop, st) : launch_gemm<128, false>(p, ggrid, coop, st);
   if (rc != IRIS_OK) return rc;
+  if (unfused) {
+    // The producers are launched first; the communication kernel follows on its own stream and takes the SMs they left.
+    // join: work enqueued on `stream` after this call sees the finished scatter.
+    cudaStream_t cst = static_cast<cudaStream_t>(comm_stream);
+    IRIS_CUDA_TRY(cudaStreamWaitEvent(cst, static_cast<cudaEvent_t>(h->ev_fork), 0));
+    if (pair)           rc = launch_scatter_comm<2, 2>(p, cst);
+    else if (bn == 256) rc = launch_scatter_comm<2, 1>(p, cst);
+    else                rc = launch_scatter_comm<1, 1>(p, cst);
+    if (rc != IRIS_OK) return rc;
+    IRIS_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(h->ev_join), cst));
+    IRIS_CUDA_TRY(cudaStreamWaitEvent(st, static_cast<cudaEvent_t>(h->ev_join), 0));
+  }
   if (a->mode == IRIS_MODE_BULK_SYNCHRONOUS) {
     // Listing 3: the second kernel on the same stream; the kernel boundary is the synchronisation.
     const int g2 = std::min(p.total_ptiles, h->sm_count * 8);
@@ -1558,6 +1680,13 @@ int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) {
     return iris_consume_bias_ranks(h, a->c_off, a->consumer_out_off, a->flag_off, a->consumer_bias, a->M, a->N, W, rank_first, rank_count, a->dtype, a->epoch, 0,
                                    a->spin_timeout_ns, stream);
   return IRIS_OK;
+}
+
+int iris_gemm_all_scatter_ex(const iris_gemm_args* a, void* stream) { return enqueue_gemm_all_scatter(a, stream, false, nullptr); }
+
+int iris_gemm_all_scatter_unfused(const iris_gemm_args* a, void* producer_stream, void* comm_stream) {
+  if (producer_stream == comm_stream) return fail(IRIS_ERR_ARG, "gemm_all_scatter_unfused: the two kernels need two different streams");
+  return enqueue_gemm_all_scatter(a, producer_stream, true, comm_stream);
 }
 
 static void short_form_layout(int M, int N, int world, uint64_t* flag_off, uint64_t* lock_off) {

@@ -109,6 +109,8 @@ int iris_heap_destroy(iris_heap* h) {
   if (h->stage_b) cudaFree(h->stage_b);
   if (h->ws) cudaFree(h->ws);
   iris::free_host_pipe(h);
+  if (h->ev_fork) cudaEventDestroy(static_cast<cudaEvent_t>(h->ev_fork));
+  if (h->ev_join) cudaEventDestroy(static_cast<cudaEvent_t>(h->ev_join));
   h->magic = 0;
   delete h;
   cudaGetLastError();

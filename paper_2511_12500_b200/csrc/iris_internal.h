@@ -60,6 +60,9 @@ struct iris_heap {
   size_t ws_bytes;
   // streams and events of the host-buffer entry point's copy/compute pipeline, created on first use
   void* host_pipe;
+  // fork / join events of the two-stream (unfused) form of the workgroup-specialised schedule, created on first use
+  void* ev_fork;
+  void* ev_join;
   iris::HeapTable table() const {
     iris::HeapTable t{};
     for (int r = 0; r < world; ++r) t.base[r] = (uint64_t)(base + (size_t)r * bytes_per_rank);

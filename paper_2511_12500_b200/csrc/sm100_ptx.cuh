@@ -83,6 +83,13 @@ __device__ __forceinline__ void bulk_wait_group() {
   asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
 }
 
+// The .read form: waits only until the sources in shared memory have been read (they may be overwritten), not
+// until the global writes have been performed.
+template <int N>
+__device__ __forceinline__ void bulk_wait_group_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+
 // ---- tensor memory ---------------------------------------------------------------------------------
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
@@ -131,10 +138,19 @@ __device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t smem_addr) {
   return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
 
+// The same for an MN-major operand tile (the operand's M or N index is the contiguous one in memory): the tile is a
+// row of [64 k][64 mn] blocks as a SWIZZLE_128B tensor map with box {64 mn, 64 k} writes them, each row 128 bytes.
+// Within a block 8 k-rows form one 1024-byte swizzle atom (stride byte offset = 1024: from one group of 8 k to the
+// next); blocks of 64 mn indices are `block_bytes` apart (leading byte offset).
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t smem_addr, uint32_t block_bytes) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)(block_bytes >> 4) << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+
 // Instruction descriptor, kind::f16: D = fp32, A/B = fp16 (0) or bf16 (1), both K-major, M x N tile.
 __host__ __device__ constexpr uint32_t idesc_f16(int m, int n, int ab_fmt) {
   return (1u << 4) | ((uint32_t)ab_fmt << 7) | ((uint32_t)ab_fmt << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
+constexpr uint32_t kIdescBMnMajor = 1u << 16;   // OR into the descriptor: B is MN-major (N contiguous) instead of K-major
 
 // ---- CTA pairs (cluster of 2, tcgen05 cta_group::2) ----------------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank() {

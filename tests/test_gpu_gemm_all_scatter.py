@@ -24,7 +24,8 @@ def run_gemm(g, A, Bs, dtype, mode, epoch=1, with_locks_zeroed=True, **kw):
     W, nl = len(Bs), Bs[0].shape[0]
     N = W * nl
     c_off, flag_off, lock_off, out_off, _ = gemm_layout(M, N, W, with_out=True)
-    dA, dB = dev16(A), [dev16(b) for b in Bs]
+    # b_layout = 1: the shards are handed over as [K, N_local] row-major (the oracle keeps reading the [N_local, K] arrays)
+    dA, dB = dev16(A), [dev16(np.ascontiguousarray(b.T) if kw.get("b_layout", 0) == 1 else b) for b in Bs]
     nt = oracle.num_tiles(M, N, W) if M and N else 0
     if with_locks_zeroed and nt:
         iris.iris_flags_fill(g.h, lock_off, nt, 0)
@@ -114,6 +115,54 @@ def test_exact_integer_gemm_full_heap_image(mode, dtype, W, M, nl, K):
         host = g.to_host()
         img, _ = expected_image(g, A, Bs, dtype, mode)
         assert np.array_equal(host, img.mem), first_diff(host, img.mem)
+
+
+B_ROW_MAJOR_SHAPES = [
+    # W, M, N_local, K, kwargs: B shards stored [K, N_local] (Listing 2's operand as printed), read as an MN-major operand
+    (1, 128, 128, 64, dict()),
+    (4, 130, 136, 72, dict()),                          # single-CTA kernel, everything ragged
+    (3, 520, 392, 328, dict()),                         # CTA pairs, ragged shard (392 = 256 + 136)
+    (3, 520, 392, 328, dict(cta_pair=-1)),              # the same on the single-CTA kernel
+    (3, 384, 904, 64, dict()),                          # 904 = 3 * 256 + 136
+    (2, 600, 448, 136, dict()),                         # 448 = 256 + 192: a 192-wide last pair tile, 96 columns per CTA
+    (2, 384, 256, 192, dict(cta_pair=-1, block_n=256)), # single-CTA kernel, 256-wide tiles: four 64-column blocks per stage
+    (8, 128, 512, 128, dict(block_n=128)),
+    (2, 1000, 512, 200, dict()),
+    (4, 100, 136, 4096, dict(stream_k=1)),              # k ranges of a tile computed by different CTAs
+    (8, 8, 8, 8, dict()),                               # a shard narrower than one 64-column block
+]
+
+
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("dtype", ["bf16", "fp16"])
+@pytest.mark.parametrize("W,M,nl,K,kw", B_ROW_MAJOR_SHAPES)
+def test_b_shards_row_major_k_by_n_full_heap_image(mode, dtype, W, M, nl, K, kw):
+    N = W * nl
+    A = inputs.matrix(71, inputs.STREAM_A, M, K, "ternary:0.5", dtype)
+    Bs = [inputs.matrix(71, inputs.STREAM_B0 + r, nl, K, "smallint:2", dtype) for r in range(W)]
+    bpr = gemm_layout(M, N, W, True)[4]
+    with GpuHeap(W, bpr) as g:
+        run_gemm(g, A, Bs, dtype, mode, b_layout=1, **kw)
+        host = g.to_host()
+        img, _ = expected_image(g, A, Bs, dtype, mode)
+        assert np.array_equal(host, img.mem), first_diff(host, img.mem)
+
+
+def test_b_layouts_agree_bit_for_bit_on_real_valued_inputs():
+    """Same sums in the same order whichever way B is stored: C from [K, N_local] shards equals C from [N_local, K] shards."""
+    W, M, nl, K, dtype = 4, 384, 320, 1024, "bf16"
+    N = W * nl
+    A, Bs = inputs.gemm_inputs(inputs.SEED0 + 2, W, M, N, K, "normal002", dtype)
+    c_ref = oracle.gemm_block(A, Bs, dtype)
+    bpr = gemm_layout(M, N, W, True)[4]
+    for kw in (dict(), dict(cta_pair=-1)):
+        outs = []
+        for b_layout in (0, 1):
+            with GpuHeap(W, bpr) as g:
+                c_off = run_gemm(g, A, Bs, dtype, iris.IRIS_MODE_FUSED_SEQUENTIAL, b_layout=b_layout, **kw)[0]
+                outs.append(c_slot(g.to_host(), g, W - 1, c_off, M, N).copy())
+        check_tolerance(outs[1], c_ref, dtype)
+        assert np.array_equal(outs[0], outs[1])
 
 
 @pytest.mark.parametrize("block_n", [128, 256])
