@@ -67,6 +67,7 @@ struct TileCfg {
 struct alignas(64) GemmParams {
   CUtensorMap tmA;                    // A [M, K], box 64 x 128, 128B swizzle
   CUtensorMap tmB[IRIS_MAX_WORLD];    // B_r [N_local, K], box 64 x BN, 128B swizzle; or B_r [K, N_local], box 64 (n) x 64 (k), 128B swizzle
+  CUtensorMap tmBn[IRIS_MAX_WORLD];   // pair kernel, fuse_last: B_r [N_local, K] with a box of 64 x (remainder columns / 2) rows
   CUtensorMap tmC[IRIS_MAX_WORLD];    // C of slot s viewed as [W][M][N_local], box 128 x 128 x 1, no swizzle
   CUtensorMap tmC4;                   // C of all slots as one tensor [slot][rank][M][N_local] (slots equally spaced: every heap
                                       // handle), box 128 x 128 x 1 x 1, no swizzle: the communication warps' copies
@@ -101,6 +102,12 @@ struct alignas(64) GemmParams {
   int32_t* backlog;     // publication tiles handed over and not yet published ([0]), tiles kept by that rule ([1])
   uint32_t t_pt_ns;     // estimate: time a communication warp needs for one publication tile, its CTA's port shared by all warps
   uint32_t t_tile_ns;   // estimate: main-loop time of one compute tile
+  int fuse_last;        // pair kernel: 1 = a shard's last full 256-column tile and the narrow remainder after it are ONE work unit
+                        // (two MMA groups on the same A stages, one accumulator each): the remainder no longer costs its own
+                        // loads of A.  ctiles_per_rank / total_ctiles then count work units, one fewer per shard than tiles
+  int stage_bytes;      // pair kernel: bytes of one operand stage (32 KB, plus the remainder's B rows with fuse_last) ...
+  int n_stages;         // ... and how many of them fit beside the store boxes (5, 4 or 3)
+  int b1_bytes;         // fuse_last: bytes of the remainder's B box per CTA
   int b_mn;             // 1 = B_r is [K, N_local] row-major (N contiguous): 64 x 64 boxes, MN-major descriptor; 0 = [N_local, K]
   int pace_stores;      // pair kernel: 1 = the epilogue spreads a tile's box stores over most of the next tile's main loop
   int raster_group;
@@ -199,7 +206,8 @@ __device__ __forceinline__ int32_t* lock_addr(const GemmParams& p, int rank, int
 // Communication CTA (workgroup-specialised mode), Listing 5's `else` branch.
 // Each of the CTA's six warps is an independent communicator with its own 32 KB tile buffer and its own
 // mbarrier.  Work items are publication tiles numbered in the producers' raster order (item k = sub-tile
-// k % SUBS of compute tile k / SUBS; a CTA pair's 256-row tile has SUBS_M = 2 rows of them), dealt round-robin to the communicator warps, so a warp sees its
+// k % SUBS of compute tile k / SUBS; a CTA pair's 256-row tile has SUBS_M = 2 rows of them; a work unit of the pair kernel may hold two compute tiles),
+// dealt round-robin to the communicator warps, so a warp sees its
 // tiles become ready roughly first-in first-out.
 //   poll     all 32 lanes watch 32 of the warp's pending items at once: one acquire-ordered load of
 //            lock[t] per lane; a ballot collects the ready set
@@ -215,7 +223,9 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
   const int W = p.tab.world;
   const int ncw = p.comm_ctas * kCommWarps;
   const int cw = comm_block * kCommWarps + warp;   // comm_block: this CTA's index among the communication CTAs
-  const int items = min(p.total_ctiles, p.seq_from) * SUBS * SUBS_M;   // the tail wave's tiles are scattered by their producers
+  const int L = p.fuse_last ? 2 : 1;               // compute tiles per work unit (pair kernel with fused shard tails: up to two)
+  const int per_unit = SUBS * SUBS_M * L;
+  const int items = min(p.total_ctiles, p.seq_from) * per_unit;   // the tail wave's tiles are scattered by their producers
   const int n_my = cw < items ? (items - cw + ncw - 1) / ncw : 0;  // items cw, cw + ncw, ...
   const int pt_n = W * p.ptiles_per_rank;
   const uint32_t buf = ptx::smem_u32(payload + warp * kTileBytes);
@@ -233,9 +243,10 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
     t = -1;
     if (widx < 0) return;
     const int k = cw + widx * ncw;
-    const TileCoord tc = decode_ctile(k / (SUBS * SUBS_M), p);
-    const int sub = k % (SUBS * SUBS_M);
-    const int pj = tc.jn * SUBS + sub % SUBS;
+    const TileCoord tc = decode_ctile(k / per_unit, p);
+    const int l = (k % per_unit) / (SUBS * SUBS_M), sub = k % (SUBS * SUBS_M);
+    if (l == 1 && tc.jn != p.ctiles_per_rank - 1) return;   // only a shard's last unit has a second tile
+    const int pj = (tc.jn + l) * SUBS + sub % SUBS;
     const int tm = tc.tm * SUBS_M + sub / SUBS;  // publication tile row
     rank = tc.rank;
     if (pj < p.ptiles_per_rank && tm < p.ptiles_m) t = tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
@@ -653,12 +664,14 @@ __device__ void consumer_warp(const GemmParams& p, CtrlBlock* ctrl, int cwarp, i
   const int W = p.tab.world;
   const int ncons = p.gemm_ctas * kConsWarps;
   const int pt_n = W * p.ptiles_per_rank;
-  const long long items = (long long)p.total_ctiles * SUBS * SUBS_M * W;
+  const int L = p.fuse_last ? 2 : 1, per_unit = SUBS * SUBS_M * L;
+  const long long items = (long long)p.total_ctiles * per_unit * W;
   for (long long q = (long long)blockIdx.x * kConsWarps + cwarp; q < items; q += ncons) {
     const int k = (int)(q / W), s = (int)(q % W);
-    const TileCoord tc = decode_ctile(k / (SUBS * SUBS_M), p);
-    const int sub = k % (SUBS * SUBS_M);
-    const int pj = tc.jn * SUBS + sub % SUBS;
+    const TileCoord tc = decode_ctile(k / per_unit, p);
+    const int l = (k % per_unit) / (SUBS * SUBS_M), sub = k % (SUBS * SUBS_M);
+    if (l == 1 && tc.jn != p.ctiles_per_rank - 1) continue;   // only a shard's last unit has a second tile
+    const int pj = (tc.jn + l) * SUBS + sub % SUBS;
     const int tm = tc.tm * SUBS_M + sub / SUBS;
     if (pj >= p.ptiles_per_rank || tm >= p.ptiles_m) continue;
     const int t = tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
@@ -832,13 +845,16 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         if (tile < 0) break;
         const TileCoord tc = decode_ctile(tile, p);
         const int ncols = pair_tile_cols(p, tc.jn);   // this CTA keeps rows [cta_rank * ncols / 2, ...) of the B tile
+        // a shard's last unit with fuse_last: the remainder tile's B rows ride in the same stage, after A and B
+        const bool fused = p.fuse_last && tc.jn == p.ctiles_per_rank - 1;
+        const int ncols1 = fused ? pair_tile_cols(p, tc.jn + 1) : 0;
         bool ok = true;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!mbar_wait(ptx::smem_u32(&ctrl->empty[stage]), phase ^ 1, p, ctrl, tile)) { ok = false; break; }
           const uint32_t full_local = ptx::smem_u32(&ctrl->full[stage]);
-          if (leader) ptx::mbar_arrive_expect_tx(full_local, 2 * kPairStageBytes);
+          if (leader) ptx::mbar_arrive_expect_tx(full_local, 2 * (kPairStageBytes + (fused ? p.b1_bytes : 0)));
           const uint32_t full_leader = ptx::mapa(full_local, 0);
-          const uint32_t sa = ptx::smem_u32(payload + stage * kPairStageBytes);
+          const uint32_t sa = ptx::smem_u32(payload + stage * p.stage_bytes);
           ptx::tma_load_2d_pair(sa, &p.tmA, kb * BK, tc.tm * 2 * BM + cta_rank * BM, full_leader);
           if (p.b_mn) {   // this CTA's half of the tile's columns as two [64 k][64 n] blocks
             const int n0 = tc.jn * kPairBN + cta_rank * (ncols / 2);
@@ -847,7 +863,8 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
           } else {
             ptx::tma_load_2d_pair(sa + BM * BK * 2, &p.tmB[tc.rank], kb * BK, tc.jn * kPairBN + cta_rank * (ncols / 2), full_leader);
           }
-          if (++stage == kPairStages) { stage = 0; phase ^= 1; }
+          if (fused) ptx::tma_load_2d_pair(sa + kPairStageBytes, &p.tmBn[tc.rank], kb * BK, (tc.jn + 1) * kPairBN + cta_rank * (ncols1 / 2), full_leader);
+          if (++stage == p.n_stages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
       }
@@ -862,27 +879,45 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         const int tile = feed_take(fj, fph, fslot);
         if (tile != -2) feed_release(fslot);
         if (tile < 0) break;
+        const TileCoord tc = decode_ctile(tile, p);
+        const bool fused = p.fuse_last && tc.jn == p.ctiles_per_rank - 1;
+        // accumulator(s): one per compute tile of the unit, taken in order from the two buffers
+        const int a0 = acc;
         if (!mbar_wait(ptx::smem_u32(&ctrl->tmem_empty[acc]), acc_phase ^ 1, p, ctrl, tile)) break;
+        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        const int a1 = acc;
+        if (fused) {
+          if (!mbar_wait(ptx::smem_u32(&ctrl->tmem_empty[acc]), acc_phase ^ 1, p, ctrl, tile)) break;
+          if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
         ptx::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kPairBN);
-        const uint32_t idesc = ptx::idesc_f16(2 * BM, pair_tile_cols(p, decode_ctile(tile, p).jn), BF16 ? 1 : 0) | (p.b_mn ? ptx::kIdescBMnMajor : 0u);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(a0 * kPairBN), d_tmem1 = tmem_base + (uint32_t)(a1 * kPairBN);
+        const uint32_t b_major = p.b_mn ? ptx::kIdescBMnMajor : 0u;
+        const uint32_t idesc = ptx::idesc_f16(2 * BM, pair_tile_cols(p, tc.jn), BF16 ? 1 : 0) | b_major;
+        const uint32_t idesc1 = fused ? ptx::idesc_f16(2 * BM, pair_tile_cols(p, tc.jn + 1), BF16 ? 1 : 0) : 0u;
         const uint64_t b_kstep = p.b_mn ? (uint64_t)(2 * 1024 >> 4) : 2u;
         bool ok = true;
         for (int kb = 0; kb < p.kblocks; ++kb) {
           if (!mbar_wait(ptx::smem_u32(&ctrl->full[stage]), phase, p, ctrl, tile)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint32_t sa = ptx::smem_u32(payload + stage * kPairStageBytes);
+          const uint32_t sa = ptx::smem_u32(payload + stage * p.stage_bytes);
           const uint64_t adesc = ptx::smem_desc_k_sw128(sa);
           const uint64_t bdesc = p.b_mn ? ptx::smem_desc_mn_sw128(sa + BM * BK * 2, kMnBlockBytes) : ptx::smem_desc_k_sw128(sa + BM * BK * 2);
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k)
             ptx::mma_f16_ss_pair(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)k * b_kstep, idesc, (kb | k) != 0);
+          if (fused) {   // the remainder tile: same A stage, its own B rows, the other accumulator
+            const uint64_t b1desc = ptx::smem_desc_k_sw128(sa + kPairStageBytes);
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k)
+              ptx::mma_f16_ss_pair(d_tmem1, adesc + (uint64_t)(k * 2), b1desc + (uint64_t)(k * 2), idesc1, (kb | k) != 0);
+          }
           ptx::mma_commit_pair(ptx::smem_u32(&ctrl->empty[stage]), 3);  // both CTAs may refill this stage
-          if (++stage == kPairStages) { stage = 0; phase ^= 1; }
+          if (++stage == p.n_stages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
-        ptx::mma_commit_pair(ptx::smem_u32(&ctrl->tmem_full[acc]), 3);  // accumulator complete in both CTAs
-        if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        ptx::mma_commit_pair(ptx::smem_u32(&ctrl->tmem_full[a0]), 3);  // accumulator complete in both CTAs
+        if (fused) ptx::mma_commit_pair(ptx::smem_u32(&ctrl->tmem_full[a1]), 3);
       }
     }
   } else {
@@ -894,15 +929,20 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
     const uint32_t tmem_base = ctrl->tmem_base;
     uint64_t prev_issue = 0;               // thread 0: when the previous tile's stores started
     uint32_t period_ns = p.t_tile_ns;      // thread 0: time between two tiles of this CTA (estimate, then measured)
-    for (;;) {
-      const int tile = feed_take(fj, fph, fslot);
+    bool stop = false;
+    while (!stop) {
+      const int tile = feed_take(fj, fph, fslot);   // a work unit: one compute tile, or a shard's last full tile plus its remainder
       __syncwarp();
       if (tile != -2 && lane == 0) feed_release(fslot);
+      const TileCoord tc0 = decode_ctile(tile >= 0 ? tile : 0, p);
+      const int nsub = (tile >= 0 && p.fuse_last && tc0.jn == p.ctiles_per_rank - 1) ? 2 : 1;
+      for (int l = 0; l < nsub; ++l) {   // the unit's compute tiles, one accumulator each, in the order the MMA thread took them
       // uniform decision for all four warps: stop on the end marker or on any failed wait
       bool ok = tile >= 0;
       if (ok) ok = mbar_wait(ptx::smem_u32(&ctrl->tmem_full[acc]), acc_phase, p, ctrl, tile);
-      if (ptx::bar_red_or(1, kEpiThreads, !ok)) break;
-      const TileCoord tc = decode_ctile(tile, p);
+      if (ptx::bar_red_or(1, kEpiThreads, !ok)) { stop = true; break; }
+      TileCoord tc = tc0;
+      tc.jn += l;
       ptx::tc_fence_after();
       const int tm = tc.tm * 2 + cta_rank;  // publication tile row of this CTA's half
       const int row_in_half = quad * 32 + lane;
@@ -1023,6 +1063,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
           }
         }
       }
+      }   // compute tiles of the unit
     }
   }
 
@@ -1270,7 +1311,7 @@ struct PlanKey {
   const void* A; const void* B[IRIS_MAX_WORLD];
   int M, N, K, world, mode, dtype;
   uint64_t c_off, flag_off, lock_off;
-  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail, fused_consumer, rank_first, rank_count, pace_stores, b_layout;
+  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail, fused_consumer, rank_first, rank_count, pace_stores, b_layout, fuse_tail;
   uint64_t spin_timeout_ns;
 };
 // A few plans are kept (round-robin replacement): a step that alternates between calls -- one per rank shard in the
@@ -1292,7 +1333,7 @@ static void make_key(PlanKey* k, const iris_gemm_args* a, const iris_heap* h) {
   k->c_off = a->c_off; k->flag_off = a->flag_off; k->lock_off = a->lock_off;
   k->comm_ctas = a->comm_ctas; k->max_ctas = a->max_ctas; k->raster_group = a->raster_group; k->block_n = a->block_n;
   k->cta_pair = a->cta_pair; k->static_schedule = a->static_schedule; k->stream_k = a->stream_k; k->wg_tail = a->wg_tail;
-  k->rank_first = a->rank_first; k->rank_count = a->rank_count; k->pace_stores = a->pace_stores; k->b_layout = a->b_layout;
+  k->rank_first = a->rank_first; k->rank_count = a->rank_count; k->pace_stores = a->pace_stores; k->b_layout = a->b_layout; k->fuse_tail = a->fuse_tail;
   k->fused_consumer = a->consumer_bias != nullptr;   // the split between producers and communicators depends on it
   k->spin_timeout_ns = a->spin_timeout_ns;
 }
@@ -1340,6 +1381,17 @@ static int build_plan(const iris_gemm_args* a, const PlanEnv& env, Plan& out) {
     }
   }
   if (pair) bn = kPairBN;
+  // Ragged shard on the pair kernel: the remainder after the last full 256-column tile is computed by the pair that
+  // computes that tile, on the same A stages (a 64-column tile of its own would pull in as much of A as a full one).
+  p.fuse_last = (pair && a->fuse_tail >= 0 && a->b_layout == IRIS_B_N_BY_K && nl > kPairBN && nl % kPairBN != 0) ? 1 : 0;
+  p.stage_bytes = kPairStageBytes;
+  p.n_stages = kPairStages;
+  if (p.fuse_last) {
+    const int rem32 = ((nl % kPairBN) + 31) & ~31;
+    p.b1_bytes = (rem32 / 2) * BK * 2;
+    p.stage_bytes = kPairStageBytes + (int)align_up((uint64_t)p.b1_bytes, 1024);
+    p.n_stages = std::min(kPairStages, (kPairStages * kPairStageBytes) / p.stage_bytes);
+  }
   p.tab = env.tab;
   p.c_off = a->c_off;
   p.flag_off = a->flag_off;
@@ -1349,7 +1401,7 @@ static int build_plan(const iris_gemm_args* a, const PlanEnv& env, Plan& out) {
   p.M = a->M; p.N = a->N; p.K = a->K; p.n_local = nl;
   p.ptiles_m = (a->M + BM - 1) / BM;
   p.tiles_m = pair ? (a->M + 2 * BM - 1) / (2 * BM) : p.ptiles_m;
-  p.ctiles_per_rank = (nl + bn - 1) / bn;
+  p.ctiles_per_rank = (nl + bn - 1) / bn - p.fuse_last;   // work units per rank along N
   p.ptiles_per_rank = (nl + IRIS_TILE - 1) / IRIS_TILE;
   p.rank_first = rank_first; p.rank_count = rank_count;
   p.total_ctiles = p.tiles_m * rank_count * p.ctiles_per_rank;
@@ -1452,6 +1504,10 @@ static int build_plan(const iris_gemm_args* a, const PlanEnv& env, Plan& out) {
         const cuuint64_t dimsB[2] = {(cuuint64_t)a->K, (cuuint64_t)nl};
         const cuuint32_t boxB[2] = {BK, (cuuint32_t)(pair ? kPairBN / 2 : bn)};   // a pair's CTA loads its half of the tile
         rc = make_map(&p.tmB[r], a->dtype, 2, const_cast<void*>(a->B_shards[r]), dimsB, strA, boxB, CU_TENSOR_MAP_SWIZZLE_128B, "B");
+        if (rc == IRIS_OK && p.fuse_last) {
+          const cuuint32_t boxBn[2] = {BK, (cuuint32_t)(p.b1_bytes / (BK * 2))};
+          rc = make_map(&p.tmBn[r], a->dtype, 2, const_cast<void*>(a->B_shards[r]), dimsB, strA, boxBn, CU_TENSOR_MAP_SWIZZLE_128B, "B (remainder columns)");
+        }
       }
       if (rc != IRIS_OK) return rc;
     }
@@ -1545,6 +1601,7 @@ static int enqueue_gemm_all_scatter(const iris_gemm_args* a, void* stream, bool 
   if (a->pace_stores < -1 || a->pace_stores > 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: pace_stores must be 0 or -1");
   if (a->wg_tail < -1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: wg_tail must be -1, 0 or a tile count");
   if (a->stream_k < -1 || a->stream_k > 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: stream_k must be -1, 0 or 1");
+  if (a->fuse_tail < -1 || a->fuse_tail > 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: fuse_tail must be 0 or -1");
   if (a->b_layout != IRIS_B_N_BY_K && a->b_layout != IRIS_B_K_BY_N) return fail(IRIS_ERR_ARG, "gemm_all_scatter: unknown b_layout %d", a->b_layout);
   if (a->rank_first < 0 || a->rank_count < 0 || a->rank_first + a->rank_count > W || (a->rank_count == 0 && a->rank_first != 0))
     return fail(IRIS_ERR_ARG, "gemm_all_scatter: rank range [%d, %d) outside [0, %d)", a->rank_first, a->rank_first + a->rank_count, W);

@@ -165,6 +165,41 @@ def test_b_layouts_agree_bit_for_bit_on_real_valued_inputs():
         assert np.array_equal(outs[0], outs[1])
 
 
+RAGGED_PAIR_SHAPES = [
+    # W, M, N_local, K: CTA-pair kernel, N_local > 256 and not a multiple of 256
+    (2, 600, 448, 136),      # 256 + 192
+    (3, 384, 904, 64),       # 3 x 256 + 136: two plain units and a fused one per shard; the remainder's last publication tile is 8 wide
+    (3, 520, 392, 328),      # 256 + 136
+    (2, 300, 640, 64),       # 2 x 256 + 128
+    (4, 1100, 576, 256),     # 2 x 256 + 64 (the paper's 4608 / 8), ragged M
+    (2, 512, 320, 128),      # 256 + 64
+    (8, 2048, 288, 64),      # 256 + 32: the narrowest remainder an MMA group can have
+    (2, 700, 504, 72),       # 256 + 248: remainder rounded up to a full 256-wide group
+]
+
+
+@pytest.mark.parametrize("kw", [dict(), dict(fuse_tail=-1), dict(max_ctas=6, comm_ctas=2), dict(static_schedule=1, raster_group=1), dict(wg_tail=0),
+                                dict(wg_tail=0, comm_ctas=2, max_ctas=12)],
+                         ids=["default", "separate_tail_tile", "small_grid", "static", "tail_rule", "takeover"])
+@pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
+@pytest.mark.parametrize("W,M,nl,K", RAGGED_PAIR_SHAPES)
+def test_ragged_shard_remainder_fused_with_last_full_tile(mode, W, M, nl, K, kw):
+    """A shard that is not a whole number of 256-column tiles: by default the pair that computes the last full tile also
+    computes the remainder columns (second MMA group on the same A stages, second accumulator); fuse_tail = -1 makes the
+    remainder a tile of its own.  Either way the heap image is the oracle's, twice in a row."""
+    N, dtype = W * nl, "bf16"
+    A = inputs.matrix(73, inputs.STREAM_A, M, K, "ternary:0.5", dtype)
+    Bs = [inputs.matrix(73, inputs.STREAM_B0 + r, nl, K, "smallint:2", dtype) for r in range(W)]
+    bpr = gemm_layout(M, N, W, True)[4]
+    with GpuHeap(W, bpr) as g:
+        c_full = None
+        for epoch in (1, 2):
+            run_gemm(g, A, Bs, dtype, mode, epoch=epoch, with_locks_zeroed=(epoch == 1), **kw)
+            host = g.to_host()
+            img, c_full = expected_image(g, A, Bs, dtype, mode, epoch=epoch, c_full=c_full)
+            assert np.array_equal(host, img.mem), (epoch, first_diff(host, img.mem))
+
+
 @pytest.mark.parametrize("block_n", [128, 256])
 @pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
 def test_exact_integer_gemm_tile_width_and_grid_knobs(block_n, mode):
