@@ -289,11 +289,13 @@ typedef struct iris_gemm_args {
                                   shared-memory blocks); results are bit-identical to the other
                                   layout's on the transposed data                                */
   int fuse_tail;               /* CTA-pair kernel, shards that are not a whole number of 256-column tiles
-                                  (N/world > 256, K-contiguous B): 0 = the remainder columns are computed
+                                  (N/world > 256, K-contiguous B): 1 = the remainder columns are computed
                                   by the pair that computes the shard's last full tile, as a second MMA
                                   group on the same A stages with its own accumulator (a narrow tile of
                                   its own would load as much of A as a full one); -1 = the remainder is
-                                  a tile of its own.  Same results either way                      */
+                                  a tile of its own; 0 = the library chooses (fused, except in
+                                  workgroup_specialized mode with fewer than three waves of work).
+                                  Same results either way                                          */
 } iris_gemm_args;
 
 /* Enqueue the whole operation on `stream` (bulk-synchronous: two kernels; otherwise one).

@@ -1005,15 +1005,18 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         // tile (measured from the previous tile; nothing is left to protect in the last wave, which goes at once).
         if (tm < p.ptiles_m) {
           const uint64_t t0 = globaltimer_ns();
-          if (prev_issue != 0) period_ns = (uint32_t)min((uint64_t)(4u * p.t_tile_ns + 1000u), t0 - prev_issue);
-          prev_issue = t0;
+          if (l == 0) {   // per work unit
+            if (prev_issue != 0) period_ns = (uint32_t)min((uint64_t)(4u * p.t_tile_ns + 1000u), t0 - prev_issue);
+            prev_issue = t0;
+          }
           int boxes = 0;
 #pragma unroll
           for (int b = 0; b < kPairBN / 64; ++b) boxes += col_in_shard + 64 * b < p.n_local ? 1 : 0;
           const bool last_wave = tile >= p.total_ctiles - (p.gemm_ctas >> 1);
           // (a tile that is handed over goes at once: the communication CTAs are waiting for it)
           const bool hand_over = !seq && p.mode == IRIS_MODE_WORKGROUP_SPECIALIZED;
-          const uint32_t gap_ns = (p.pace_stores && !last_wave && !hand_over) ? (period_ns / 4u * 3u) / (uint32_t)(boxes * (seq ? W : 1)) : 0u;
+          // (nor is the first tile of a two-tile unit: the second accumulator waits behind it and the MMA thread behind both)
+          const uint32_t gap_ns = (p.pace_stores && !last_wave && !hand_over && l == nsub - 1) ? (period_ns / 4u * 3u) / (uint32_t)(boxes * (seq ? W : 1)) : 0u;
           uint64_t due = t0;
           for (int s = 0; s < W; ++s) {
             if (!seq && s != tc.rank) continue;
@@ -1384,6 +1387,13 @@ static int build_plan(const iris_gemm_args* a, const PlanEnv& env, Plan& out) {
   // Ragged shard on the pair kernel: the remainder after the last full 256-column tile is computed by the pair that
   // computes that tile, on the same A stages (a 64-column tile of its own would pull in as much of A as a full one).
   p.fuse_last = (pair && a->fuse_tail >= 0 && a->b_layout == IRIS_B_N_BY_K && nl > kPairBN && nl % kPairBN != 0) ? 1 : 0;
+  if (p.fuse_last && wg && a->fuse_tail == 0) {
+    // workgroup_specialized hands the last wave to the producers: with fewer than three waves of the (longer, fewer) fused
+    // units that wave is too large a share of the work (measured: 4096 x 2560 x 8192, two waves, 0.247 vs 0.223 ms)
+    const int64_t units = (int64_t)((a->M + 2 * BM - 1) / (2 * BM)) * rank_count * (nl / kPairBN);
+    const int pairs_guess = std::max(1, (a->max_ctas ? std::min(a->max_ctas, env.sm_count) : env.sm_count) / 2);
+    if (units < 3 * (int64_t)pairs_guess) p.fuse_last = 0;
+  }
   p.stage_bytes = kPairStageBytes;
   p.n_stages = kPairStages;
   if (p.fuse_last) {
@@ -1601,7 +1611,7 @@ static int enqueue_gemm_all_scatter(const iris_gemm_args* a, void* stream, bool 
   if (a->pace_stores < -1 || a->pace_stores > 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: pace_stores must be 0 or -1");
   if (a->wg_tail < -1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: wg_tail must be -1, 0 or a tile count");
   if (a->stream_k < -1 || a->stream_k > 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: stream_k must be -1, 0 or 1");
-  if (a->fuse_tail < -1 || a->fuse_tail > 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: fuse_tail must be 0 or -1");
+  if (a->fuse_tail < -1 || a->fuse_tail > 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: fuse_tail must be -1, 0 or 1");
   if (a->b_layout != IRIS_B_N_BY_K && a->b_layout != IRIS_B_K_BY_N) return fail(IRIS_ERR_ARG, "gemm_all_scatter: unknown b_layout %d", a->b_layout);
   if (a->rank_first < 0 || a->rank_count < 0 || a->rank_first + a->rank_count > W || (a->rank_count == 0 && a->rank_first != 0))
     return fail(IRIS_ERR_ARG, "gemm_all_scatter: rank range [%d, %d) outside [0, %d)", a->rank_first, a->rank_first + a->rank_count, W);

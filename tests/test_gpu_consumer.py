@@ -122,8 +122,8 @@ FUSED_SHAPES = [
     (4, 640, 512, 128, dict(static_schedule=1, max_ctas=12, comm_ctas=4)),
     (4, 130, 136, 72, dict()),                       # ragged: single-CTA kernel, consumer follows as a kernel
     (2, 384, 256, 192, dict(cta_pair=-1)),
-    (3, 520, 392, 328, dict()),                      # CTA pairs, ragged shard: the remainder rides with the last full tile
-    (2, 600, 576, 136, dict(comm_ctas=4)),           # 576 = 2 x 256 + 64: one plain unit and one fused unit per shard
+    (3, 520, 392, 328, dict(fuse_tail=1)),           # CTA pairs, ragged shard: the remainder rides with the last full tile
+    (2, 600, 576, 136, dict(fuse_tail=1, comm_ctas=4)),   # 576 = 2 x 256 + 64: one plain unit and one fused unit per shard
     (2, 600, 576, 136, dict(fuse_tail=-1)),          # the same with the remainder as a tile of its own
 ]
 

@@ -178,9 +178,10 @@ RAGGED_PAIR_SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("kw", [dict(), dict(fuse_tail=-1), dict(max_ctas=6, comm_ctas=2), dict(static_schedule=1, raster_group=1), dict(wg_tail=0),
-                                dict(wg_tail=0, comm_ctas=2, max_ctas=12)],
-                         ids=["default", "separate_tail_tile", "small_grid", "static", "tail_rule", "takeover"])
+@pytest.mark.parametrize("kw", [dict(), dict(fuse_tail=1), dict(fuse_tail=-1), dict(fuse_tail=1, max_ctas=6, comm_ctas=2),
+                                dict(fuse_tail=1, static_schedule=1, raster_group=1), dict(fuse_tail=1, wg_tail=0),
+                                dict(fuse_tail=1, wg_tail=0, comm_ctas=2, max_ctas=12)],
+                         ids=["default", "fused", "separate_tail_tile", "small_grid", "static", "tail_rule", "takeover"])
 @pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
 @pytest.mark.parametrize("W,M,nl,K", RAGGED_PAIR_SHAPES)
 def test_ragged_shard_remainder_fused_with_last_full_tile(mode, W, M, nl, K, kw):
