@@ -35,6 +35,7 @@ WORKLOADS = {
     # name: (W, M, N, K, dist, dtype)
     "cfg5_w8_m8192_n16384_k16384": (8, 8192, 16384, 16384, "uniform", "bf16"),
     "cfg5_w8_m1024_n16384_k16384": (8, 1024, 16384, 16384, "uniform", "bf16"),
+    "cfg5_w8_m2048_n16384_k16384": (8, 2048, 16384, 16384, "uniform", "bf16"),   # a quarter of the headline's rows: the size ncu's full set is taken on
     "cfg5_w4_m8192_n16384_k16384": (4, 8192, 16384, 16384, "uniform", "bf16"),
     "cfg5_w4_m1024_n16384_k16384": (4, 1024, 16384, 16384, "uniform", "bf16"),
     "cfg5_w2_m8192_n16384_k16384": (2, 8192, 16384, 16384, "uniform", "bf16"),
@@ -444,8 +445,12 @@ def run_ours(args):
 
         # ---------------- consumer launched on a second stream right after the producer (it overlaps the GEMM) ----------------
         # End-to-end time from the producer's launch to the end of the last kernel, next to the same two kernels on one stream.
-        if args.mode_iters > 0:
+        # (not in bulk_synchronous mode: there the flags come from the second kernel of the call, after the GEMM has ended, so
+        # nothing of the consumer can overlap the GEMM -- and a consumer grid that fills every SM's thread slots while it
+        # waits would keep that second kernel from ever starting; the consumer's deadline, not a hang, is what ends that)
+        if args.mode_iters > 0 and args.mode != "bulk_synchronous":
             cons_stream = torch.cuda.Stream()
+            sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
             joined = torch.cuda.Event()
             ts2, ts1 = [], []
             for it in range(1 + args.mode_iters):
@@ -456,7 +461,8 @@ def run_ours(args):
                     e0.record(stream)
                     gemm(epoch)
                     if overlapped:
-                        iris.iris_consume_bias(h, 0, out_off, flag_off, dbias, M, N, W, dt, epoch, stream=cons_stream)
+                        # 4 CTAs per SM: half the thread slots stay free for whatever the producer side still has to launch
+                        iris.iris_consume_bias(h, 0, out_off, flag_off, dbias, M, N, W, dt, epoch, ctas=4 * sm_count, stream=cons_stream)
                         joined.record(cons_stream)
                         stream.wait_event(joined)
                     else:
