@@ -275,6 +275,7 @@ def run_ours(args):
     def gemm(epoch, m=mode, fused=False, wg_tail=None, **kw):
         kw.setdefault("stream", None)
         kw.setdefault("fuse_tail", args.fuse_tail)
+        kw.setdefault("stage_k", args.stage_k)
         iris.iris_gemm_all_scatter_ex(h, dA, dB, M, N, K, W, m, dt, 0, flag_off, lock_off, epoch, comm_ctas=args.comm_ctas,
                                       raster_group=args.raster_group, block_n=args.block_n, cta_pair=args.cta_pair, static_schedule=args.static_schedule, stream_k=args.stream_k,
                                       wg_tail=args.wg_tail if wg_tail is None else wg_tail,
@@ -701,6 +702,7 @@ def main():
     ap.add_argument("--stream-k", type=int, default=0)
     ap.add_argument("--wg-tail", type=int, default=0, help="workgroup_specialized: 0 = producers scatter the last wave themselves, -1 = never, n = last n tiles")
     ap.add_argument("--fuse-tail", type=int, default=0, help="-1 = a ragged shard's remainder columns are a tile of their own")
+    ap.add_argument("--stage-k", type=int, default=0, help="pair kernel: 64 or 128 columns of K per operand stage (0 = 128)")
     ap.add_argument("--mode-iters", type=int, default=3)
     ap.add_argument("--steady-seconds", type=float, default=1.0, help="length of the back-to-back loop behind roofline.steady (0 = skip)")
     ap.add_argument("--e2e-steps", type=int, default=2)

@@ -50,7 +50,7 @@ class GemmArgs(C.Structure):
         ("c_off", C.c_uint64), ("flag_off", C.c_uint64), ("lock_off", C.c_uint64),
         ("epoch", C.c_int32), ("comm_ctas", C.c_int), ("max_ctas", C.c_int), ("raster_group", C.c_int),
         ("block_n", C.c_int), ("spin_timeout_ns", C.c_uint64), ("cta_pair", C.c_int), ("static_schedule", C.c_int), ("stream_k", C.c_int), ("wg_tail", C.c_int), ("rank_first", C.c_int), ("rank_count", C.c_int), ("pace_stores", C.c_int),
-        ("consumer_bias", C.c_void_p), ("consumer_out_off", C.c_uint64), ("b_layout", C.c_int), ("fuse_tail", C.c_int),
+        ("consumer_bias", C.c_void_p), ("consumer_out_off", C.c_uint64), ("b_layout", C.c_int), ("fuse_tail", C.c_int), ("stage_k", C.c_int),
     ]
 
 
@@ -292,10 +292,10 @@ def _shards(B_shards):
 
 
 def iris_gemm_all_scatter_ex(heap, A, B_shards, M, N, K, world, mode, dtype, c_off, flag_off, lock_off=0, epoch=1,
-                             comm_ctas=0, max_ctas=0, raster_group=0, block_n=0, spin_timeout_ns=0, cta_pair=0, static_schedule=0, stream_k=0, wg_tail=0, rank_first=0, rank_count=0, pace_stores=0, consumer_bias=None, consumer_out_off=0, b_layout=0, fuse_tail=0, stream=None, comm_stream=None):
+                             comm_ctas=0, max_ctas=0, raster_group=0, block_n=0, spin_timeout_ns=0, cta_pair=0, static_schedule=0, stream_k=0, wg_tail=0, rank_first=0, rank_count=0, pace_stores=0, consumer_bias=None, consumer_out_off=0, b_layout=0, fuse_tail=0, stage_k=0, stream=None, comm_stream=None):
     arr = _shards(B_shards)
     a = GemmArgs(_ptr(A), C.cast(arr, C.POINTER(C.c_void_p)), heap, M, N, K, world, mode, dtype, c_off, flag_off, lock_off,
-                 epoch, comm_ctas, max_ctas, raster_group, block_n, spin_timeout_ns, cta_pair, static_schedule, stream_k, wg_tail, rank_first, rank_count, pace_stores, _ptr(consumer_bias), consumer_out_off, b_layout, fuse_tail)
+                 epoch, comm_ctas, max_ctas, raster_group, block_n, spin_timeout_ns, cta_pair, static_schedule, stream_k, wg_tail, rank_first, rank_count, pace_stores, _ptr(consumer_bias), consumer_out_off, b_layout, fuse_tail, stage_k)
     if comm_stream is not None:     # the two-kernel, two-stream form (producers on `stream`, communication kernel on `comm_stream`)
         _ck(lib().iris_gemm_all_scatter_unfused(C.byref(a), _stream(stream), _stream(comm_stream)))
     else:

@@ -105,8 +105,9 @@ struct alignas(64) GemmParams {
   int fuse_last;        // pair kernel: 1 = a shard's last full 256-column tile and the narrow remainder after it are ONE work unit
                         // (two MMA groups on the same A stages, one accumulator each): the remainder no longer costs its own
                         // loads of A.  ctiles_per_rank / total_ctiles then count work units, one fewer per shard than tiles
-  int stage_bytes;      // pair kernel: bytes of one operand stage (32 KB, plus the remainder's B rows with fuse_last) ...
-  int n_stages;         // ... and how many of them fit beside the store boxes (5, 4 or 3)
+  int kb_per_stage;     // pair kernel: 64-wide k-blocks per operand stage (2: the boxes of two adjacent k-blocks are requested together)
+  int stage_bytes;      // pair kernel: bytes of one operand stage (32 KB per k-block, plus the remainder's B rows with fuse_last) ...
+  int n_stages;         // ... and how many of them the 192 KB ring holds (3 to 6)
   int b1_bytes;         // fuse_last: bytes of the remainder's B box per CTA
   int b_mn;             // 1 = B_r is [K, N_local] row-major (N contiguous): 64 x 64 boxes, MN-major descriptor; 0 = [N_local, K]
   int pace_stores;      // pair kernel: 1 = the epilogue spreads a tile's box stores over most of the next tile's main loop
@@ -753,15 +754,16 @@ __device__ __forceinline__ int pair_tile_cols(const GemmParams& p, int jn) {
   const int left = p.n_local - jn * kPairBN;
   return left >= kPairBN ? kPairBN : ((left + 31) & ~31);
 }
-constexpr int kPairStageBytes = 2 * BM * BK * 2;            // 32 KB: A slice + B half
-constexpr int kPairStages = 5;
-constexpr int kPairStoreBytes = (kPairBN / 64) * kStoreBoxBytes;   // 64 KB: this CTA's 128 x 256 half of the converted tile
-constexpr int kPairSmemPayload = kPairStages * kPairStageBytes + kPairStoreBytes;   // 224 KB
+constexpr int kPairStageBytes = 2 * BM * BK * 2;            // 32 KB: A slice + B half of one 64-wide k-block
+constexpr int kPairRingBytes = 192 * 1024;                  // operand stages: 3 x 64 KB (two k-blocks per stage), 6 x 32 KB, or fewer, larger ones
+constexpr int kPairMaxStages = 6;
+constexpr int kPairStoreBytes = 2 * kStoreBoxBytes;         // 32 KB: 128 converted columns of this CTA's half tile on their way out
+constexpr int kPairSmemPayload = kPairRingBytes + kPairStoreBytes;   // 224 KB
 constexpr int kPairSmemTotal = kPairSmemPayload + kSmemCtrl + 1024;
 static_assert(kPairSmemPayload >= kCommWarps * kTileBytes, "communication warps' tile buffers share the payload area");
 static_assert(kPairSmemTotal <= 232448, "shared memory per CTA");
 
-template <bool BF16, bool STATIC_LOCKS = false, bool CONSUMER = false>
+template <bool BF16, bool STATIC_LOCKS = false, bool CONSUMER = false, int KBS = 2>
 __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1) gemm_all_scatter_pair_kernel(const __grid_constant__ GemmParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* payload = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -774,7 +776,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
   const int W = p.tab.world;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < kPairStages; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->empty[i]), 1); }
+    for (int i = 0; i < kPairMaxStages; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->empty[i]), 1); }
     for (int i = 0; i < 2; ++i) { ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_full[i]), 1); ptx::mbar_init(ptx::smem_u32(&ctrl->tmem_empty[i]), 8); }
     for (int i = 0; i < kCommWarps; ++i) ptx::mbar_init(ptx::smem_u32(&ctrl->comm_full[i]), 1);
     // tile feed: one publisher; readers = the leader's MMA thread + 4 epilogue warps, the peer's producer + 4 epilogue warps
@@ -849,19 +851,32 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         const bool fused = p.fuse_last && tc.jn == p.ctiles_per_rank - 1;
         const int ncols1 = fused ? pair_tile_cols(p, tc.jn + 1) : 0;
         bool ok = true;
-        for (int kb = 0; kb < p.kblocks; ++kb) {
+        constexpr int kbs = KBS;   // 64-wide k-blocks per stage (= p.kb_per_stage)
+        for (int kb = 0; kb < p.kblocks; kb += kbs) {
+          const int nk = min(kbs, p.kblocks - kb);   // k-blocks in this stage (the last stage of an odd count holds one)
           if (!mbar_wait(ptx::smem_u32(&ctrl->empty[stage]), phase ^ 1, p, ctrl, tile)) { ok = false; break; }
           const uint32_t full_local = ptx::smem_u32(&ctrl->full[stage]);
-          if (leader) ptx::mbar_arrive_expect_tx(full_local, 2 * (kPairStageBytes + (fused ? p.b1_bytes : 0)));
+          if (leader) ptx::mbar_arrive_expect_tx(full_local, 2 * (nk * kPairStageBytes + (fused ? p.b1_bytes : 0)));
           const uint32_t full_leader = ptx::mapa(full_local, 0);
           const uint32_t sa = ptx::smem_u32(payload + stage * p.stage_bytes);
-          ptx::tma_load_2d_pair(sa, &p.tmA, kb * BK, tc.tm * 2 * BM + cta_rank * BM, full_leader);
-          if (p.b_mn) {   // this CTA's half of the tile's columns as two [64 k][64 n] blocks
+          // A stage is nk sub-stages [A 16 KB | B 16 KB].  The boxes of adjacent k-blocks (the next 128 bytes of the same rows)
+          // are requested back to back: measured with a load-only probe on L2-resident data, one SM sustains 46-55 B/clk with
+          // one k-block per stage and 76-88 B/clk with two, and this main loop needs 64.
+#pragma unroll
+          for (int j = 0; j < kbs; ++j)
+            if (j < nk) ptx::tma_load_2d_pair(sa + j * kPairStageBytes, &p.tmA, (kb + j) * BK, tc.tm * 2 * BM + cta_rank * BM, full_leader);
+          if (p.b_mn) {   // this CTA's half of the tile's columns as two [64 k][64 n] blocks per k-block
             const int n0 = tc.jn * kPairBN + cta_rank * (ncols / 2);
-            ptx::tma_load_2d_pair(sa + BM * BK * 2, &p.tmB[tc.rank], n0, kb * BK, full_leader);
-            ptx::tma_load_2d_pair(sa + BM * BK * 2 + kMnBlockBytes, &p.tmB[tc.rank], n0 + 64, kb * BK, full_leader);
+#pragma unroll
+            for (int j = 0; j < kbs; ++j)
+              if (j < nk) {
+                ptx::tma_load_2d_pair(sa + j * kPairStageBytes + BM * BK * 2, &p.tmB[tc.rank], n0, (kb + j) * BK, full_leader);
+                ptx::tma_load_2d_pair(sa + j * kPairStageBytes + BM * BK * 2 + kMnBlockBytes, &p.tmB[tc.rank], n0 + 64, (kb + j) * BK, full_leader);
+              }
           } else {
-            ptx::tma_load_2d_pair(sa + BM * BK * 2, &p.tmB[tc.rank], kb * BK, tc.jn * kPairBN + cta_rank * (ncols / 2), full_leader);
+#pragma unroll
+            for (int j = 0; j < kbs; ++j)
+              if (j < nk) ptx::tma_load_2d_pair(sa + j * kPairStageBytes + BM * BK * 2, &p.tmB[tc.rank], (kb + j) * BK, tc.jn * kPairBN + cta_rank * (ncols / 2), full_leader);
           }
           if (fused) ptx::tma_load_2d_pair(sa + kPairStageBytes, &p.tmBn[tc.rank], kb * BK, (tc.jn + 1) * kPairBN + cta_rank * (ncols1 / 2), full_leader);
           if (++stage == p.n_stages) { stage = 0; phase ^= 1; }
@@ -897,16 +912,24 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         const uint32_t idesc1 = fused ? ptx::idesc_f16(2 * BM, pair_tile_cols(p, tc.jn + 1), BF16 ? 1 : 0) : 0u;
         const uint64_t b_kstep = p.b_mn ? (uint64_t)(2 * 1024 >> 4) : 2u;
         bool ok = true;
-        for (int kb = 0; kb < p.kblocks; ++kb) {
+        constexpr int kbs = KBS;
+        for (int kb = 0; kb < p.kblocks; kb += kbs) {
+          const int nk = min(kbs, p.kblocks - kb);
           if (!mbar_wait(ptx::smem_u32(&ctrl->full[stage]), phase, p, ctrl, tile)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t sa = ptx::smem_u32(payload + stage * p.stage_bytes);
-          const uint64_t adesc = ptx::smem_desc_k_sw128(sa);
-          const uint64_t bdesc = p.b_mn ? ptx::smem_desc_mn_sw128(sa + BM * BK * 2, kMnBlockBytes) : ptx::smem_desc_k_sw128(sa + BM * BK * 2);
 #pragma unroll
-          for (int k = 0; k < BK / UMMA_K; ++k)
-            ptx::mma_f16_ss_pair(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)k * b_kstep, idesc, (kb | k) != 0);
-          if (fused) {   // the remainder tile: same A stage, its own B rows, the other accumulator
+          for (int j = 0; j < kbs; ++j) {
+            if (j >= nk) break;
+            const uint32_t sj = sa + j * kPairStageBytes;
+            const uint64_t adesc = ptx::smem_desc_k_sw128(sj);
+            const uint64_t bdesc = p.b_mn ? ptx::smem_desc_mn_sw128(sj + BM * BK * 2, kMnBlockBytes) : ptx::smem_desc_k_sw128(sj + BM * BK * 2);
+#pragma unroll
+            for (int k = 0; k < BK / UMMA_K; ++k)
+              ptx::mma_f16_ss_pair(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)k * b_kstep, idesc, (kb | j | k) != 0);
+          }
+          if (fused) {   // the remainder tile (one k-block per stage here): same A stage, its own B rows, the other accumulator
+            const uint64_t adesc = ptx::smem_desc_k_sw128(sa);
             const uint64_t b1desc = ptx::smem_desc_k_sw128(sa + kPairStageBytes);
 #pragma unroll
             for (int k = 0; k < BK / UMMA_K; ++k)
@@ -950,90 +973,108 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
       // Scatter to every slot (Listing 4) or store locally and hand over (Listings 3, 5).  Below seq_from the
       // workgroup-specialised schedule hands over unless the takeover rule (decided by thread 0 further down) keeps the tile.
       bool seq = tile >= p.seq_from;
-      // Convert and stage this CTA's 128 x 256 half in shared memory as four 64-column boxes in the 128B-swizzle
-      // layout of the store maps: a lane owns a row, so its 16-byte pieces go to (piece ^ row % 8) and a warp's
-      // 512 bytes per instruction spread over all banks.  (The previous tile's stores have been waited for
-      // before the barrier at the top of this loop, so the boxes are free.)
-      const uint32_t stg = ptx::smem_u32(payload + kPairStages * kPairStageBytes);
+      // Convert and stage this CTA's 128 x 256 half in shared memory, 128 columns at a time, as two 64-column boxes in the
+      // 128B-swizzle layout of the store maps: a lane owns a row, so its 16-byte pieces go to (piece ^ row % 8) and a
+      // warp's 512 bytes per instruction spread over all banks.  One thread sends the boxes out with TMA: whole 128-byte
+      // lines, clipped by the maps at row M and column N_local, to the owner's slot or (Listing 4's loop over all ranks)
+      // to all.  (The previous tile's stores have been waited for before the barrier at the top of this loop.)
+      // Stores and operand loads leave the SM through one queue: a burst of W x 4 boxes (512 KB, 9 us of the port) holds
+      // up the loads of the tile that is being multiplied meanwhile for longer than the stage ring covers.  So the boxes
+      // go out one at a time, spread over three quarters of the time this CTA takes per tile (measured from the previous
+      // tile; nothing is left to protect in the last wave, which goes at once).  The accumulator goes back to the MMA
+      // warp when its last column has been read, before the second half's stores.
+      constexpr int cpr = 4;                              // 32-column chunks per round: 128 columns, two store boxes
+      const uint32_t stg = ptx::smem_u32(payload + kPairRingBytes);
       const int chunks = pair_tile_cols(p, tc.jn) / 32;   // 8, fewer for the narrow last tile of a ragged shard
+      const int halves = (chunks + cpr - 1) / cpr;
+      const int a_cur = acc;
+      uint32_t gap_ns = 0;     // thread 0: pause between two boxes
+      uint64_t due = 0;        // thread 0: when the next box may go
+      for (int hf = 0; hf < halves; ++hf) {
+        const int ch_end = min(chunks, cpr * hf + cpr);
 #pragma unroll 1
-      for (int ch = 0; ch < chunks; ++ch) {
-        uint32_t v[32];
-        ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * kPairBN + ch * 32), v);
-        ptx::tmem_wait_ld();
-        const uint32_t row_base = stg + (uint32_t)((ch >> 1) * kStoreBoxBytes + row_in_half * 128);
+        for (int ch = cpr * hf; ch < ch_end; ++ch) {
+          uint32_t v[32];
+          ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(a_cur * kPairBN + ch * 32), v);
+          ptx::tmem_wait_ld();
+          const uint32_t row_base = stg + (uint32_t)((((ch - cpr * hf) >> 1)) * kStoreBoxBytes + row_in_half * 128);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          uint4 q;
-          if (p.kblocks == 0) {
-            q = make_uint4(0, 0, 0, 0);   // K == 0: the sum is empty
-          } else {
-            q.x = pack2<BF16>(v[8 * i + 0], v[8 * i + 1]);
-            q.y = pack2<BF16>(v[8 * i + 2], v[8 * i + 3]);
-            q.z = pack2<BF16>(v[8 * i + 4], v[8 * i + 5]);
-            q.w = pack2<BF16>(v[8 * i + 6], v[8 * i + 7]);
+          for (int i = 0; i < 4; ++i) {
+            uint4 q;
+            if (p.kblocks == 0) {
+              q = make_uint4(0, 0, 0, 0);   // K == 0: the sum is empty
+            } else {
+              q.x = pack2<BF16>(v[8 * i + 0], v[8 * i + 1]);
+              q.y = pack2<BF16>(v[8 * i + 2], v[8 * i + 3]);
+              q.z = pack2<BF16>(v[8 * i + 4], v[8 * i + 5]);
+              q.w = pack2<BF16>(v[8 * i + 6], v[8 * i + 7]);
+            }
+            const int piece = (ch & 1) * 4 + i;
+            ptx::st_shared_v4(row_base + (uint32_t)(((piece ^ (row_in_half & 7)) << 4)), q);
           }
-          const int piece = (ch & 1) * 4 + i;
-          ptx::st_shared_v4(row_base + (uint32_t)(((piece ^ (row_in_half & 7)) << 4)), q);
         }
-      }
-      // accumulator drained: hand it back to the MMA warp before the stores go out
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&ctrl->tmem_empty[acc]), 0));
-      if (++acc == 2) { acc = 0; acc_phase ^= 1; }
-      fence_proxy_async();   // this thread's shared-memory writes -> the TMA unit's reads
-      asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
-      if (et == 0) {
-        if (p.takeover && !seq && tm < p.ptiles_m) {
-          // Hand over only what the communication warps can still finish: their backlog plus this CTA's publication
-          // tiles, at t_pt_ns each spread over all of them, against the main-loop time of the waves still to come.
-          // Near the end of the kernel (and whenever they fall behind) the producers' own store ports take the rest.
-          const int mine = min(kPairBN / IRIS_TILE, p.ptiles_per_rank - tc.jn * (kPairBN / IRIS_TILE));
-          const int waves_left = (p.total_ctiles - 1 - tile) / (p.gemm_ctas >> 1);
-          const int queued = ld_relaxed_gpu(p.backlog);
-          seq = (uint64_t)(queued + mine) * p.t_pt_ns > (uint64_t)waves_left * p.t_tile_ns * (uint64_t)(p.comm_ctas * kCommWarps);
-          if (seq) atomicAdd(p.backlog + 1, 1);
-          else atomicAdd(p.backlog, mine);
+        if (hf == halves - 1) {   // accumulator drained: hand it back to the MMA warp before the last stores go out
+          ptx::tc_fence_before();
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive_cluster(ptx::mapa(ptx::smem_u32(&ctrl->tmem_empty[acc]), 0));
+          if (++acc == 2) { acc = 0; acc_phase ^= 1; }
         }
-        ctrl->keep_tile = seq ? 1 : 0;
-        // One thread stores the boxes with TMA: whole 128-byte lines, clipped by the maps at row M and column
-        // N_local, to the owner's slot or (Listing 4's loop over all ranks) to all.
-        // Stores and operand loads leave the SM through one queue: a burst of W x 4 boxes (512 KB, 9 us of the
-        // port) holds up the loads of the tile that is being multiplied meanwhile for longer than the stage ring
-        // covers.  So the boxes go out one at a time, spread over three quarters of the time this CTA takes per
-        // tile (measured from the previous tile; nothing is left to protect in the last wave, which goes at once).
-        if (tm < p.ptiles_m) {
-          const uint64_t t0 = globaltimer_ns();
-          if (l == 0) {   // per work unit
-            if (prev_issue != 0) period_ns = (uint32_t)min((uint64_t)(4u * p.t_tile_ns + 1000u), t0 - prev_issue);
-            prev_issue = t0;
+        fence_proxy_async();   // this thread's shared-memory writes -> the TMA unit's reads
+        asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
+        if (et == 0) {
+          if (hf == 0) {
+            if (p.takeover && !seq && tm < p.ptiles_m) {
+              // Hand over only what the communication warps can still finish: their backlog plus this CTA's publication
+              // tiles, at t_pt_ns each spread over all of them, against the main-loop time of the waves still to come.
+              // Near the end of the kernel (and whenever they fall behind) the producers' own store ports take the rest.
+              const int mine = min(kPairBN / IRIS_TILE, p.ptiles_per_rank - tc.jn * (kPairBN / IRIS_TILE));
+              const int waves_left = (p.total_ctiles - 1 - tile) / (p.gemm_ctas >> 1);
+              const int queued = ld_relaxed_gpu(p.backlog);
+              seq = (uint64_t)(queued + mine) * p.t_pt_ns > (uint64_t)waves_left * p.t_tile_ns * (uint64_t)(p.comm_ctas * kCommWarps);
+              if (seq) atomicAdd(p.backlog + 1, 1);
+              else atomicAdd(p.backlog, mine);
+            }
+            ctrl->keep_tile = seq ? 1 : 0;
+            const uint64_t t0 = globaltimer_ns();
+            if (l == 0) {   // per work unit
+              if (prev_issue != 0) period_ns = (uint32_t)min((uint64_t)(4u * p.t_tile_ns + 1000u), t0 - prev_issue);
+              prev_issue = t0;
+            }
+            int boxes = 0;
+#pragma unroll
+            for (int b = 0; b < kPairBN / 64; ++b) boxes += col_in_shard + 64 * b < p.n_local ? 1 : 0;
+            const bool last_wave = tile >= p.total_ctiles - (p.gemm_ctas >> 1);
+            // (a tile that is handed over goes at once: the communication CTAs are waiting for it)
+            const bool hand_over = !seq && p.mode == IRIS_MODE_WORKGROUP_SPECIALIZED;
+            // (nor is the first tile of a two-tile unit paced: the second accumulator waits behind it and the MMA thread behind both)
+            gap_ns = (p.pace_stores && !last_wave && !hand_over && l == nsub - 1) ? (period_ns / 4u * 3u) / (uint32_t)(boxes * (seq ? W : 1)) : 0u;
+            due = t0;
           }
-          int boxes = 0;
+          if (tm < p.ptiles_m) {
+            for (int s = 0; s < W; ++s) {
+              if (!seq && s != tc.rank) continue;
 #pragma unroll
-          for (int b = 0; b < kPairBN / 64; ++b) boxes += col_in_shard + 64 * b < p.n_local ? 1 : 0;
-          const bool last_wave = tile >= p.total_ctiles - (p.gemm_ctas >> 1);
-          // (a tile that is handed over goes at once: the communication CTAs are waiting for it)
-          const bool hand_over = !seq && p.mode == IRIS_MODE_WORKGROUP_SPECIALIZED;
-          // (nor is the first tile of a two-tile unit: the second accumulator waits behind it and the MMA thread behind both)
-          const uint32_t gap_ns = (p.pace_stores && !last_wave && !hand_over && l == nsub - 1) ? (period_ns / 4u * 3u) / (uint32_t)(boxes * (seq ? W : 1)) : 0u;
-          uint64_t due = t0;
-          for (int s = 0; s < W; ++s) {
-            if (!seq && s != tc.rank) continue;
-#pragma unroll
-            for (int b = 0; b < kPairBN / 64; ++b)
-              if (col_in_shard + 64 * b < p.n_local) {
-                if (gap_ns) {
-                  while (globaltimer_ns() < due) __nanosleep(64);
-                  due += gap_ns;
+              for (int b = 0; b < cpr / 2; ++b) {
+                const int col = col_in_shard + hf * cpr * 32 + 64 * b;
+                if (col < p.n_local) {
+                  if (gap_ns) {
+                    while (globaltimer_ns() < due) __nanosleep(64);
+                    due += gap_ns;
+                  }
+                  ptx::tma_store_4d(&p.tmC4s, col, tm * BM, tc.rank, s, stg + (uint32_t)(b * kStoreBoxBytes));
                 }
-                ptx::tma_store_4d(&p.tmC4s, col_in_shard + 64 * b, tm * BM, tc.rank, s, stg + (uint32_t)(b * kStoreBoxBytes));
               }
+            }
+            ptx::bulk_commit_group();
           }
-          ptx::bulk_commit_group();
+          if (hf == halves - 1) {
+            ptx::bulk_wait_group<0>();   // stores performed: the boxes are free and the tile may be published
+            fence_proxy_async();         // async-proxy writes above -> the generic-proxy release (flags or lock) after the barrier
+          } else {
+            ptx::bulk_wait_group_read<0>();   // the boxes have been read and may be refilled
+          }
         }
-        ptx::bulk_wait_group<0>();   // stores performed: the boxes are free and the tile may be published
-        fence_proxy_async();         // async-proxy writes above -> the generic-proxy release (flags or lock) after the barrier
+        if (hf != halves - 1) asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
       }
       if (p.mode != IRIS_MODE_BULK_SYNCHRONOUS) {
         asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
@@ -1213,9 +1254,19 @@ static int launch_gemm(const GemmParams& p, int grid, bool cooperative, cudaStre
   return IRIS_OK;
 }
 
+template <bool BF16, bool STATIC_LOCKS, bool CONSUMER, int KBS>
+static int launch_gemm_pair_kbs(const GemmParams& p, int grid, cudaStream_t st, int* max_pairs_out);
+
+// (the kernel is instantiated for one and for two k-blocks per operand stage: p.kb_per_stage selects)
 template <bool BF16, bool STATIC_LOCKS = false, bool CONSUMER = false>
 static int launch_gemm_pair(const GemmParams& p, int grid, cudaStream_t st, int* max_pairs_out) {
-  auto kern = gemm_all_scatter_pair_kernel<BF16, STATIC_LOCKS, CONSUMER>;
+  return p.kb_per_stage == 1 ? launch_gemm_pair_kbs<BF16, STATIC_LOCKS, CONSUMER, 1>(p, grid, st, max_pairs_out)
+                             : launch_gemm_pair_kbs<BF16, STATIC_LOCKS, CONSUMER, 2>(p, grid, st, max_pairs_out);
+}
+
+template <bool BF16, bool STATIC_LOCKS, bool CONSUMER, int KBS>
+static int launch_gemm_pair_kbs(const GemmParams& p, int grid, cudaStream_t st, int* max_pairs_out) {
+  auto kern = gemm_all_scatter_pair_kernel<BF16, STATIC_LOCKS, CONSUMER, KBS>;
   static bool configured[kMaxDevices] = {};
   if (int rc = ensure_smem_limit(reinterpret_cast<const void*>(kern), kPairSmemTotal, configured)) return rc;
   cudaLaunchConfig_t cfg{};
@@ -1314,7 +1365,7 @@ struct PlanKey {
   const void* A; const void* B[IRIS_MAX_WORLD];
   int M, N, K, world, mode, dtype;
   uint64_t c_off, flag_off, lock_off;
-  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail, fused_consumer, rank_first, rank_count, pace_stores, b_layout, fuse_tail;
+  int comm_ctas, max_ctas, raster_group, block_n, cta_pair, static_schedule, stream_k, wg_tail, fused_consumer, rank_first, rank_count, pace_stores, b_layout, fuse_tail, stage_k;
   uint64_t spin_timeout_ns;
 };
 // A few plans are kept (round-robin replacement): a step that alternates between calls -- one per rank shard in the
@@ -1336,7 +1387,7 @@ static void make_key(PlanKey* k, const iris_gemm_args* a, const iris_heap* h) {
   k->c_off = a->c_off; k->flag_off = a->flag_off; k->lock_off = a->lock_off;
   k->comm_ctas = a->comm_ctas; k->max_ctas = a->max_ctas; k->raster_group = a->raster_group; k->block_n = a->block_n;
   k->cta_pair = a->cta_pair; k->static_schedule = a->static_schedule; k->stream_k = a->stream_k; k->wg_tail = a->wg_tail;
-  k->rank_first = a->rank_first; k->rank_count = a->rank_count; k->pace_stores = a->pace_stores; k->b_layout = a->b_layout; k->fuse_tail = a->fuse_tail;
+  k->rank_first = a->rank_first; k->rank_count = a->rank_count; k->pace_stores = a->pace_stores; k->b_layout = a->b_layout; k->fuse_tail = a->fuse_tail; k->stage_k = a->stage_k;
   k->fused_consumer = a->consumer_bias != nullptr;   // the split between producers and communicators depends on it
   k->spin_timeout_ns = a->spin_timeout_ns;
 }
@@ -1394,14 +1445,16 @@ static int build_plan(const iris_gemm_args* a, const PlanEnv& env, Plan& out) {
     const int pairs_guess = std::max(1, (a->max_ctas ? std::min(a->max_ctas, env.sm_count) : env.sm_count) / 2);
     if (units < 3 * (int64_t)pairs_guess) p.fuse_last = 0;
   }
-  p.stage_bytes = kPairStageBytes;
-  p.n_stages = kPairStages;
+  // Operand stages of the pair kernel: two 64-wide k-blocks per stage (3 stages of 64 KB) unless the caller asks for
+  // one (6 of 32 KB) or the stage also carries a fused remainder's B rows (one k-block, 5 or 4 stages).
+  p.kb_per_stage = (p.fuse_last || a->stage_k == 64) ? 1 : 2;
+  p.stage_bytes = p.kb_per_stage * kPairStageBytes;
   if (p.fuse_last) {
     const int rem32 = ((nl % kPairBN) + 31) & ~31;
     p.b1_bytes = (rem32 / 2) * BK * 2;
     p.stage_bytes = kPairStageBytes + (int)align_up((uint64_t)p.b1_bytes, 1024);
-    p.n_stages = std::min(kPairStages, (kPairStages * kPairStageBytes) / p.stage_bytes);
   }
+  p.n_stages = std::min(kPairMaxStages, kPairRingBytes / p.stage_bytes);
   p.tab = env.tab;
   p.c_off = a->c_off;
   p.flag_off = a->flag_off;
@@ -1611,6 +1664,7 @@ static int enqueue_gemm_all_scatter(const iris_gemm_args* a, void* stream, bool 
   if (a->pace_stores < -1 || a->pace_stores > 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: pace_stores must be 0 or -1");
   if (a->wg_tail < -1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: wg_tail must be -1, 0 or a tile count");
   if (a->stream_k < -1 || a->stream_k > 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: stream_k must be -1, 0 or 1");
+  if (a->stage_k != 0 && a->stage_k != 64 && a->stage_k != 128) return fail(IRIS_ERR_ARG, "gemm_all_scatter: stage_k must be 0, 64 or 128");
   if (a->fuse_tail < -1 || a->fuse_tail > 1) return fail(IRIS_ERR_ARG, "gemm_all_scatter: fuse_tail must be -1, 0 or 1");
   if (a->b_layout != IRIS_B_N_BY_K && a->b_layout != IRIS_B_K_BY_N) return fail(IRIS_ERR_ARG, "gemm_all_scatter: unknown b_layout %d", a->b_layout);
   if (a->rank_first < 0 || a->rank_count < 0 || a->rank_first + a->rank_count > W || (a->rank_count == 0 && a->rank_first != 0))

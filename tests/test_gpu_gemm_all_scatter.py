@@ -178,10 +178,10 @@ RAGGED_PAIR_SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("kw", [dict(), dict(fuse_tail=1), dict(fuse_tail=-1), dict(fuse_tail=1, max_ctas=6, comm_ctas=2),
+@pytest.mark.parametrize("kw", [dict(), dict(fuse_tail=1), dict(fuse_tail=-1), dict(fuse_tail=-1, stage_k=64), dict(fuse_tail=1, max_ctas=6, comm_ctas=2),
                                 dict(fuse_tail=1, static_schedule=1, raster_group=1), dict(fuse_tail=1, wg_tail=0),
                                 dict(fuse_tail=1, wg_tail=0, comm_ctas=2, max_ctas=12)],
-                         ids=["default", "fused", "separate_tail_tile", "small_grid", "static", "tail_rule", "takeover"])
+                         ids=["default", "fused", "separate_tail_tile", "separate_tail_tile_k64", "small_grid", "static", "tail_rule", "takeover"])
 @pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
 @pytest.mark.parametrize("W,M,nl,K", RAGGED_PAIR_SHAPES)
 def test_ragged_shard_remainder_fused_with_last_full_tile(mode, W, M, nl, K, kw):
@@ -212,7 +212,8 @@ def test_exact_integer_gemm_tile_width_and_grid_knobs(block_n, mode):
     with GpuHeap(W, bpr) as g:
         img = None
         for kw in (dict(), dict(max_ctas=7, comm_ctas=3, raster_group=2), dict(max_ctas=148, comm_ctas=32, raster_group=1),
-                   dict(cta_pair=-1), dict(cta_pair=-1, max_ctas=5, comm_ctas=2), dict(cta_pair=1 if block_n == 256 else 0, comm_ctas=8), dict(static_schedule=1), dict(static_schedule=1, max_ctas=10, raster_group=3)):
+                   dict(cta_pair=-1), dict(cta_pair=-1, max_ctas=5, comm_ctas=2), dict(cta_pair=1 if block_n == 256 else 0, comm_ctas=8), dict(static_schedule=1), dict(static_schedule=1, max_ctas=10, raster_group=3),
+                   dict(stage_k=64), dict(stage_k=64, max_ctas=6, comm_ctas=2), dict(stage_k=128, static_schedule=1)):
             g.mem.fill_(SENTINEL)
             run_gemm(g, A, Bs, dtype, mode, block_n=block_n, **kw)
             host = g.to_host()
