@@ -1057,7 +1057,9 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
               for (int b = 0; b < cpr / 2; ++b) {
                 const int col = col_in_shard + hf * cpr * 32 + 64 * b;
                 if (col < p.n_local) {
-                  if (gap_ns) {
+                  // (with two-tile units among the work only the round after the accumulator's release is paced: a unit
+                  // that needs both accumulators would wait behind a paced first round for 3/8 of a tile time)
+                  if (gap_ns && (!p.fuse_last || hf == halves - 1)) {
                     while (globaltimer_ns() < due) __nanosleep(64);
                     due += gap_ns;
                   }
