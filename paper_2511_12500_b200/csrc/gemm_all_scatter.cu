@@ -738,8 +738,10 @@ __device__ void consumer_warp(const GemmParams& p, CtrlBlock* ctrl, int cwarp, i
 // tensor core reads its A slice locally and both B halves.  Per CTA and k-step 32 KB are pulled in instead
 // of 48 KB for the same flops per SM: 64 B/clk, which the SM's port to the L2 sustains, instead of 96, which
 // it does not (the single-CTA kernel's tensor pipe is 67 % busy, this one's 92 %).
-// Accumulators: 2 x 256 columns of TMEM in each CTA (rows of its own half).  Shared memory: 5 stages of
-// 32 KB + four 16 KB store boxes (the CTA's converted 128 x 256 half, 128B-swizzled for the TMA stores).
+// Accumulators: 2 x 256 columns of TMEM in each CTA (rows of its own half).  Shared memory: a 192 KB ring of operand
+// stages -- 3 stages of 64 KB holding two 64-wide k-blocks each (sub-stages [A 16 KB | B 16 KB]), whose boxes are
+// requested back to back; or one k-block per stage when asked for or when the stage also carries a fused remainder's
+// B rows -- and two 16 KB store boxes (128 converted columns of the CTA's half tile, 128B-swizzled for the TMA stores).
 //   full[s]        leader only; the leader's producer expects 64 KB, all four loads (two per CTA) complete on it
 //   empty[s]       both CTAs; the leader's tcgen05.commit multicasts the arrival to the pair
 //   tmem_full[a]   both CTAs; multicast commit after a tile's last MMA
