@@ -91,6 +91,38 @@ iris_heap* iris_heap_create(int world, size_t bytes_per_rank);
  * iris_gemm_all_scatter_host() choose their own layout and clear their flag and lock arrays themselves. */
 int iris_heap_create_ex(int world, size_t bytes_per_rank, void* external_base, iris_heap** out);
 
+/* A heap over several processes or devices (Section 3.1: one slot per rank, each in its owner's memory; Section 3.2
+ * steps 3-6: allocate, exchange handles, open the peers' slots, build the table of bases).  bases[0..world) are HOST
+ * values: the device address, in THIS process, of every rank's slot of bytes_per_rank bytes, each 256-byte aligned,
+ * none overlapping another; bases[local_rank] is this process's own allocation, the others are mappings of the
+ * peers' (iris_ipc_open, or any mapping the caller made).  The heap owns none of them and the caller keeps them
+ * alive until iris_heap_destroy.  Nothing is cleared.  What changes on such a heap:
+ *   - ready flags are released and acquired at SYSTEM scope (every other scope in this header stays as written);
+ *   - iris_gemm_all_scatter_ex / _unfused compute this rank's shard only: rank_first must be local_rank and
+ *     rank_count 1 (IRIS_ERR_ARG otherwise).  The locks of the workgroup-specialised schedule are the local
+ *     slot's; tiles go to every slot with TMA stores through one tensor map per slot;
+ *   - iris_consume_bias[_ranks] reads and writes the local slot only;
+ *   - gemm_all_scatter(), iris_gemm_all_scatter_host(), consumer_bias inside the launch and iris_all_store_bench
+ *     emulate all ranks in one process and return IRIS_ERR_UNSUPPORTED.
+ * Between ranks the caller orders things on the host (a barrier before the first launch, so that every rank's flags
+ * are in their initial state, and before the memory is released).  Kernels of different ranks never wait for one
+ * another except the consumer for flags, with the usual deadline. */
+int iris_heap_create_from_bases(int world, size_t bytes_per_rank, const uint64_t* bases, int local_rank, iris_heap** out);
+int iris_heap_local_rank(const iris_heap* heap); /* the local rank of a heap made from bases; -1 for a one-process heap */
+
+/* One rank's slot as memory that other processes can map.  iris_ipc_alloc: `bytes` of device memory on the current
+ * device, cleared to zero (a plain allocation of its own, so that the handle names exactly this range).
+ * iris_ipc_export: writes IRIS_IPC_HANDLE_BYTES bytes that another process passes to iris_ipc_open (in that process:
+ * a device address of the same memory, valid until iris_ipc_close).  A handle cannot be opened by the process that
+ * exported it.  iris_ipc_free / iris_ipc_close synchronise the device first; NULL is a no-op.
+ * Errors: IRIS_ERR_ARG (NULL), IRIS_ERR_NOMEM, IRIS_ERR_CUDA with the runtime's message in iris_last_error(). */
+#define IRIS_IPC_HANDLE_BYTES 64
+int iris_ipc_alloc(size_t bytes, void** ptr_out);
+int iris_ipc_free(void* ptr);
+int iris_ipc_export(void* ptr, unsigned char* handle_out);
+int iris_ipc_open(const unsigned char* handle, void** ptr_out);
+int iris_ipc_close(void* ptr);
+
 /* Free the heap (and its memory if the library owns it).  Synchronises the device first. */
 int iris_heap_destroy(iris_heap* heap);
 

@@ -33,7 +33,8 @@ EXPORTS = [
     "iris_atomic_add_contended", "iris_atomic_cas_contended", "iris_flags_fill", "iris_all_store_bench",
     "iris_gemm_all_scatter_ex", "iris_gemm_all_scatter_unfused", "gemm_all_scatter", "iris_gemm_heap_bytes", "iris_heap_epoch", "iris_num_tiles",
     "iris_consume_bias", "iris_consume_bias_ranks", "iris_gemm_all_scatter_host", "iris_gemm_out_offset", "iris_gemm_takeover_stats",
-    "iris_gemm_all_scatter_noalloc", "iris_atomic_add_u64", "iris_atomic_cas_u64", "iris_copy_tile", "iris_load_tile", "iris_store_tile", "iris_atomic_rmw",
+    "iris_gemm_all_scatter_noalloc", "iris_heap_create_from_bases", "iris_heap_local_rank", "iris_ipc_alloc", "iris_ipc_free", "iris_ipc_export",
+    "iris_ipc_open", "iris_ipc_close", "iris_atomic_add_u64", "iris_atomic_cas_u64", "iris_copy_tile", "iris_load_tile", "iris_store_tile", "iris_atomic_rmw",
 ]
 
 
@@ -71,6 +72,13 @@ def lib() -> C.CDLL:
     L.iris_heap_create.restype = vp
     L.iris_heap_create.argtypes = [ci, sz]
     L.iris_heap_create_ex.argtypes = [ci, sz, vp, C.POINTER(vp)]
+    L.iris_heap_create_from_bases.argtypes = [ci, sz, C.POINTER(u64), ci, C.POINTER(vp)]
+    L.iris_heap_local_rank.argtypes = [vp]
+    L.iris_ipc_alloc.argtypes = [sz, C.POINTER(vp)]
+    L.iris_ipc_free.argtypes = [vp]
+    L.iris_ipc_export.argtypes = [vp, C.c_char_p]
+    L.iris_ipc_open.argtypes = [C.c_char_p, C.POINTER(vp)]
+    L.iris_ipc_close.argtypes = [vp]
     L.iris_heap_destroy.argtypes = [vp]
     L.iris_heap_world.argtypes = [vp]
     L.iris_heap_bytes_per_rank.restype = sz
@@ -153,6 +161,51 @@ def iris_heap_create(world: int, bytes_per_rank: int, external_base=None) -> int
     h = C.c_void_p()
     _ck(lib().iris_heap_create_ex(world, bytes_per_rank, _ptr(external_base), C.byref(h)))
     return h.value
+
+
+def iris_heap_create_from_bases(world: int, bytes_per_rank: int, bases, local_rank: int) -> int:
+    """Heap over several processes: bases[r] = this process's device address of rank r's slot."""
+    if len(bases) != world:
+        raise ValueError("one base per rank")
+    arr = (C.c_uint64 * world)(*[int(b) for b in bases])
+    h = C.c_void_p()
+    _ck(lib().iris_heap_create_from_bases(world, bytes_per_rank, arr, local_rank, C.byref(h)))
+    return h.value
+
+
+def iris_heap_local_rank(heap: int) -> int:
+    return lib().iris_heap_local_rank(heap)
+
+
+IRIS_IPC_HANDLE_BYTES = 64
+
+
+def iris_ipc_alloc(nbytes: int) -> int:
+    p = C.c_void_p()
+    _ck(lib().iris_ipc_alloc(nbytes, C.byref(p)))
+    return p.value
+
+
+def iris_ipc_free(ptr: int):
+    _ck(lib().iris_ipc_free(ptr))
+
+
+def iris_ipc_export(ptr: int) -> bytes:
+    buf = C.create_string_buffer(IRIS_IPC_HANDLE_BYTES)
+    _ck(lib().iris_ipc_export(ptr, buf))
+    return buf.raw
+
+
+def iris_ipc_open(handle: bytes) -> int:
+    if len(handle) != IRIS_IPC_HANDLE_BYTES:
+        raise ValueError("an exported handle has IRIS_IPC_HANDLE_BYTES bytes")
+    p = C.c_void_p()
+    _ck(lib().iris_ipc_open(handle, C.byref(p)))
+    return p.value
+
+
+def iris_ipc_close(ptr: int):
+    _ck(lib().iris_ipc_close(ptr))
 
 
 def iris_heap_destroy(heap: int):

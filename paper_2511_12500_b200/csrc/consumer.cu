@@ -1,4 +1,4 @@
-// Flag-gated consumer: waits (acquire, gpu scope) for a publication tile's ready flag in a slot, then
+// Flag-gated consumer: waits (acquire; gpu scope, system scope on a heap over several processes) for a publication tile's ready flag in a slot, then
 // reads that tile of C and writes OUT = C + bias.  This is the consumer side of the paper's
 // producer-consumer handshake (Section 4.1): poll the tile's flag with acquire-ordered loads and touch
 // the data only once it has been seen set.  HBM-bound: 16-byte coalesced accesses, one warp
@@ -12,25 +12,25 @@ constexpr int kConsThreads = 256;
 template <bool BF16>
 __global__ void __launch_bounds__(kConsThreads) consume_bias_kernel(const __grid_constant__ HeapTable tab, uint64_t c_off, uint64_t out_off, uint64_t flag_off,
                                                                     const uint8_t* bias, int M, int N, int n_local, int tiles_m,
-                                                                    int ptiles_per_rank, int rank_first, int rank_count, int32_t epoch,
-                                                                    uint64_t timeout_ns, int32_t* status) {
+                                                                    int ptiles_per_rank, int rank_first, int rank_count, int slot_first, int slot_count,
+                                                                    int32_t epoch, uint64_t timeout_ns, int32_t* status) {
   const int W = tab.world;
   const int pt_n = W * ptiles_per_rank;            // publication tiles per tile row, all ranks (the flag index uses this)
   const int pt_sel = rank_count * ptiles_per_rank; // ... of the ranks this call covers
-  const int items = tiles_m * pt_sel * W;  // (tile, slot) pairs, tile-major so early tiles are consumed first everywhere
+  const int items = tiles_m * pt_sel * slot_count;  // (tile, slot) pairs, tile-major so early tiles are consumed first everywhere
   for (int it = blockIdx.x; it < items; it += gridDim.x) {
-    const int ti = it / W, s = it % W;
+    const int ti = it / slot_count, s = slot_first + it % slot_count;
     const int tm = ti / pt_sel, rank = rank_first + (ti % pt_sel) / ptiles_per_rank, pj = (ti % pt_sel) % ptiles_per_rank;
     const int t = tm * pt_n + rank * ptiles_per_rank + pj;
     // ---- acquire the tile in slot s ----
     int failed = 0;
     if (threadIdx.x == 0) {
       const int32_t* flag = reinterpret_cast<const int32_t*>(tab.base[s] + flag_off) + t;
-      int32_t seen = ld_acquire_gpu(flag);
+      int32_t seen = ld_acquire_flag(flag, tab.flags_sys);
       if (seen < epoch) {
         const uint64_t start = globaltimer_ns();
         uint32_t spins = 0;
-        while ((seen = ld_acquire_gpu(flag)) < epoch) {
+        while ((seen = ld_acquire_flag(flag, tab.flags_sys)) < epoch) {
           __nanosleep(256);   // the tile is still being produced: leave the issue slots to whoever shares this SM
           if ((++spins & 31u) == 0 && globaltimer_ns() - start > timeout_ns) {
             report_timeout(status, KID_CONSUMER, t, s, seen, epoch);
@@ -103,15 +103,17 @@ extern "C" int iris_consume_bias_ranks(iris_heap* h, uint64_t c_off, uint64_t ou
   if (c_off > bpr || bytes > bpr - c_off || out_off > bpr || bytes > bpr - out_off || flag_off > bpr || nt * 4 > bpr - flag_off)
     return fail(IRIS_ERR_RANGE, "iris_consume_bias: a region leaves the slot");
   if (c_off < out_off + bytes && out_off < c_off + bytes) return fail(IRIS_ERR_ARG, "iris_consume_bias: C and OUT overlap");
-  const uint64_t items = (uint64_t)tiles_m * rank_count * ptr_ * world;
+  // every slot of a one-process heap (each emulated rank consumes its copy); this process's own slot otherwise
+  const int slot_first = h->local_rank >= 0 ? h->local_rank : 0, slot_count = h->local_rank >= 0 ? 1 : world;
+  const uint64_t items = (uint64_t)tiles_m * rank_count * ptr_ * slot_count;
   uint64_t grid = ctas > 0 ? (uint64_t)ctas : (uint64_t)h->sm_count * 8;
   if (grid > items) grid = items;
   const uint64_t to = timeout_ns ? timeout_ns : kDefaultTimeoutNs;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (dtype == IRIS_BF16)
-    consume_bias_kernel<true><<<(int)grid, kConsThreads, 0, st>>>(h->table(), c_off, out_off, flag_off, static_cast<const uint8_t*>(bias), M, N, nl, tiles_m, ptr_, rank_first, rank_count, epoch, to, h->status);
+    consume_bias_kernel<true><<<(int)grid, kConsThreads, 0, st>>>(h->table(), c_off, out_off, flag_off, static_cast<const uint8_t*>(bias), M, N, nl, tiles_m, ptr_, rank_first, rank_count, slot_first, slot_count, epoch, to, h->status);
   else
-    consume_bias_kernel<false><<<(int)grid, kConsThreads, 0, st>>>(h->table(), c_off, out_off, flag_off, static_cast<const uint8_t*>(bias), M, N, nl, tiles_m, ptr_, rank_first, rank_count, epoch, to, h->status);
+    consume_bias_kernel<false><<<(int)grid, kConsThreads, 0, st>>>(h->table(), c_off, out_off, flag_off, static_cast<const uint8_t*>(bias), M, N, nl, tiles_m, ptr_, rank_first, rank_count, slot_first, slot_count, epoch, to, h->status);
   IRIS_CUDA_TRY(cudaGetLastError());
   return IRIS_OK;
 }

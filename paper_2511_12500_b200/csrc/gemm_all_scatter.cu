@@ -312,7 +312,7 @@ __device__ void comm_cta(const GemmParams& p, CtrlBlock* ctrl, uint8_t* payload,
       // bar.warp.sync orders lane 0's wait for the bulk stores (and its proxy fence) before the other lanes' flag
       // releases: a vote converges the warp but is not a memory barrier
       __syncwarp();
-      if (lane < W) st_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[lane] + p.flag_off) + rt, p.epoch);
+      if (lane < W) st_release_flag(reinterpret_cast<int32_t*>(p.tab.base[lane] + p.flag_off) + rt, p.epoch, p.tab.flags_sys);
       if (p.takeover && lane == 0) atomicAdd(p.backlog, -1);
       __syncwarp();
     }
@@ -627,7 +627,7 @@ __global__ void __launch_bounds__(kGemmThreads, 1) gemm_all_scatter_kernel(const
             const int pj = tc.jn * subs + sub;
             if (pj < p.ptiles_per_rank) {
               const int t = tc.tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
-              st_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[s] + p.flag_off) + t, p.epoch);
+              st_release_flag(reinterpret_cast<int32_t*>(p.tab.base[s] + p.flag_off) + t, p.epoch, p.tab.flags_sys);
             }
           }
         } else if (et < subs) {
@@ -790,7 +790,8 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
       ptx::prefetch_tensormap(&p.tmA);
       for (int r = p.rank_first; r < p.rank_first + p.rank_count; ++r) ptx::prefetch_tensormap(&p.tmB[r]);
     }
-    ptx::prefetch_tensormap(is_comm ? &p.tmC4 : &p.tmC4s);
+    if (p.one_map) ptx::prefetch_tensormap(is_comm ? &p.tmC4 : &p.tmC4s);
+    else for (int r = 0; r < p.tab.world; ++r) ptx::prefetch_tensormap(is_comm ? &p.tmC[r] : &p.tmCs[r]);
   }
   if (warp == 1 && !is_comm) {
     ptx::tmem_alloc_pair(ptx::smem_u32(&ctrl->tmem_base), 2 * kPairBN);
@@ -1065,7 +1066,8 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
                     while (globaltimer_ns() < due) __nanosleep(64);
                     due += gap_ns;
                   }
-                  ptx::tma_store_4d(&p.tmC4s, col, tm * BM, tc.rank, s, stg + (uint32_t)(b * kStoreBoxBytes));
+                  if (p.one_map) ptx::tma_store_4d(&p.tmC4s, col, tm * BM, tc.rank, s, stg + (uint32_t)(b * kStoreBoxBytes));
+                  else ptx::tma_store_3d(&p.tmCs[s], col, tm * BM, tc.rank, stg + (uint32_t)(b * kStoreBoxBytes));
                 }
               }
             }
@@ -1092,7 +1094,7 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
               const int pj = tc.jn * subs + sub;
               if (pj < p.ptiles_per_rank) {   // a ragged shard's last tile may have only one publication tile
                 const int t = tm * pt_n + tc.rank * p.ptiles_per_rank + pj;
-                st_release_gpu(reinterpret_cast<int32_t*>(p.tab.base[s] + p.flag_off) + t, p.epoch);
+                st_release_flag(reinterpret_cast<int32_t*>(p.tab.base[s] + p.flag_off) + t, p.epoch, p.tab.flags_sys);
               }
             } else if (p.takeover && tile < p.seq_from && et >= 64 && et < 64 + subs) {
               // a tile the communication warps are watching: tell its warp that only the lock is left to reset
@@ -1187,7 +1189,7 @@ __global__ void __launch_bounds__(256) all_scatter_kernel(const __grid_constant_
       }
     }
     __syncthreads();
-    if ((int)threadIdx.x < W) st_release_gpu(reinterpret_cast<int32_t*>(tab.base[threadIdx.x] + flag_off) + t, epoch);
+    if ((int)threadIdx.x < W) st_release_flag(reinterpret_cast<int32_t*>(tab.base[threadIdx.x] + flag_off) + t, epoch, tab.flags_sys);
   }
 }
 
@@ -1346,10 +1348,11 @@ static int auto_comm_ctas_pair(int total_ctiles, int kblocks, double remote_byte
 // the handle) or raw addresses (base == NULL: one tensor map per slot, single-CTA kernel only).
 struct PlanEnv {
   HeapTable tab;
-  char* base;
+  char* base;          // slots bytes_per_rank apart from here, or nullptr: slots wherever tab.base says
   uint64_t bpr;
   int sm_count;
   int32_t* status;
+  bool pair_any_base;  // with base == nullptr: the CTA-pair kernel may still be chosen (it then stores through per-slot maps)
 };
 struct Plan { GemmParams p; int bn, grid; bool pair, streamk; };
 
@@ -1365,7 +1368,7 @@ static int default_block_n(int M, int nl, int W, int sm_count) {
 }
 
 struct PlanKey {
-  const void* heap; const void* base; const void* status; uint64_t bytes_per_rank;
+  const void* heap; const void* slot[IRIS_MAX_WORLD]; const void* status; uint64_t bytes_per_rank; int flags_sys;
   const void* A; const void* B[IRIS_MAX_WORLD];
   int M, N, K, world, mode, dtype;
   uint64_t c_off, flag_off, lock_off;
@@ -1383,7 +1386,8 @@ static int g_plan_next = 0;
 
 static void make_key(PlanKey* k, const iris_gemm_args* a, const iris_heap* h) {
   std::memset(k, 0, sizeof(*k));   // padding too: keys are compared with memcmp
-  k->heap = h; k->base = h->base; k->status = h->status; k->bytes_per_rank = h->bytes_per_rank;
+  k->heap = h; k->status = h->status; k->bytes_per_rank = h->bytes_per_rank; k->flags_sys = h->flags_sys;
+  for (int r = 0; r < h->world && r < IRIS_MAX_WORLD; ++r) k->slot[r] = h->slot_base[r];
   k->A = a->A;
   const int r_end = a->rank_count ? a->rank_first + a->rank_count : a->world;
   for (int r = a->rank_first; r < r_end && r < IRIS_MAX_WORLD; ++r) k->B[r] = a->B_shards ? a->B_shards[r] : nullptr;
@@ -1419,7 +1423,7 @@ static int build_plan(const iris_gemm_args* a, const PlanEnv& env, Plan& out) {
   // CTA pairs (256 x 256 tiles) need at least two tile rows.  A shard that is not a whole number of 256-column
   // tiles is fine: TMA zero-fills the missing B rows, stores and flags are masked, and the last tile's MMA is only
   // as wide as what is left of the shard (rounded up to 32 columns), so the padding costs next to nothing.
-  const bool pair_ok = a->M > BM && nl > BM && a->block_n != 128 && env.sm_count >= 4 && env.base != nullptr;
+  const bool pair_ok = a->M > BM && nl > BM && a->block_n != 128 && env.sm_count >= 4 && (env.base != nullptr || env.pair_any_base);
   if (a->cta_pair > 0 && !pair_ok) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: cta_pair needs M > 128, N/world > 128 and block_n != 128");
   pair = pair_ok && a->cta_pair >= 0;
   int max_pairs = 0;
@@ -1674,6 +1678,10 @@ static int enqueue_gemm_all_scatter(const iris_gemm_args* a, void* stream, bool 
   if (a->rank_first < 0 || a->rank_count < 0 || a->rank_first + a->rank_count > W || (a->rank_count == 0 && a->rank_first != 0))
     return fail(IRIS_ERR_ARG, "gemm_all_scatter: rank range [%d, %d) outside [0, %d)", a->rank_first, a->rank_first + a->rank_count, W);
   const int rank_first = a->rank_first, rank_count = a->rank_count ? a->rank_count : W;   // 0, 0 = every rank
+  // A heap over several processes: the locks of a shard live in its owner's slot and are handled with gpu-scope atomics,
+  // and only the owner holds that shard of B, so a process computes its own rank's shard and nothing else.
+  if (h->local_rank >= 0 && (rank_first != h->local_rank || rank_count != 1))
+    return fail(IRIS_ERR_ARG, "gemm_all_scatter: on a heap over several processes rank_first must be the local rank (%d) and rank_count 1", h->local_rank);
   const int64_t nt = num_tiles(a->M, a->N, W);
   const uint64_t bpr = h->bytes_per_rank;
   const uint64_t c_bytes = (uint64_t)a->M * a->N * 2;
@@ -1685,6 +1693,8 @@ static int enqueue_gemm_all_scatter(const iris_gemm_args* a, void* stream, bool 
   if (overlaps(a->c_off, c_bytes, a->flag_off, (uint64_t)nt * 4) || (wg && (overlaps(a->c_off, c_bytes, a->lock_off, (uint64_t)nt * 4) || overlaps(a->flag_off, (uint64_t)nt * 4, a->lock_off, (uint64_t)nt * 4))))
     return fail(IRIS_ERR_ARG, "gemm_all_scatter: C, flag and lock regions overlap");
   const bool fused_consumer = a->consumer_bias != nullptr;
+  if (fused_consumer && h->local_rank >= 0)
+    return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: consumer_bias consumes every slot; on a heap over several processes call iris_consume_bias, which reads the local slot");
   if (unfused) {
     if (!wg) return fail(IRIS_ERR_ARG, "gemm_all_scatter_unfused: the two-kernel form is the workgroup_specialized schedule (mode %d given)", a->mode);
     // consumer warps inside the producer kernel would wait for flags that the second kernel publishes, while that one
@@ -1723,7 +1733,7 @@ static int enqueue_gemm_all_scatter(const iris_gemm_args* a, void* stream, bool 
     }
   }
   auto build = [&]() -> int {
-    PlanEnv env{h->table(), h->base, h->bytes_per_rank, h->sm_count, h->status};
+    PlanEnv env{h->table(), h->base, h->bytes_per_rank, h->sm_count, h->status, true};
     Plan pl;
     const int rc = build_plan(a, env, pl);
     p = pl.p; bn = pl.bn; grid = pl.grid; pair = pl.pair; streamk = pl.streamk;
@@ -1833,7 +1843,7 @@ static int short_form_init(iris_heap* heap, int M, int N, int world, cudaStream_
   if (nt > 0) {
     if (flag_off > heap->bytes_per_rank || bytes > heap->bytes_per_rank - flag_off) return fail(IRIS_ERR_RANGE, "gemm_all_scatter: flags and locks leave the slot");
     for (int s = 0; s < world; ++s)
-      IRIS_CUDA_TRY(cudaMemsetAsync(heap->base + (size_t)s * heap->bytes_per_rank + flag_off, 0, bytes, st));
+      IRIS_CUDA_TRY(cudaMemsetAsync(heap->slot_base[s] + flag_off, 0, bytes, st));
   }
   heap->sf_M = M; heap->sf_N = N;
   return IRIS_OK;
@@ -1842,6 +1852,7 @@ static int short_form_init(iris_heap* heap, int M, int N, int world, cudaStream_
 static int short_form(const void* A, const void* const* B_shards, iris_heap* heap, int M, int N, int K, int world, int mode, int dtype, void* stream,
                       const void* bias = nullptr, uint64_t out_off = 0) {
   if (!heap_ok(heap)) return fail(IRIS_ERR_STATE, "gemm_all_scatter: bad heap handle");
+  if (heap->local_rank >= 0) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter: the short form computes every rank's shard; on a heap over several processes call iris_gemm_all_scatter_ex with rank_first = the local rank");
   if (num_tiles(M, N, world) < 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter: bad M/N/world");
   iris_gemm_args a;
   std::memset(&a, 0, sizeof(a));
@@ -1883,6 +1894,7 @@ uint64_t iris_gemm_out_offset(int M, int N, int world) {
 int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_host, void* C_host, int32_t* flags_host, const void* bias_host,
                                void* OUT_host, iris_heap* heap, int M, int N, int K, int world, int mode, int dtype, int out_slot) {
   if (!heap_ok(heap)) return fail(IRIS_ERR_STATE, "gemm_all_scatter_host: bad heap handle");
+  if (heap->local_rank >= 0) return fail(IRIS_ERR_UNSUPPORTED, "gemm_all_scatter_host: not available on a heap over several processes");
   if (world != heap->world || out_slot < 0 || out_slot >= world) return fail(IRIS_ERR_ARG, "gemm_all_scatter_host: bad world or out_slot");
   const int64_t nt = num_tiles(M, N, world);
   if (nt < 0 || K < 0) return fail(IRIS_ERR_ARG, "gemm_all_scatter_host: bad M/N/K/world");
@@ -1952,7 +1964,7 @@ int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_h
   IRIS_CUDA_TRY(cudaEventRecord(hp->b_ready, s_in));
   IRIS_CUDA_TRY(cudaStreamWaitEvent(s_run, hp->b_ready, 0));
 
-  char* slot = heap->base + (size_t)out_slot * heap->bytes_per_rank;
+  char* slot = heap->slot_base[out_slot];
   if (int irc = short_form_init(heap, M, N, world, s_run)) return irc;
   const int32_t epoch = heap->epoch + 1;
   for (int blk = 0; blk < blocks; ++blk) {
@@ -1997,7 +2009,7 @@ int iris_gemm_all_scatter_host(const void* A_host, const void* const* B_shards_h
   heap->epoch = epoch;
   if (flags_host && nt > 0)
     for (int s = 0; s < world; ++s)
-      IRIS_CUDA_TRY(cudaMemcpyAsync(flags_host + (size_t)s * nt, heap->base + (size_t)s * heap->bytes_per_rank + flag_off, (size_t)nt * 4, cudaMemcpyDeviceToHost, s_out));
+      IRIS_CUDA_TRY(cudaMemcpyAsync(flags_host + (size_t)s * nt, heap->slot_base[s] + flag_off, (size_t)nt * 4, cudaMemcpyDeviceToHost, s_out));
   IRIS_CUDA_TRY(cudaStreamSynchronize(s_out));
   IRIS_CUDA_TRY(cudaStreamSynchronize(s_in));
   return iris_status_check(heap, s_run, nullptr);

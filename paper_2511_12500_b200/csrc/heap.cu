@@ -81,6 +81,8 @@ int iris_heap_create_ex(int world, size_t bytes_per_rank, void* external_base, i
       return fail(IRIS_ERR_CUDA, "iris_heap_create: cudaMemset: %s", cudaGetErrorString(e));
     }
   }
+  for (int r = 0; r < world; ++r) h->slot_base[r] = h->base + (size_t)r * bytes_per_rank;
+  h->local_rank = -1;
   h->sf_M = h->sf_N = -1;
   cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&h->status), 256);
   if (e == cudaSuccess) e = cudaMemset(h->status, 0, 256);
@@ -92,6 +94,112 @@ int iris_heap_create_ex(int world, size_t bytes_per_rank, void* external_base, i
   }
   h->magic = kHeapMagic;
   *out = h;
+  return IRIS_OK;
+}
+
+int iris_heap_create_from_bases(int world, size_t bytes_per_rank, const uint64_t* bases, int local_rank, iris_heap** out) {
+  if (!out) return fail(IRIS_ERR_ARG, "iris_heap_create_from_bases: out is NULL");
+  *out = nullptr;
+  if (!bases) return fail(IRIS_ERR_ARG, "iris_heap_create_from_bases: bases is NULL");
+  if (world < 1 || world > IRIS_MAX_WORLD) return fail(IRIS_ERR_ARG, "iris_heap_create_from_bases: world=%d not in [1,%d]", world, IRIS_MAX_WORLD);
+  if (local_rank < 0 || local_rank >= world) return fail(IRIS_ERR_ARG, "iris_heap_create_from_bases: local_rank=%d not in [0,%d)", local_rank, world);
+  if (bytes_per_rank == 0 || bytes_per_rank % 256 != 0)
+    return fail(IRIS_ERR_ARG, "iris_heap_create_from_bases: bytes_per_rank=%zu must be a positive multiple of 256", bytes_per_rank);
+  for (int r = 0; r < world; ++r) {
+    if (bases[r] == 0 || bases[r] % 256 != 0) return fail(IRIS_ERR_ARG, "iris_heap_create_from_bases: base of slot %d must be a 256-byte aligned device address", r);
+    for (int q = 0; q < r; ++q) {
+      const uint64_t lo = bases[q] < bases[r] ? bases[q] : bases[r], hi = bases[q] < bases[r] ? bases[r] : bases[q];
+      if (hi - lo < bytes_per_rank) return fail(IRIS_ERR_ARG, "iris_heap_create_from_bases: slots %d and %d overlap", q, r);
+    }
+  }
+  int dev = 0;
+  IRIS_CUDA_TRY(cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  IRIS_CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
+  if (prop.major != 10) return fail(IRIS_ERR_UNSUPPORTED, "iris_heap_create_from_bases: device is sm_%d%d, this library is sm_100a only", prop.major, prop.minor);
+  iris_heap* h = new iris_heap();
+  std::memset(h, 0, sizeof(*h));
+  h->world = world;
+  h->device = dev;
+  h->bytes_per_rank = bytes_per_rank;
+  h->sm_count = prop.multiProcessorCount;
+  h->base = nullptr;
+  h->owns = false;
+  for (int r = 0; r < world; ++r) h->slot_base[r] = reinterpret_cast<char*>(bases[r]);
+  h->local_rank = local_rank;
+  h->flags_sys = 1;
+  h->sf_M = h->sf_N = -1;
+  cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&h->status), 256);
+  if (e == cudaSuccess) e = cudaMemset(h->status, 0, 256);
+  if (e != cudaSuccess) {
+    delete h;
+    cudaGetLastError();
+    return fail(IRIS_ERR_NOMEM, "iris_heap_create_from_bases: status block: %s", cudaGetErrorString(e));
+  }
+  h->magic = kHeapMagic;
+  *out = h;
+  return IRIS_OK;
+}
+
+int iris_heap_local_rank(const iris_heap* h) { return heap_ok(h) ? h->local_rank : fail(IRIS_ERR_STATE, "bad heap handle"); }
+
+// ---- one rank's slot as memory other processes can map (Section 3.2, steps 3-5: allocate, exchange handles, open) ----
+int iris_ipc_alloc(size_t bytes, void** ptr_out) {
+  if (!ptr_out) return fail(IRIS_ERR_ARG, "iris_ipc_alloc: ptr_out is NULL");
+  *ptr_out = nullptr;
+  if (bytes == 0) return fail(IRIS_ERR_ARG, "iris_ipc_alloc: bytes must be positive");
+  void* p = nullptr;
+  cudaError_t e = cudaMalloc(&p, bytes);
+  if (e != cudaSuccess) {
+    cudaGetLastError();
+    return fail(IRIS_ERR_NOMEM, "iris_ipc_alloc: cudaMalloc(%zu) failed: %s", bytes, cudaGetErrorString(e));
+  }
+  e = cudaMemset(p, 0, bytes);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  if (e != cudaSuccess) {
+    cudaFree(p);
+    cudaGetLastError();
+    return fail(IRIS_ERR_CUDA, "iris_ipc_alloc: cudaMemset: %s", cudaGetErrorString(e));
+  }
+  *ptr_out = p;
+  return IRIS_OK;
+}
+
+int iris_ipc_free(void* ptr) {
+  if (!ptr) return IRIS_OK;
+  IRIS_CUDA_TRY(cudaDeviceSynchronize());
+  IRIS_CUDA_TRY(cudaFree(ptr));
+  return IRIS_OK;
+}
+
+int iris_ipc_export(void* ptr, unsigned char* handle_out) {
+  static_assert(sizeof(cudaIpcMemHandle_t) == IRIS_IPC_HANDLE_BYTES, "handle size");
+  if (!ptr || !handle_out) return fail(IRIS_ERR_ARG, "iris_ipc_export: NULL argument");
+  cudaIpcMemHandle_t hd;
+  IRIS_CUDA_TRY(cudaIpcGetMemHandle(&hd, ptr));
+  std::memcpy(handle_out, &hd, sizeof(hd));
+  return IRIS_OK;
+}
+
+int iris_ipc_open(const unsigned char* handle, void** ptr_out) {
+  if (!handle || !ptr_out) return fail(IRIS_ERR_ARG, "iris_ipc_open: NULL argument");
+  *ptr_out = nullptr;
+  cudaIpcMemHandle_t hd;
+  std::memcpy(&hd, handle, sizeof(hd));
+  void* p = nullptr;
+  const cudaError_t e = cudaIpcOpenMemHandle(&p, hd, cudaIpcMemLazyEnablePeerAccess);
+  if (e != cudaSuccess) {
+    cudaGetLastError();   // a refused handle must not show up as the next launch's error
+    return fail(IRIS_ERR_CUDA, "iris_ipc_open: %s", cudaGetErrorString(e));
+  }
+  *ptr_out = p;
+  return IRIS_OK;
+}
+
+int iris_ipc_close(void* ptr) {
+  if (!ptr) return IRIS_OK;
+  IRIS_CUDA_TRY(cudaDeviceSynchronize());
+  IRIS_CUDA_TRY(cudaIpcCloseMemHandle(ptr));
   return IRIS_OK;
 }
 
@@ -126,12 +234,12 @@ void* iris_heap_base(const iris_heap* h, int rank) {
     set_error("iris_heap_base: bad handle or rank");
     return nullptr;
   }
-  return h->base + (size_t)rank * h->bytes_per_rank;
+  return h->slot_base[rank];
 }
 
 int iris_heap_bases(const iris_heap* h, uint64_t* out) {
   if (!heap_ok(h) || !out) return fail(IRIS_ERR_ARG, "iris_heap_bases: bad handle or NULL out");
-  for (int r = 0; r < h->world; ++r) out[r] = (uint64_t)(h->base + (size_t)r * h->bytes_per_rank);
+  for (int r = 0; r < h->world; ++r) out[r] = (uint64_t)h->slot_base[r];
   return IRIS_OK;
 }
 
@@ -157,8 +265,8 @@ int iris_translate(const iris_heap* h, const void* ptr, int from_rank, int to_ra
   if (!heap_ok(h) || !out) return fail(IRIS_ERR_ARG, "iris_translate: bad handle or NULL out");
   if (from_rank < 0 || from_rank >= h->world || to_rank < 0 || to_rank >= h->world)
     return fail(IRIS_ERR_ARG, "iris_translate: rank out of range (from=%d to=%d world=%d)", from_rank, to_rank, h->world);
-  const uint64_t from_base = (uint64_t)(h->base + (size_t)from_rank * h->bytes_per_rank);
-  const uint64_t to_base = (uint64_t)(h->base + (size_t)to_rank * h->bytes_per_rank);
+  const uint64_t from_base = (uint64_t)h->slot_base[from_rank];
+  const uint64_t to_base = (uint64_t)h->slot_base[to_rank];
   const uint64_t p = (uint64_t)ptr;
   if (p < from_base || p - from_base >= h->bytes_per_rank)
     return fail(IRIS_ERR_RANGE, "iris_translate: pointer is outside rank %d's heap", from_rank);

@@ -37,6 +37,18 @@ __device__ __forceinline__ int32_t ld_relaxed_gpu(const int32_t* p) {
 __device__ __forceinline__ void st_release_gpu(int32_t* p, int32_t v) {
   asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
+// Ready flags: gpu scope while every slot lives on this device, system scope when the heap spans processes or
+// devices (the writer's release has to reach a reader on another GPU, and the reader's acquire has to see it).
+__device__ __forceinline__ void st_release_flag(int32_t* p, int32_t v, int sys) {
+  if (sys) asm volatile("st.release.sys.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+  else st_release_gpu(p, v);
+}
+__device__ __forceinline__ int32_t ld_acquire_flag(const int32_t* p, int sys) {
+  if (!sys) return ld_acquire_gpu(p);
+  int32_t v;
+  asm volatile("ld.acquire.sys.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ void fence_acq_rel_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
 // Orders generic-proxy accesses against async-proxy (TMA / bulk copy) accesses.
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }

@@ -24,6 +24,7 @@ struct HeapTable {
   uint64_t base[IRIS_MAX_WORLD];
   uint64_t bytes_per_rank;
   int world;
+  int flags_sys;   // 1 = slots may live on other devices or in other processes: ready flags are released and acquired at system scope
 };
 
 void set_error(const char* fmt, ...);
@@ -44,7 +45,10 @@ struct iris_heap {
   int world;
   int device;
   size_t bytes_per_rank;
-  char* base;          // device
+  char* base;          // device; nullptr when the slots are not one contiguous range (iris_heap_create_from_bases)
+  char* slot_base[IRIS_MAX_WORLD];   // slot r starts here (base + r * bytes_per_rank for a contiguous heap)
+  int local_rank;      // heap over several processes / devices: the slot that lives in this process's own memory; -1 otherwise
+  int flags_sys;       // see HeapTable
   bool owns;
   uint64_t bump;       // next free offset
   int32_t* status;     // device, kStatusWords int32
@@ -65,9 +69,10 @@ struct iris_heap {
   void* ev_join;
   iris::HeapTable table() const {
     iris::HeapTable t{};
-    for (int r = 0; r < world; ++r) t.base[r] = (uint64_t)(base + (size_t)r * bytes_per_rank);
+    for (int r = 0; r < world; ++r) t.base[r] = (uint64_t)slot_base[r];
     t.bytes_per_rank = bytes_per_rank;
     t.world = world;
+    t.flags_sys = flags_sys;
     return t;
   }
 };

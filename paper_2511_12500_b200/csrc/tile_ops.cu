@@ -201,7 +201,7 @@ __global__ void __launch_bounds__(kAllStoreThreads) all_store_kernel(const __gri
 }
 
 static int check_region(const iris_heap* h, const void* p, int rank, size_t rows, size_t row_bytes, size_t pitch, const char* what) {
-  const uint64_t base = (uint64_t)(h->base + (size_t)rank * h->bytes_per_rank);
+  const uint64_t base = (uint64_t)h->slot_base[rank];
   const uint64_t a = (uint64_t)p;
   if (a < base || a - base >= h->bytes_per_rank) return fail(IRIS_ERR_RANGE, "%s: address is outside rank %d's heap", what, rank);
   // span = (rows - 1) * pitch + row_bytes must fit in what is left of the slot; compared by division so that huge
@@ -364,6 +364,7 @@ int iris_atomic_cas_contended(iris_heap* h, void* ptr, size_t threads, int from_
 int iris_all_store_bench(iris_heap* h, uint64_t payload_off, uint64_t recv_off, uint64_t flag_off, size_t S, size_t tile_bytes, int32_t epoch,
                          int ctas, int pull, void* stream) {
   if (!heap_ok(h)) return fail(IRIS_ERR_STATE, "iris_all_store_bench: bad heap handle");
+  if (h->local_rank >= 0) return fail(IRIS_ERR_UNSUPPORTED, "iris_all_store_bench: emulates every rank in one process; not available on a heap over several processes");
   if (S == 0) return IRIS_OK;
   if (S % 16 != 0 || tile_bytes == 0 || tile_bytes % 16 != 0 || tile_bytes > 32768) return fail(IRIS_ERR_ARG, "iris_all_store_bench: S and tile_bytes must be multiples of 16, tile_bytes <= 32768");
   if (payload_off % 16 != 0 || recv_off % 16 != 0 || flag_off % 4 != 0) return fail(IRIS_ERR_ARG, "iris_all_store_bench: misaligned offsets");
