@@ -32,6 +32,7 @@ CASES = [
     (WG, "bf16", 1000, 512, 200, {"wg_tail": -1}),             # CTA-pair tiles, communication CTAs copy to the peer's slot
     (WG, "fp16", 768, 256, 256, {}),                           # default tail rule: producers scatter the last wave themselves
     (BSP, "fp16", 512, 384, 64, {}),
+    (WG, "bf16", 640, 256, 192, {"wg_tail": -1, "two_streams": True}),   # the unfused form: communication kernel on a second stream
 ]
 
 
@@ -68,6 +69,10 @@ def main():
                     assert e.code == iris.IRIS_ERR_ARG, e
                 else:
                     raise AssertionError(f"accepted {bad}")
+            kw = dict(kw)
+            if kw.pop("two_streams", False):
+                kw["comm_stream"] = torch.cuda.Stream()
+                kw["stream"] = torch.cuda.current_stream()
             iris.iris_gemm_all_scatter_ex(heap.handle, dA, shards, M, N, K, W, mode, iris.DTYPES[dtype], c_off, flag_off, lock_off, epoch,
                                           rank_first=rank, rank_count=1, **kw)
             iris.iris_status_check(heap.handle)                 # synchronises: this rank's tiles and flags are in every slot
