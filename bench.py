@@ -216,6 +216,16 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def gpu_gate(torch):
+    """Keep the GPU busy for ~0.2 ms before a single launch is timed between two synchronisations.
+
+    A start event recorded on an idle GPU is stamped at once, so everything the host still does before the kernel is
+    queued (argument marshalling, plan lookup, the launch call itself: 20-25 us, for the library GEMM as for this
+    path) would be counted as kernel time -- a fifth of a 0.1 ms kernel.  With the GPU busy the host runs ahead and the
+    interval between the two events is device time only."""
+    torch.cuda._sleep(400_000)
+
+
 def max_over_ranks(value: float, device=None) -> float:
     """Max of a per-rank scalar over the process group (the job's time is its slowest rank's)."""
     import torch
@@ -318,6 +328,7 @@ def run_ours(args):
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     barrier()
     sampler.mark()
+    gpu_gate(torch)
     for i in range(args.steps):
         epoch += 1
         step(epoch, ev[i])
@@ -391,6 +402,7 @@ def run_ours(args):
             ts = []
             for _ in range(4):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                gpu_gate(torch)
                 e0.record(stream)
                 consume(epoch)
                 e1.record(stream)
@@ -416,6 +428,7 @@ def run_ours(args):
             for name, m in variants:
                 epoch += 1
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                gpu_gate(torch)
                 e0.record(stream)
                 if m is None:
                     tC = tA @ tB.t()
@@ -459,7 +472,12 @@ def run_ours(args):
                     epoch += 1
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     torch.cuda.synchronize()
+                    gpu_gate(torch)
                     e0.record(stream)
+                    if overlapped:
+                        # the consumer must not become resident before the producer does (it would hold the SMs' registers
+                        # while it waits for flags): its stream starts behind the same busy kernel as the producer's
+                        cons_stream.wait_event(e0)
                     gemm(epoch)
                     if overlapped:
                         # 4 CTAs per SM: half the thread slots stay free for whatever the producer side still has to launch
@@ -611,6 +629,7 @@ def all_store_sweep(iris, pk, kind, pull=0):
         iris.iris_all_store_bench(h, payload_off, recv_off, flag_off, S, tile, 2, 0, pull)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
+        gpu_gate(torch)
         e0.record(stream)
         for i in range(iters):
             iris.iris_all_store_bench(h, payload_off, recv_off, flag_off, S, tile, 3 + i, 0, pull)
@@ -654,6 +673,7 @@ def p2p_microbench(iris, pk):
         fn(); fn()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
+        gpu_gate(torch)
         e0.record(stream)
         for _ in range(iters):
             fn()
