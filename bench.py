@@ -480,8 +480,8 @@ def run_ours(args):
                         cons_stream.wait_event(e0)
                     gemm(epoch)
                     if overlapped:
-                        # 4 CTAs per SM: half the thread slots stay free for whatever the producer side still has to launch
-                        iris.iris_consume_bias(h, 0, out_off, flag_off, dbias, M, N, W, dt, epoch, ctas=4 * sm_count, stream=cons_stream)
+                        # 3 CTAs per SM: a GEMM CTA still fits beside them (threads, registers) should the consumer become resident first
+                        iris.iris_consume_bias(h, 0, out_off, flag_off, dbias, M, N, W, dt, epoch, ctas=3 * sm_count, stream=cons_stream)
                         joined.record(cons_stream)
                         stream.wait_event(joined)
                     else:

@@ -376,11 +376,13 @@ int64_t iris_num_tiles(int M, int N, int world);
  * of `dtype`, broadcast over rows; the sum is formed in fp32 and rounded once.  OUT is a second
  * row-major [M, N] region at out_off in every slot.  ctas: grid size (0 = 8 per SM).
  * On a stream of its own the consumer may be launched while its producer is still running (that is the point of
- * the flags).  Launch it after every kernel that publishes the flags it waits for has been launched, and when one
- * of those kernels can only start later (the second kernel of bulk_synchronous mode starts when the GEMM ends)
- * pass ctas <= 4 per SM: the default grid fills every SM's thread slots, its CTAs leave only once their tiles are
- * published, and a publisher that finds no room would never run -- the wait would end by its deadline
- * (IRIS_ERR_TIMEOUT), not by making progress. */
+ * the flags).  Launch it after every kernel that publishes the flags it waits for has been launched.  Its CTAs leave
+ * only once their tiles are published, so a publisher that finds no room on the SMs they occupy would never run and
+ * the wait would end by its deadline (IRIS_ERR_TIMEOUT), not by making progress: the default grid fills every SM's
+ * thread slots, and four CTAs per SM still hold too many registers for a GEMM CTA of this library to fit beside
+ * them.  Whenever a publishing kernel may become resident after the consumer (the second kernel of bulk_synchronous
+ * mode starts when the GEMM ends; two streams released by the same event start in no fixed order) pass
+ * ctas <= 3 per SM: that leaves threads, registers and all shared memory for one CTA of any kernel here. */
 int iris_consume_bias(iris_heap* heap, uint64_t c_off, uint64_t out_off, uint64_t flag_off, const void* bias, int M,
                       int N, int world, int dtype, int32_t epoch, int ctas, uint64_t timeout_ns, void* stream);
 /* The same for the publication tiles of ranks [rank_first, rank_first + rank_count) only (the column
