@@ -328,12 +328,14 @@ typedef struct iris_gemm_args {
                                   a tile of its own; 0 = the library chooses (fused, except in
                                   workgroup_specialized mode with fewer than three waves of work).
                                   Same results either way                                          */
-  int stage_k;                 /* CTA-pair kernel: K extent of one operand stage in shared memory.  128 (and 0, the
-                                  default) = two 64-wide k-blocks per stage, their TMA boxes requested back to
-                                  back (3 stages of 64 KB): adjacent 128-byte pieces of the same operand rows in
-                                  flight together is what lets one SM's loads keep up with its tensor core;
-                                  64 = one k-block per stage (6 stages of 32 KB).  A stage that also carries a
-                                  fused remainder (fuse_tail) always holds one k-block.  Same results     */
+  int stage_k;                 /* CTA-pair kernel: K extent of one operand stage in shared memory.  128 = two 64-wide
+                                  k-blocks per stage, their TMA boxes requested back to back (3 stages of 64 KB):
+                                  adjacent 128-byte pieces of the same operand rows in flight together is what lets
+                                  one SM's loads keep up with its tensor core; 64 = one k-block per stage (6 stages
+                                  of 32 KB).  0 = the library chooses: 128, except that stages which also carry a
+                                  fused remainder (fuse_tail) of more than 96 columns hold one k-block (two such
+                                  stages would be all that fits).  With a remainder of up to 96 columns the ring is
+                                  two two-k-block stages and one one-k-block stage.  Same results              */
 } iris_gemm_args;
 
 /* Enqueue the whole operation on `stream` (bulk-synchronous: two kernels; otherwise one).

@@ -109,6 +109,8 @@ struct alignas(64) GemmParams {
   int stage_bytes;      // pair kernel: bytes of one operand stage (32 KB per k-block, plus the remainder's B rows with fuse_last) ...
   int n_stages;         // ... and how many of them the 192 KB ring holds (3 to 6)
   int b1_bytes;         // fuse_last: bytes of the remainder's B box per CTA
+  int sub_bytes;        // pair kernel: bytes of one k-block's operands inside a stage (32 KB, plus the remainder's B rows with fuse_last)
+  int half_stage;       // pair kernel, two k-blocks per stage: 1 = the last stage of the ring has room for one k-block only
   int b_mn;             // 1 = B_r is [K, N_local] row-major (N contiguous): 64 x 64 boxes, MN-major descriptor; 0 = [N_local, K]
   int pace_stores;      // pair kernel: 1 = the epilogue spreads a tile's box stores over most of the next tile's main loop
   int raster_group;
@@ -740,8 +742,9 @@ __device__ void consumer_warp(const GemmParams& p, CtrlBlock* ctrl, int cwarp, i
 // it does not (the single-CTA kernel's tensor pipe is 67 % busy, this one's 92 %).
 // Accumulators: 2 x 256 columns of TMEM in each CTA (rows of its own half).  Shared memory: a 192 KB ring of operand
 // stages -- 3 stages of 64 KB holding two 64-wide k-blocks each (sub-stages [A 16 KB | B 16 KB]), whose boxes are
-// requested back to back; or one k-block per stage when asked for or when the stage also carries a fused remainder's
-// B rows -- and two 16 KB store boxes (128 converted columns of the CTA's half tile, 128B-swizzled for the TMA stores).
+// requested back to back; with a fused remainder's B rows in every sub-stage, two such stages and a last one of a
+// single k-block (or one k-block per stage when asked for or when five k-blocks would not fit) -- and two 16 KB
+// store boxes (128 converted columns of the CTA's half tile, 128B-swizzled for the TMA stores).
 //   full[s]        leader only; the leader's producer expects 64 KB, all four loads (two per CTA) complete on it
 //   empty[s]       both CTAs; the leader's tcgen05.commit multicasts the arrival to the pair
 //   tmem_full[a]   both CTAs; multicast commit after a tile's last MMA
@@ -855,33 +858,39 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         const int ncols1 = fused ? pair_tile_cols(p, tc.jn + 1) : 0;
         bool ok = true;
         constexpr int kbs = KBS;   // 64-wide k-blocks per stage (= p.kb_per_stage)
-        for (int kb = 0; kb < p.kblocks; kb += kbs) {
-          const int nk = min(kbs, p.kblocks - kb);   // k-blocks in this stage (the last stage of an odd count holds one)
+        for (int kb = 0, nk; kb < p.kblocks; kb += nk) {
+          // k-blocks in this stage: kbs, one in the ring's short last stage, one at the end of an odd count
+          nk = min((kbs == 2 && p.half_stage && stage == p.n_stages - 1) ? 1 : kbs, p.kblocks - kb);
           if (!mbar_wait(ptx::smem_u32(&ctrl->empty[stage]), phase ^ 1, p, ctrl, tile)) { ok = false; break; }
           const uint32_t full_local = ptx::smem_u32(&ctrl->full[stage]);
-          if (leader) ptx::mbar_arrive_expect_tx(full_local, 2 * (nk * kPairStageBytes + (fused ? p.b1_bytes : 0)));
+          if (leader) ptx::mbar_arrive_expect_tx(full_local, 2 * nk * (kPairStageBytes + (fused ? p.b1_bytes : 0)));
           const uint32_t full_leader = ptx::mapa(full_local, 0);
           const uint32_t sa = ptx::smem_u32(payload + stage * p.stage_bytes);
-          // A stage is nk sub-stages [A 16 KB | B 16 KB].  The boxes of adjacent k-blocks (the next 128 bytes of the same rows)
-          // are requested back to back: measured with a load-only probe on L2-resident data, one SM sustains 46-55 B/clk with
-          // one k-block per stage and 76-88 B/clk with two, and this main loop needs 64.
+          const uint32_t sub = (uint32_t)p.sub_bytes;
+          // A stage is nk sub-stages [A 16 KB | B 16 KB | (fused unit) the remainder's B rows].  The boxes of adjacent k-blocks
+          // (the next 128 bytes of the same rows) are requested back to back: measured with a load-only probe on L2-resident
+          // data, one SM sustains 46-55 B/clk with one k-block per stage and 76-88 B/clk with two, and this main loop needs 64.
 #pragma unroll
           for (int j = 0; j < kbs; ++j)
-            if (j < nk) ptx::tma_load_2d_pair(sa + j * kPairStageBytes, &p.tmA, (kb + j) * BK, tc.tm * 2 * BM + cta_rank * BM, full_leader);
+            if (j < nk) ptx::tma_load_2d_pair(sa + j * sub, &p.tmA, (kb + j) * BK, tc.tm * 2 * BM + cta_rank * BM, full_leader);
           if (p.b_mn) {   // this CTA's half of the tile's columns as two [64 k][64 n] blocks per k-block
             const int n0 = tc.jn * kPairBN + cta_rank * (ncols / 2);
 #pragma unroll
             for (int j = 0; j < kbs; ++j)
               if (j < nk) {
-                ptx::tma_load_2d_pair(sa + j * kPairStageBytes + BM * BK * 2, &p.tmB[tc.rank], n0, (kb + j) * BK, full_leader);
-                ptx::tma_load_2d_pair(sa + j * kPairStageBytes + BM * BK * 2 + kMnBlockBytes, &p.tmB[tc.rank], n0 + 64, (kb + j) * BK, full_leader);
+                ptx::tma_load_2d_pair(sa + j * sub + BM * BK * 2, &p.tmB[tc.rank], n0, (kb + j) * BK, full_leader);
+                ptx::tma_load_2d_pair(sa + j * sub + BM * BK * 2 + kMnBlockBytes, &p.tmB[tc.rank], n0 + 64, (kb + j) * BK, full_leader);
               }
           } else {
 #pragma unroll
             for (int j = 0; j < kbs; ++j)
-              if (j < nk) ptx::tma_load_2d_pair(sa + j * kPairStageBytes + BM * BK * 2, &p.tmB[tc.rank], (kb + j) * BK, tc.jn * kPairBN + cta_rank * (ncols / 2), full_leader);
+              if (j < nk) ptx::tma_load_2d_pair(sa + j * sub + BM * BK * 2, &p.tmB[tc.rank], (kb + j) * BK, tc.jn * kPairBN + cta_rank * (ncols / 2), full_leader);
           }
-          if (fused) ptx::tma_load_2d_pair(sa + kPairStageBytes, &p.tmBn[tc.rank], kb * BK, (tc.jn + 1) * kPairBN + cta_rank * (ncols1 / 2), full_leader);
+          if (fused) {
+#pragma unroll
+            for (int j = 0; j < kbs; ++j)
+              if (j < nk) ptx::tma_load_2d_pair(sa + j * sub + kPairStageBytes, &p.tmBn[tc.rank], (kb + j) * BK, (tc.jn + 1) * kPairBN + cta_rank * (ncols1 / 2), full_leader);
+          }
           if (++stage == p.n_stages) { stage = 0; phase ^= 1; }
         }
         if (!ok) break;
@@ -916,27 +925,26 @@ __global__ void __launch_bounds__(CONSUMER ? kGemmThreadsFused : kGemmThreads, 1
         const uint64_t b_kstep = p.b_mn ? (uint64_t)(2 * 1024 >> 4) : 2u;
         bool ok = true;
         constexpr int kbs = KBS;
-        for (int kb = 0; kb < p.kblocks; kb += kbs) {
-          const int nk = min(kbs, p.kblocks - kb);
+        for (int kb = 0, nk; kb < p.kblocks; kb += nk) {
+          nk = min((kbs == 2 && p.half_stage && stage == p.n_stages - 1) ? 1 : kbs, p.kblocks - kb);
           if (!mbar_wait(ptx::smem_u32(&ctrl->full[stage]), phase, p, ctrl, tile)) { ok = false; break; }
           ptx::tc_fence_after();
           const uint32_t sa = ptx::smem_u32(payload + stage * p.stage_bytes);
 #pragma unroll
           for (int j = 0; j < kbs; ++j) {
             if (j >= nk) break;
-            const uint32_t sj = sa + j * kPairStageBytes;
+            const uint32_t sj = sa + j * (uint32_t)p.sub_bytes;
             const uint64_t adesc = ptx::smem_desc_k_sw128(sj);
             const uint64_t bdesc = p.b_mn ? ptx::smem_desc_mn_sw128(sj + BM * BK * 2, kMnBlockBytes) : ptx::smem_desc_k_sw128(sj + BM * BK * 2);
 #pragma unroll
             for (int k = 0; k < BK / UMMA_K; ++k)
               ptx::mma_f16_ss_pair(d_tmem, adesc + (uint64_t)(k * 2), bdesc + (uint64_t)k * b_kstep, idesc, (kb | j | k) != 0);
-          }
-          if (fused) {   // the remainder tile (one k-block per stage here): same A stage, its own B rows, the other accumulator
-            const uint64_t adesc = ptx::smem_desc_k_sw128(sa);
-            const uint64_t b1desc = ptx::smem_desc_k_sw128(sa + kPairStageBytes);
+            if (fused) {   // the remainder tile: same A sub-stage, its own B rows, the other accumulator
+              const uint64_t b1desc = ptx::smem_desc_k_sw128(sj + kPairStageBytes);
 #pragma unroll
-            for (int k = 0; k < BK / UMMA_K; ++k)
-              ptx::mma_f16_ss_pair(d_tmem1, adesc + (uint64_t)(k * 2), b1desc + (uint64_t)(k * 2), idesc1, (kb | k) != 0);
+              for (int k = 0; k < BK / UMMA_K; ++k)
+                ptx::mma_f16_ss_pair(d_tmem1, adesc + (uint64_t)(k * 2), b1desc + (uint64_t)(k * 2), idesc1, (kb | j | k) != 0);
+            }
           }
           ptx::mma_commit_pair(ptx::smem_u32(&ctrl->empty[stage]), 3);  // both CTAs may refill this stage
           if (++stage == p.n_stages) { stage = 0; phase ^= 1; }
@@ -1453,16 +1461,24 @@ static int build_plan(const iris_gemm_args* a, const PlanEnv& env, Plan& out) {
     const int pairs_guess = std::max(1, (a->max_ctas ? std::min(a->max_ctas, env.sm_count) : env.sm_count) / 2);
     if (units < 3 * (int64_t)pairs_guess) p.fuse_last = 0;
   }
-  // Operand stages of the pair kernel: two 64-wide k-blocks per stage (3 stages of 64 KB) unless the caller asks for
-  // one (6 of 32 KB) or the stage also carries a fused remainder's B rows (one k-block, 5 or 4 stages).
-  p.kb_per_stage = (p.fuse_last || a->stage_k == 64) ? 1 : 2;
-  p.stage_bytes = p.kb_per_stage * kPairStageBytes;
+  // Operand stages of the pair kernel: two 64-wide k-blocks per stage (3 stages of 64 KB; with a fused remainder of up to
+  // 96 columns two stages and a one-k-block stage, e.g. 72 + 72 + 36 KB) unless the caller asks for one (6 of 32 KB) or
+  // the fused remainder's B rows leave no room for five k-blocks (then one k-block per stage, 4 stages).
+  p.kb_per_stage = a->stage_k == 64 ? 1 : 2;
+  p.sub_bytes = kPairStageBytes;
   if (p.fuse_last) {
     const int rem32 = ((nl % kPairBN) + 31) & ~31;
     p.b1_bytes = (rem32 / 2) * BK * 2;
-    p.stage_bytes = kPairStageBytes + (int)align_up((uint64_t)p.b1_bytes, 1024);
+    p.sub_bytes = kPairStageBytes + (int)align_up((uint64_t)p.b1_bytes, 1024);
   }
+  // Two k-blocks per stage need five k-blocks' worth of ring to pay (measured: with room for two such stages only, the
+  // 448-column shard runs 9-13 % slower than with four or five one-k-block stages); unless the caller insists, fall back.
+  if (p.kb_per_stage == 2 && a->stage_k == 0 && kPairRingBytes < 5 * p.sub_bytes) p.kb_per_stage = 1;
+  p.stage_bytes = p.kb_per_stage * p.sub_bytes;
   p.n_stages = std::min(kPairMaxStages, kPairRingBytes / p.stage_bytes);
+  // what is left of the ring after the two-k-block stages holds one more k-block (remainders up to 96 columns: 72 + 72 + 36 KB)
+  p.half_stage = (p.kb_per_stage == 2 && p.n_stages < kPairMaxStages && kPairRingBytes - p.n_stages * p.stage_bytes >= p.sub_bytes) ? 1 : 0;
+  p.n_stages += p.half_stage;
   p.tab = env.tab;
   p.c_off = a->c_off;
   p.flag_off = a->flag_off;

@@ -175,13 +175,16 @@ RAGGED_PAIR_SHAPES = [
     (2, 512, 320, 128),      # 256 + 64
     (8, 2048, 288, 64),      # 256 + 32: the narrowest remainder an MMA group can have
     (2, 700, 504, 72),       # 256 + 248: remainder rounded up to a full 256-wide group
+    (2, 512, 320, 1096),     # 256 + 64, 18 k-blocks (the last one 8 wide): the 2 + 2 + 1 k-block ring goes round several times
+    (4, 520, 352, 840),      # 256 + 96: the widest remainder that still gets two k-blocks per stage by default
 ]
 
 
-@pytest.mark.parametrize("kw", [dict(), dict(fuse_tail=1), dict(fuse_tail=-1), dict(fuse_tail=-1, stage_k=64), dict(fuse_tail=1, max_ctas=6, comm_ctas=2),
+@pytest.mark.parametrize("kw", [dict(), dict(fuse_tail=1), dict(fuse_tail=-1), dict(fuse_tail=-1, stage_k=64), dict(fuse_tail=1, stage_k=64), dict(fuse_tail=1, stage_k=128),
+                                dict(fuse_tail=1, max_ctas=6, comm_ctas=2),
                                 dict(fuse_tail=1, static_schedule=1, raster_group=1), dict(fuse_tail=1, wg_tail=0),
                                 dict(fuse_tail=1, wg_tail=0, comm_ctas=2, max_ctas=12)],
-                         ids=["default", "fused", "separate_tail_tile", "separate_tail_tile_k64", "small_grid", "static", "tail_rule", "takeover"])
+                         ids=["default", "fused", "separate_tail_tile", "separate_tail_tile_k64", "fused_k64", "fused_k128", "small_grid", "static", "tail_rule", "takeover"])
 @pytest.mark.parametrize("mode", MODES, ids=MODE_IDS)
 @pytest.mark.parametrize("W,M,nl,K", RAGGED_PAIR_SHAPES)
 def test_ragged_shard_remainder_fused_with_last_full_tile(mode, W, M, nl, K, kw):
