@@ -472,16 +472,14 @@ def run_ours(args):
                     epoch += 1
                     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                     torch.cuda.synchronize()
-                    gpu_gate(torch)
+                    # (no busy kernel in front here: two streams released by one event start in no fixed order, and a consumer
+                    # that becomes resident first keeps the GEMM's CTAs off the SMs; 20 us of host time in 4 ms do not matter)
                     e0.record(stream)
-                    if overlapped:
-                        # the consumer must not become resident before the producer does (it would hold the SMs' registers
-                        # while it waits for flags): its stream starts behind the same busy kernel as the producer's
-                        cons_stream.wait_event(e0)
                     gemm(epoch)
                     if overlapped:
-                        # 3 CTAs per SM: a GEMM CTA still fits beside them (threads, registers) should the consumer become resident first
-                        iris.iris_consume_bias(h, 0, out_off, flag_off, dbias, M, N, W, dt, epoch, ctas=3 * sm_count, stream=cons_stream)
+                        # launched after the producer, whose CTAs are all resident by then; beside a GEMM CTA of the pair kernel
+                        # one consumer CTA fits per SM (shared memory), the rest of the grid follows as the GEMM's CTAs leave
+                        iris.iris_consume_bias(h, 0, out_off, flag_off, dbias, M, N, W, dt, epoch, ctas=4 * sm_count, stream=cons_stream)
                         joined.record(cons_stream)
                         stream.wait_event(joined)
                     else:

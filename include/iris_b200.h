@@ -378,13 +378,16 @@ int64_t iris_num_tiles(int M, int N, int world);
  * of `dtype`, broadcast over rows; the sum is formed in fp32 and rounded once.  OUT is a second
  * row-major [M, N] region at out_off in every slot.  ctas: grid size (0 = 8 per SM).
  * On a stream of its own the consumer may be launched while its producer is still running (that is the point of
- * the flags).  Launch it after every kernel that publishes the flags it waits for has been launched.  Its CTAs leave
- * only once their tiles are published, so a publisher that finds no room on the SMs they occupy would never run and
- * the wait would end by its deadline (IRIS_ERR_TIMEOUT), not by making progress: the default grid fills every SM's
- * thread slots, and four CTAs per SM still hold too many registers for a GEMM CTA of this library to fit beside
- * them.  Whenever a publishing kernel may become resident after the consumer (the second kernel of bulk_synchronous
- * mode starts when the GEMM ends; two streams released by the same event start in no fixed order) pass
- * ctas <= 3 per SM: that leaves threads, registers and all shared memory for one CTA of any kernel here. */
+ * the flags).  Launch it AFTER every kernel that publishes the flags it waits for has been launched: those kernels are
+ * persistent, all their CTAs are resident from the start, and the consumer's CTAs then fill whatever the SMs have left
+ * (beside a GEMM CTA, which takes all but 1 KB of an SM's shared memory, that is one consumer CTA per SM; the rest of
+ * the grid follows as the GEMM's CTAs leave).  The other order is not supported.  A consumer CTA leaves only once its
+ * tiles are published, every resident CTA reserves 1 KB of shared memory, and a GEMM CTA that arrives later fits only
+ * on an SM holding at most one of them (the single-CTA workgroup-specialised kernel, a cooperative launch, did not
+ * start at all behind a waiting consumer of 64 CTAs).  A publisher that finds no room never runs, and the wait ends by
+ * its deadline (IRIS_ERR_TIMEOUT), not by making progress.  The same holds when a publishing kernel can only start
+ * later (the second kernel of bulk_synchronous mode starts when the GEMM ends) or when two streams are released by
+ * the same event and start in no fixed order: keep the consumer off the device until the publishers are running. */
 int iris_consume_bias(iris_heap* heap, uint64_t c_off, uint64_t out_off, uint64_t flag_off, const void* bias, int M,
                       int N, int world, int dtype, int32_t epoch, int ctas, uint64_t timeout_ns, void* stream);
 /* The same for the publication tiles of ranks [rank_first, rank_first + rank_count) only (the column

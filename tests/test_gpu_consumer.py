@@ -171,3 +171,4 @@ def test_consumer_arguments_are_checked():
             assert e.value.code == code, (out, e.value)
         torch.cuda.synchronize()
         assert bool(torch.all(g.mem == SENTINEL))
+
