@@ -156,3 +156,17 @@ def test_config5_sweep_members_sampled_tiles(W, M):
     """The other members of the W x M sweep on N = K = 16384 (bench.py times them in all schedules; here the
     workgroup-specialised one, 48 random tiles plus the corner tiles of the output)."""
     _run_fullsize(W, M, 16384, 16384, "uniform", "bf16", "workgroup_specialized", inputs.SEED0 + 4, n_random=48)
+
+
+@pytest.mark.parametrize("mode", ["fused_sequential", "workgroup_specialized", "bulk_synchronous"])
+@pytest.mark.parametrize("N,K", [(3584, 14336), (4608, 36864)], ids=["8192x3584x14336", "8192x4608x36864"])
+def test_paper_shapes_with_global_n_ragged_shards(N, K, mode):
+    """The two shapes Section 5.2 names, read with N global (W=8, M=8192, bf16 normal(0, 0.02)): shards of 448 = 256 + 192
+    and 576 = 2 x 256 + 64 columns, so every shard ends in a fused unit (and, for 576, on the ring of two two-k-block
+    stages and one one-k-block stage) and in a narrow publication tile.  24 random tiles plus the corner tiles."""
+    _run_fullsize(8, 8192, N, K, "normal002", "bf16", mode, inputs.SEED0 + 6, n_random=24)
+
+
+def test_paper_shape_with_n_per_rank():
+    """8192 x (8 x 3584) x 14336, the same shape read with N per rank (bench.py's sweep times it): 16 random tiles."""
+    _run_fullsize(8, 8192, 8 * 3584, 14336, "normal002", "bf16", "workgroup_specialized", inputs.SEED0 + 7, n_random=16)
