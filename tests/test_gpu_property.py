@@ -72,3 +72,98 @@ def test_any_small_problem_leaves_the_oracles_heap_image(problem):
             host = g.to_host()
             img, c_full = expected_image(g, A, Bs, dtype, mode, epoch=epoch, c_full=c_full)
             assert np.array_equal(host, img.mem), (problem, epoch, first_diff(host, img.mem))
+
+
+# ------------------------------------------------------------------------------------------------
+# Table 3 on random arguments: a sequence of put / get / copy / atomic operations with arbitrary (legal) sizes, pitches,
+# alignments and rank triples, applied to the GPU heap and to the oracle's image; the two must agree byte for byte after
+# the whole sequence (any misplaced, missing or extra byte shows), and the atomics' returned old values must agree too.
+# ------------------------------------------------------------------------------------------------
+BPR = 1 << 16
+
+
+@st.composite
+def region_op(draw, W):
+    kind = draw(st.sampled_from(["put", "get", "copy"]))
+    vec = draw(st.booleans())                       # 16-byte aligned everything (vector path) or arbitrary (byte path)
+    unit = 16 if vec else 1
+    rows = draw(st.integers(1, 40))
+    row_bytes = unit * draw(st.integers(1, 600 // unit if vec else 300))
+    sp = row_bytes + unit * draw(st.integers(0, 8))
+    dp = row_bytes + unit * draw(st.integers(0, 8))
+    span_s, span_d = (rows - 1) * sp + row_bytes, (rows - 1) * dp + row_bytes
+    so = unit * draw(st.integers(0, (BPR - span_s) // unit))
+    do = unit * draw(st.integers(0, (BPR - span_d) // unit))
+    ranks = [draw(st.integers(0, W - 1)) for _ in range(3)]
+    return kind, rows, row_bytes, sp, dp, so, do, ranks
+
+
+@st.composite
+def atomic_op(draw, W):
+    op = draw(st.sampled_from(["add", "xchg", "and", "or", "xor", "min", "max", "cas", "add64", "cas64"]))
+    wide = op.endswith("64")
+    word = 8 if wide else 4
+    count = draw(st.integers(1, 300))
+    stride = word * draw(st.integers(1, 5))
+    off = word * draw(st.integers(0, (BPR - ((count - 1) * stride + word)) // word))
+    frm, to = draw(st.integers(0, W - 1)), draw(st.integers(0, W - 1))
+    val = draw(st.integers(0, (1 << 64) - 1) if wide else st.integers(-(1 << 31), (1 << 31) - 1))
+    cmp_ = draw(st.integers(0, 3))
+    return op, count, stride, off, frm, to, val, cmp_
+
+
+@st.composite
+def op_sequences(draw):
+    W = draw(st.integers(1, 5))
+    n = draw(st.integers(1, 8))
+    ops = [draw(st.one_of(region_op(W), atomic_op(W))) for _ in range(n)]
+    return W, ops, draw(st.integers(0, 1 << 20))
+
+
+@settings(max_examples=int(os.environ.get("IRIS_PROPERTY_EXAMPLES", "150")), deadline=None, derandomize=True, suppress_health_check=list(HealthCheck))
+@given(op_sequences())
+def test_any_sequence_of_tile_operations_and_atomics_matches_the_oracle(case):
+    import torch
+    W, ops, seed = case
+    with GpuHeap(W, BPR) as g:
+        img = g.image()
+        img.mem[:] = inputs.payload_bytes(seed, 7, img.mem.size)
+        # a sprinkling of small values so that cas (compare with 0..3) and min/max take both branches
+        img.mem[::97] = 0
+        g.mem.copy_(torch.from_numpy(img.mem).cuda())
+        for op in ops:
+            if op[0] in ("put", "get", "copy"):
+                kind, rows, rb, sp, dp, so, do, (a, b, c) = op
+                overlap = so < do + (rows - 1) * dp + rb and do < so + (rows - 1) * sp + rb
+                # source and destination overlapping in one slot: the order of the bytes is unspecified
+                if overlap and ((kind in ("put", "get") and a == b) or (kind == "copy" and b == c)):
+                    continue
+                if kind == "put":
+                    iris.iris_put_tile(g.h, g.addr(a, so), g.addr(a, do), rows, rb, sp, dp, a, b)
+                    img.put(so, do, rows, rb, sp, dp, a, b)
+                elif kind == "get":
+                    iris.iris_get_tile(g.h, g.addr(a, so), g.addr(a, do), rows, rb, sp, dp, a, b)
+                    img.get(so, do, rows, rb, sp, dp, a, b)
+                else:
+                    iris.iris_copy_tile(g.h, g.addr(a, so), g.addr(a, do), rows, rb, sp, dp, a, b, c)
+                    img.copy(so, do, rows, rb, sp, dp, b, c)
+                continue
+            name, count, stride, off, frm, to, val, cmp_ = op
+            wide = name.endswith("64")
+            old = torch.empty(count, dtype=torch.int64 if wide else torch.int32, device="cuda")
+            ptr = g.addr(frm, off)
+            if name == "add64":
+                iris.iris_atomic_add_u64(g.h, ptr, count, stride, frm, to, val, old_out=old)
+                exp = img.atomic_add_u64(off, count, stride, to, val)
+            elif name == "cas64":
+                iris.iris_atomic_cas_u64(g.h, ptr, count, stride, frm, to, cmp_, val, old_out=old)
+                exp = img.atomic_cas_u64(off, count, stride, to, cmp_, val)
+            elif name == "cas":
+                iris.iris_atomic_cas(g.h, ptr, count, stride, frm, to, cmp_, val, old_out=old)
+                exp = img.atomic_cas(off, count, stride, to, cmp_, val)
+            else:
+                iris.iris_atomic_rmw(g.h, iris.ATOMIC_OPS[name], ptr, count, stride, frm, to, val, old_out=old)
+                exp = img.atomic_rmw(name, off, count, stride, to, val)
+            got = old.cpu().numpy()
+            assert np.array_equal(got.view(exp.dtype), exp), (op, "returned old values differ")
+        assert np.array_equal(g.to_host(), img.mem), (case, first_diff(g.to_host(), img.mem))
