@@ -14,7 +14,7 @@ from hypothesis import strategies as st
 
 import paper_2511_12500_b200 as iris
 from paper_2511_12500_b200 import inputs
-from gpu_util import GpuHeap, first_diff, gemm_layout
+from gpu_util import GpuHeap, dev16, first_diff, gemm_layout
 from test_gpu_gemm_all_scatter import expected_image, run_gemm
 
 pytestmark = pytest.mark.gpu
@@ -72,6 +72,14 @@ def test_any_small_problem_leaves_the_oracles_heap_image(problem):
             host = g.to_host()
             img, c_full = expected_image(g, A, Bs, dtype, mode, epoch=epoch, c_full=c_full)
             assert np.array_equal(host, img.mem), (problem, epoch, first_diff(host, img.mem))
+        # ... and the flag-gated consumer on top of it: OUT = C + bias in every slot, nothing else touched
+        bias = inputs.matrix(seed, inputs.STREAM_BIAS, 1, N, "smallint:2", dtype).reshape(-1)
+        c_off, flag_off, _, out_off, _ = gemm_layout(M, N, W, True)
+        iris.iris_consume_bias(g.h, c_off, out_off, flag_off, dev16(bias), M, N, W, iris.DTYPES[dtype], 2)
+        iris.iris_status_check(g.h)
+        img.consume_bias(dtype, c_off, out_off, M, N, bias)
+        host = g.to_host()
+        assert np.array_equal(host, img.mem), (problem, "consumer", first_diff(host, img.mem))
 
 
 # ------------------------------------------------------------------------------------------------
