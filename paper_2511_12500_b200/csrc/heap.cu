@@ -117,6 +117,14 @@ int iris_heap_create_from_bases(int world, size_t bytes_per_rank, const uint64_t
   cudaDeviceProp prop;
   IRIS_CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
   if (prop.major != 10) return fail(IRIS_ERR_UNSUPPORTED, "iris_heap_create_from_bases: device is sm_%d%d, this library is sm_100a only", prop.major, prop.minor);
+  for (int r = 0; r < world; ++r) {   // every slot must be device memory this process can address (its own or a mapped peer's)
+    cudaPointerAttributes pa;
+    const cudaError_t e = cudaPointerGetAttributes(&pa, reinterpret_cast<const void*>(bases[r]));
+    if (e != cudaSuccess || (pa.type != cudaMemoryTypeDevice && pa.type != cudaMemoryTypeManaged)) {
+      cudaGetLastError();
+      return fail(IRIS_ERR_ARG, "iris_heap_create_from_bases: base of slot %d is not device memory known to this process", r);
+    }
+  }
   iris_heap* h = new iris_heap();
   std::memset(h, 0, sizeof(*h));
   h->world = world;

@@ -71,6 +71,7 @@ def test_heap_from_bases_rejects_bad_tables():
     for bases, local, bpr in (([b, b + 2048], 0, 4096),        # overlap
                               ([b, b + 4096 + 8], 0, 4096),    # misaligned
                               ([b, 0], 0, 4096),               # missing
+                              ([b, 1 << 20], 0, 4096),         # not memory of this process
                               ([b, b + 4096], 2, 4096),        # local rank outside the world
                               ([b, b + 4096], 0, 100)):        # slot size
         with pytest.raises(iris.IrisError) as e:
