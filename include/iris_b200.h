@@ -94,8 +94,9 @@ int iris_heap_create_ex(int world, size_t bytes_per_rank, void* external_base, i
 /* A heap over several processes or devices (Section 3.1: one slot per rank, each in its owner's memory; Section 3.2
  * steps 3-6: allocate, exchange handles, open the peers' slots, build the table of bases).  bases[0..world) are HOST
  * values: the device address, in THIS process, of every rank's slot of bytes_per_rank bytes, each 256-byte aligned,
- * none overlapping another, each device memory this process can address (IRIS_ERR_ARG otherwise); bases[local_rank] is this process's own allocation, the others are mappings of the
- * peers' (iris_ipc_open, or any mapping the caller made).  The heap owns none of them and the caller keeps them
+ * none overlapping another, each device memory this process can address (IRIS_ERR_ARG otherwise);
+ * bases[local_rank] is this process's own allocation, the others are mappings of the peers' (iris_ipc_open, or any
+ * mapping the caller made).  The heap owns none of them and the caller keeps them
  * alive until iris_heap_destroy.  Nothing is cleared.  What changes on such a heap:
  *   - ready flags are released and acquired at SYSTEM scope (every other scope in this header stays as written);
  *   - iris_gemm_all_scatter_ex / _unfused compute this rank's shard only: rank_first must be local_rank and
