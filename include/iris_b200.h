@@ -459,9 +459,11 @@ int iris_gemm_takeover_stats(const iris_heap* heap, int32_t out[2]);
  * calls whose GPU work overlaps (different streams, different host threads) race on it and must be
  * serialised by the caller.
  * Other arguments, checks, layout and results are those of iris_gemm_all_scatter_ex in
- * IRIS_MODE_WORKGROUP_SPECIALIZED with single-CTA tiles (cta_pair = -1) and default tuning: the
- * launch plan (tile width, grid split, which tiles the producers scatter themselves) is built by
- * the same code, and the results are bit-identical to that call's. */
+ * IRIS_MODE_WORKGROUP_SPECIALIZED with default tuning: the launch plan (CTA-pair or single-CTA
+ * tiles, tile width, grid split, which tiles the producers scatter themselves) is built by the
+ * same code and the same kernels run -- with the locks and the work-unit counter in the static
+ * array and, the slots being wherever the caller says, one store map per slot -- so the results
+ * are bit-identical to that call's. */
 int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, const uint64_t* slot_bases,
                                   size_t bytes_per_rank, int M, int N, int K, int world, int dtype, uint64_t c_off,
                                   uint64_t flag_off, int32_t epoch, void* stream);

@@ -2079,14 +2079,14 @@ int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, co
   // The array keeps the previous call's contents: the status block and the locks in use must start at zero.
   IRIS_CUDA_TRY(cudaMemsetAsync(scratch, 0, (size_t)(kNoAllocStatusWords + nt) * 4, st));
 
-  // The plan is the one iris_gemm_all_scatter_ex builds for workgroup_specialized with single-CTA tiles and default
-  // tuning (same function), with the slots at the caller's addresses and the locks and status block in the scratch.
+  // The plan is the one iris_gemm_all_scatter_ex builds for workgroup_specialized with default tuning (same function:
+  // CTA-pair tiles where the shape allows them, single-CTA tiles otherwise), with the slots at the caller's addresses
+  // (one store map per slot) and the locks, the work-unit counter and the status block in the scratch.
   iris_gemm_args a;
   std::memset(&a, 0, sizeof(a));
   a.A = A; a.B_shards = B_shards;
   a.M = M; a.N = N; a.K = K; a.world = world; a.mode = IRIS_MODE_WORKGROUP_SPECIALIZED; a.dtype = dtype;
   a.c_off = c_off; a.flag_off = flag_off; a.epoch = epoch;
-  a.cta_pair = -1;
   PlanEnv env{};
   for (int r = 0; r < world; ++r) env.tab.base[r] = slot_bases[r];
   env.tab.bytes_per_rank = bytes_per_rank;
@@ -2095,13 +2095,19 @@ int iris_gemm_all_scatter_noalloc(const void* A, const void* const* B_shards, co
   env.bpr = bytes_per_rank;
   env.sm_count = sms;
   env.status = scratch;
+  env.pair_any_base = true;
   Plan pl;
   int rc = build_plan(&a, env, pl);
   if (rc != IRIS_OK) return rc;
-  if (pl.pair || pl.streamk) return fail(IRIS_ERR_STATE, "gemm_all_scatter_noalloc: unexpected plan");
+  if (pl.streamk) return fail(IRIS_ERR_STATE, "gemm_all_scatter_noalloc: unexpected plan");
   pl.p.epoch = epoch;
   const bool bf = dtype == IRIS_BF16;
-  if (pl.bn == 256) rc = bf ? launch_gemm<256, true, true>(pl.p, pl.grid, true, st) : launch_gemm<256, false, true>(pl.p, pl.grid, true, st);
+  if (pl.pair) {
+    pl.p.dynamic = 1;
+    pl.p.tile_counter = scratch + 16;   // spare words of the scratch's status block, zeroed above with the rest
+    pl.p.backlog = scratch + 17;
+    rc = bf ? launch_gemm_pair<true, true>(pl.p, pl.grid, st, nullptr) : launch_gemm_pair<false, true>(pl.p, pl.grid, st, nullptr);
+  } else if (pl.bn == 256) rc = bf ? launch_gemm<256, true, true>(pl.p, pl.grid, true, st) : launch_gemm<256, false, true>(pl.p, pl.grid, true, st);
   else              rc = bf ? launch_gemm<128, true, true>(pl.p, pl.grid, true, st) : launch_gemm<128, false, true>(pl.p, pl.grid, true, st);
   if (rc != IRIS_OK) return rc;
   // the status words come back on the caller's stream (no other stream is touched), then one wait for that stream

@@ -5,8 +5,8 @@ already handed out to a framework's pool, a loop that cannot take the synchronis
 it takes raw slot addresses instead of a heap handle and keeps its locks and status block in a fixed array
 inside the library.  That array is shared by all calls and keeps its old contents, so the test calls it twice
 in a row, with different inputs, and compares every byte of C and every flag in every slot with what
-iris_gemm_all_scatter_ex (workgroup-specialised, single-CTA tiles) produced for the same inputs.  Both paths run
-the same main loop, so the comparison is bit-exact, which is tighter than the tolerance the other GPU tests use.
+iris_gemm_all_scatter_ex (workgroup-specialised, default tuning) produced for the same inputs.  Both paths build
+their plan with the same code and run the same kernels, so the comparison is bit-exact, which is tighter than the tolerance the other GPU tests use.
 
 This file is named so that pytest collects it last.
 """
@@ -29,17 +29,19 @@ def _reference_run(W, M, N, K, dtype, A, Bs, epoch):
     with GpuHeap(W, bpr) as g:
         iris.iris_flags_fill(g.h, lock_off, nt, 0)
         iris.iris_gemm_all_scatter_ex(g.h, dev16(A), [dev16(b) for b in Bs], M, N, K, W, iris.IRIS_MODE_WORKGROUP_SPECIALIZED,
-                                      iris.DTYPES[dtype], c_off, flag_off, lock_off, epoch, cta_pair=-1)
+                                      iris.DTYPES[dtype], c_off, flag_off, lock_off, epoch)
         iris.iris_status_check(g.h)
         host = g.to_host().reshape(W, bpr)
         return (host[:, c_off:c_off + M * N * 2].copy(), host[:, flag_off:flag_off + nt * 4].copy())
 
 
 @pytest.mark.parametrize("W,M,nl,K,dtype", [
-    (4, 520, 392, 328, "bf16"),      # 128-wide compute tiles; several tiles, ragged in M, N_local and K
-    (8, 640, 512, 192, "fp16"),      # N_local a multiple of 256 and more tiles than SMs: the 256-wide kernel, five tile rows
-    (2, 900, 1280, 136, "bf16"),     # 256-wide kernel (160 narrow tiles would not fit one wave), ragged M and K
-], ids=["bn128_bf16", "bn256_fp16", "bn256_bf16_ragged"])
+    (4, 128, 392, 328, "bf16"),      # single-CTA kernel, 128-wide compute tiles; ragged in N_local and K
+    (8, 100, 512, 192, "fp16"),      # single-CTA kernel (one tile row), N_local a multiple of 256
+    (4, 520, 392, 328, "bf16"),      # CTA-pair kernel, ragged in M, N_local (256 + 136: a fused unit) and K
+    (8, 640, 512, 192, "fp16"),      # CTA-pair kernel, more units than pairs
+    (2, 900, 1280, 136, "bf16"),     # CTA-pair kernel, five units per shard, ragged M and K
+], ids=["single_bn128_bf16", "single_fp16", "pair_ragged_bf16", "pair_fp16", "pair_bf16_wide"])
 def test_noalloc_matches_regular_entry_point_twice_in_a_row(W, M, nl, K, dtype):
     N = W * nl
     c_off, flag_off, _, _, bpr = gemm_layout(M, N, W)
